@@ -1,0 +1,246 @@
+/*
+ * csd.h -- C ABI of the verification-and-rescue step of Calibrated Speculative
+ * Decoding (CSD) for NVIDIA B200 (sm_100a).
+ *
+ * One step takes the target model's logits for the gamma drafted positions plus
+ * the bonus position, the gamma draft tokens, the Online Correction Memory (OCM)
+ * and the gate threshold tau, and returns the number of accepted draft tokens,
+ * the token to emit after them, and the rejections to feed back to the memory:
+ * the verification loop of Algorithm 1 in its greedy (T = 0) form, the mode of
+ * the paper's evaluation (Sec. 5.1).
+ *
+ * Notation: B batch rows, K = gamma draft tokens per row, V vocabulary size,
+ * z[b,i,v] target logits, d[b,i] draft token, t[b,i] = argmax_v z[b,i,v]
+ * (lowest index on ties), m[b,i] = z[b,i,t].
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless the
+ *     argument is documented as a host pointer.  The library owns only the
+ *     memory behind a csd_ocm_t.
+ *   - All work is enqueued on the CUDA stream passed as `stream` (a cudaStream_t
+ *     cast to void*; NULL is the legacy default stream).  Nothing synchronises
+ *     unless documented.  Calls on one csd_ocm_t must be stream-ordered.
+ *   - Every function returns a csd_status_t and never throws or aborts.  Misuse
+ *     that the host can see is refused before anything is launched.  Conditions
+ *     only the device can see (a NaN logit, a draft id outside [0,V), a full
+ *     table) set sticky flags / counters readable with csd_ocm_stats; the device
+ *     never traps and never waits on another block.
+ *   - Determinism: for fixed (B,K,V,dtype) every output, including the sums s,
+ *     is bit-reproducible from run to run.
+ */
+#ifndef CSD_H_
+#define CSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct csd_ocm csd_ocm_t;
+
+typedef enum {
+    CSD_OK = 0,
+    CSD_ERR_INVALID_ARG = 1,
+    CSD_ERR_CUDA = 2,
+    CSD_ERR_OOM = 3,
+    CSD_ERR_UNSUPPORTED = 4,
+    CSD_ERR_WORKSPACE = 5
+} csd_status_t;
+
+typedef enum { CSD_F32 = 0, CSD_BF16 = 1 } csd_dtype_t;
+
+/* Largest K (draft tokens per row) a step accepts: one warp lane per position. */
+#define CSD_MAX_K 32
+
+/* sticky device flags reported in csd_stats_t.flags */
+#define CSD_FLAG_NAN_LOGIT      0x1u  /* a row's sum came out NaN (NaN / +inf logit, or a row of -inf) */
+#define CSD_FLAG_BAD_DRAFT      0x2u  /* a draft id outside [0, V) was seen                            */
+#define CSD_FLAG_PROBE_EXHAUSTED 0x4u /* a hash probe visited every slot (cannot happen below capacity) */
+#define CSD_FLAG_COUNT_SATURATED 0x8u /* a count reached 2^32 - 1                                      */
+
+/* Optional per-position diagnostics.  Any member may be NULL.  Row arrays have
+ * B*(K+1) entries, position arrays B*K, both row-major.  Values are defined for
+ * every position, also past a row's first un-rescued rejection. */
+typedef struct {
+    float   *m;      /* [B,K+1] max logit                                                  */
+    float   *s;      /* [B,K+1] sum_v exp(z_v - m): the soft-max normaliser of Eq. 3      */
+    float   *lse;    /* [B,K+1] m + ln s                                                   */
+    int32_t *t;      /* [B,K+1] argmax, lowest index on ties (t* of Algorithm 1 at T = 0) */
+    float   *zd;     /* [B,K]   z[b,i,d[b,i]]   (NaN if d is outside [0,V))                */
+    float   *score;  /* [B,K]   exp(zd - m) = p(d)/p(t*), the Score of Fig. 1 / Eq. 3      */
+    float   *p_d;    /* [B,K]   soft-max probability of the draft token                    */
+    float   *p_t;    /* [B,K]   soft-max probability of t*                                 */
+    uint32_t *cnt;   /* [B,K]   OCM count of (d, t*) at the start of the step (0 = absent) */
+} csd_diag_t;
+
+typedef struct {
+    uint64_t n_slots;       /* capacity in slots (power of two)                      */
+    uint64_t key_limit;     /* most distinct pairs the table admits (= n_slots / 2)  */
+    uint64_t n_keys;        /* distinct pairs stored                                 */
+    uint64_t n_dropped;     /* update occurrences dropped because the table was full */
+    uint64_t steps;         /* csd_verify / csd_step calls                           */
+    uint64_t positions;     /* draft positions verified (B*K per step)               */
+    uint64_t matches;       /* reached positions with d == t*                        */
+    uint64_t rescues;       /* reached mismatches accepted through OCM + SCG         */
+    uint64_t rejections;    /* pairs handed to the memory update                     */
+    uint32_t lambda;        /* frequency threshold in force                          */
+    uint32_t flags;         /* CSD_FLAG_* (sticky until csd_ocm_reset)               */
+} csd_stats_t;
+
+/* ---- Online Correction Memory (Sec. 4.2): frequency table of ordered pairs ----
+ *
+ * The table T of Algorithm 1: (draft token, target token) -> count, an
+ * open-addressed hash table in device memory (16-byte slots, linear probing).
+ * The paper fixes no capacity rule; this library's rule is: at most n_slots/2
+ * distinct pairs; a pair already present always counts; a new pair is admitted,
+ * in the canonical order of the update (index order), only while fewer than
+ * n_slots/2 pairs are stored, else that occurrence is dropped and counted in
+ * n_dropped; nothing is evicted.  Counts are 32-bit and saturate.
+ */
+
+/* Allocate an empty table on `device` (cudaSetDevice is called and left set).
+ * n_slots: power of two, >= 64.  lambda: frequency threshold of the candidate
+ * proposal test T[(d,t*)] >= lambda (the paper's main protocol uses 6; 0 makes
+ * every divergence a candidate).  Synchronises the device once.
+ * Errors: INVALID_ARG (null out, bad n_slots), OOM, CUDA. */
+csd_status_t csd_ocm_create(csd_ocm_t **out, uint64_t n_slots, uint32_t lambda, int device);
+
+/* Empty the table and zero its statistics and flags (asynchronous on `stream`). */
+csd_status_t csd_ocm_reset(csd_ocm_t *ocm, void *stream);
+
+/* Free the table.  The caller makes sure no work using it is still running. */
+csd_status_t csd_ocm_destroy(csd_ocm_t *ocm);
+
+/* Change lambda for subsequent calls (host side; stream-ordered like any call). */
+csd_status_t csd_ocm_set_lambda(csd_ocm_t *ocm, uint32_t lambda);
+
+/* ---- one verification step ---------------------------------------------------- */
+
+/* Bytes of scratch csd_verify / csd_step need for this shape (0 on invalid shape).
+ * The scratch holds per-tile partial reductions and arrival counters. */
+size_t csd_workspace_bytes(int B, int K, int V, csd_dtype_t dtype);
+
+/* Zero a workspace.  Required once before its first use (and after any aborted
+ * launch); the kernels leave the counters zeroed again on completion, so the
+ * same workspace can be reused step after step without further clearing.  One
+ * workspace serves one step at a time. */
+csd_status_t csd_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/* The verification loop of Algorithm 1 (greedy) for all B rows, read-only on the
+ * memory.  For each row b and position i < K:
+ *     t* = argmax z[b,i,:]                     (residual resample at T = 0)
+ *     match   = (d[b,i] == t*)                 (acceptance test at T = 0)
+ *     is_freq = T[(d[b,i], t*)] >= lambda      (candidate proposal, Sec. 4.2)
+ *     is_safe = z[b,i,d] - z[b,i,t*] >= ln tau (Eq. 3; decided in double on the
+ *               exact inputs against (float) log((double) tau); equality passes)
+ *     position accepted iff  match or (is_freq and is_safe)
+ * accept_len[b] = number of leading accepted positions (n of Algorithm 1);
+ * next_token[b] = t* of the first non-accepted position, or argmax z[b,K,:] (the
+ * bonus token) when all K are accepted; rescued_mask[b,i] = 1 for non-matching
+ * positions inside the accepted prefix.  rej_draft/rej_target[b,i] hold the pair
+ * (d, t*) for every divergence the loop reaches (rescued ones and the one that
+ * ends the row), -1 elsewhere: exactly the UpdateMemory calls of Algorithm 1.
+ * All look-ups see the table as it is when the call starts.
+ *
+ * logits : [B, K+1, V], element (b,i,v) at  b*stride_b + i*stride_k + v  (strides
+ *          in elements, V contiguous); CSD_F32 or CSD_BF16.  128-bit loads are
+ *          used when the base and both strides are 16-byte multiples, a slower
+ *          element-wise path otherwise.
+ * draft  : [B, K] int32.  An id outside [0,V) is a mismatch that cannot be
+ *          rescued and is not recorded (flag CSD_FLAG_BAD_DRAFT).
+ * tau    : gate threshold, >= 0 and not NaN.  0 disables the gate (memory only);
+ *          tau > 1 can never pass.
+ * accept_len, next_token : [B] int32.   rescued_mask : [B,K] uint8.
+ * rej_draft, rej_target  : [B,K] int32.
+ * diag   : NULL, or a HOST pointer to a struct of optional device arrays.
+ * workspace : >= csd_workspace_bytes(B,K,V,dtype) bytes, 16-byte aligned,
+ *          initialised with csd_workspace_init.
+ * Errors: INVALID_ARG (null pointer, B,K,V <= 0, bad tau or strides),
+ *         UNSUPPORTED (K > CSD_MAX_K), WORKSPACE (too small / misaligned), CUDA.
+ * One kernel launch; asynchronous. */
+csd_status_t csd_verify(const void *logits, csd_dtype_t dtype, int B, int K, int V,
+                        int64_t stride_b, int64_t stride_k,
+                        const int32_t *draft, const csd_ocm_t *ocm, float tau,
+                        int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                        int32_t *rej_draft, int32_t *rej_target,
+                        const csd_diag_t *diag,
+                        void *workspace, size_t workspace_bytes, void *stream);
+
+/* UpdateMemory of Algorithm 1 for a batch of n pairs: count[(rej_draft[j],
+ * rej_target[j])] += 1 for j = 0..n-1 in index order (the order only matters for
+ * admission when the table is nearly full).  Entries with a negative member are
+ * skipped.  Duplicates each count.  n may be any size >= 0.  Asynchronous. */
+csd_status_t csd_ocm_update(csd_ocm_t *ocm, const int32_t *rej_draft, const int32_t *rej_target,
+                            int64_t n, void *stream);
+
+/* csd_verify followed by csd_ocm_update of the step's rejections in (b,i) order,
+ * fused into the same single launch: the online adaptation of Sec. 4.2 (look-up
+ * before update: a pair recorded in this step can reach lambda only for later
+ * steps).  Arguments as csd_verify. */
+csd_status_t csd_step(const void *logits, csd_dtype_t dtype, int B, int K, int V,
+                      int64_t stride_b, int64_t stride_k,
+                      const int32_t *draft, csd_ocm_t *ocm, float tau,
+                      int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                      int32_t *rej_draft, int32_t *rej_target,
+                      const csd_diag_t *diag,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/* csd_step for callers whose tensors live in HOST memory (pinned memory gives
+ * the full copy rate).  Copies logits and draft to `staging`, runs the step, and
+ * copies accept_len, next_token and rescued_mask back; returns after the stream
+ * has been synchronised, so the host outputs are valid on return.
+ * logits_host is dense [B,K+1,V].  staging: DEVICE scratch of at least
+ * csd_host_staging_bytes(B,K,V,dtype) bytes, 256-byte aligned; it needs no
+ * initialisation and may be reused. */
+size_t csd_host_staging_bytes(int B, int K, int V, csd_dtype_t dtype);
+csd_status_t csd_step_host(const void *logits_host, csd_dtype_t dtype, int B, int K, int V,
+                           const int32_t *draft_host, csd_ocm_t *ocm, float tau,
+                           int32_t *accept_len_host, int32_t *next_token_host,
+                           uint8_t *rescued_mask_host,
+                           void *staging, size_t staging_bytes, void *stream);
+
+/* ---- memory life cycle: checkpoint / restore (prior calibration, Sec. 4.2 Phase 1) ---- */
+
+/* Write every stored pair to the DEVICE arrays d, t, cnt (capacity `cap` triples,
+ * order unspecified) and the number of stored pairs to the HOST word *n_out.
+ * Synchronises `stream`.  If more than `cap` pairs are stored only `cap` are
+ * written and *n_out still reports the total. */
+csd_status_t csd_ocm_export(const csd_ocm_t *ocm, int32_t *d, int32_t *t, uint32_t *cnt,
+                            uint64_t cap, uint64_t *n_out, void *stream);
+
+/* Add n weighted pairs: count[(d[j], t[j])] += cnt[j] (saturating), admission as
+ * in csd_ocm_update.  Loading a table built offline (Phase 1) or restoring an
+ * export is csd_ocm_reset followed by csd_ocm_import.  Device arrays; asynchronous. */
+csd_status_t csd_ocm_import(csd_ocm_t *ocm, const int32_t *d, const int32_t *t, const uint32_t *cnt,
+                            uint64_t n, void *stream);
+
+/* Copy the statistics block to the HOST struct.  Synchronises `stream`. */
+csd_status_t csd_ocm_stats(const csd_ocm_t *ocm, csd_stats_t *host_out, void *stream);
+
+/* ---- helpers ---- */
+
+/* (float) log((double) tau): the threshold the gate of Eq. 3 compares against.
+ * -inf for tau == 0.  Host function. */
+float csd_scg_threshold(float tau);
+
+/* Launch shape a step of this size uses: grid blocks, threads per block, elements
+ * per tile and tiles per logit row.  Host function; for reports and tests. */
+csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype,
+                              int *grid, int *block, int *tile_elems, int *tiles_per_row);
+
+/* Expert knob, process-wide: override the automatic tiling.  tile_bytes: bytes of
+ * logits reduced by one warp at a time (multiple of 4096; 0 = automatic);
+ * ctas_per_sm: resident blocks per SM of the persistent grid (1..4; 0 = automatic,
+ * which is 4).  Changes csd_workspace_bytes: size workspaces after calling it.
+ * Results stay bit-reproducible for a fixed setting; the low-order bits of the
+ * sums s may differ between settings (different summation trees).  Host function. */
+csd_status_t csd_set_tuning(int tile_bytes, int ctas_per_sm);
+
+const char *csd_status_string(csd_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSD_H_ */

@@ -1,0 +1,277 @@
+"""ctypes binding of libcsd.so: argument marshalling only.
+
+Every function mirrors one entry point of include/csd.h under the same name.
+Tensors are torch CUDA tensors (device memory and streams are torch's); all
+arithmetic happens in the library's kernels.  There is no fallback: if the
+library cannot be loaded, or a call fails, an exception is raised.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int64, c_size_t, c_uint32, c_uint64, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcsd.so")
+
+CSD_F32, CSD_BF16 = 0, 1
+CSD_MAX_K = 32
+FLAG_NAN_LOGIT, FLAG_BAD_DRAFT, FLAG_PROBE_EXHAUSTED, FLAG_COUNT_SATURATED = 1, 2, 4, 8
+
+EXPORTS = [
+    "csd_ocm_create", "csd_ocm_reset", "csd_ocm_destroy", "csd_ocm_set_lambda",
+    "csd_workspace_bytes", "csd_workspace_init", "csd_verify", "csd_ocm_update", "csd_step",
+    "csd_host_staging_bytes", "csd_step_host", "csd_ocm_export", "csd_ocm_import", "csd_ocm_stats",
+    "csd_scg_threshold", "csd_launch_shape", "csd_set_tuning", "csd_status_string",
+]
+
+
+class CsdError(RuntimeError):
+    pass
+
+
+class Diag(Structure):
+    _fields_ = [(n, c_void_p) for n in ("m", "s", "lse", "t", "zd", "score", "p_d", "p_t", "cnt")]
+
+
+class Stats(Structure):
+    _fields_ = [(n, c_uint64) for n in ("n_slots", "key_limit", "n_keys", "n_dropped", "steps", "positions",
+                                         "matches", "rescues", "rejections")] + [("lambda_", c_uint32), ("flags", c_uint32)]
+
+    def as_dict(self):
+        d = {n: int(getattr(self, n)) for n, _ in self._fields_}
+        d["lambda"] = d.pop("lambda_")
+        return d
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library.  Raises if it has not been built (see build.py)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise CsdError(f"{LIB_PATH} is missing: build it with `python -m paper_2604_13634_b200.build`")
+    L = ctypes.CDLL(LIB_PATH)
+    step_args = [c_void_p, c_int, c_int, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_float,
+                 c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, POINTER(Diag), c_void_p, c_size_t, c_void_p]
+    sigs = {
+        "csd_ocm_create": (c_int, [POINTER(c_void_p), c_uint64, c_uint32, c_int]),
+        "csd_ocm_reset": (c_int, [c_void_p, c_void_p]),
+        "csd_ocm_destroy": (c_int, [c_void_p]),
+        "csd_ocm_set_lambda": (c_int, [c_void_p, c_uint32]),
+        "csd_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int]),
+        "csd_workspace_init": (c_int, [c_void_p, c_size_t, c_void_p]),
+        "csd_verify": (c_int, step_args),
+        "csd_step": (c_int, step_args),
+        "csd_ocm_update": (c_int, [c_void_p, c_void_p, c_void_p, c_int64, c_void_p]),
+        "csd_host_staging_bytes": (c_size_t, [c_int, c_int, c_int, c_int]),
+        "csd_step_host": (c_int, [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_float,
+                                  c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]),
+        "csd_ocm_export": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_uint64, POINTER(c_uint64), c_void_p]),
+        "csd_ocm_import": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_uint64, c_void_p]),
+        "csd_ocm_stats": (c_int, [c_void_p, POINTER(Stats), c_void_p]),
+        "csd_scg_threshold": (c_float, [c_float]),
+        "csd_launch_shape": (c_int, [c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
+        "csd_set_tuning": (c_int, [c_int, c_int]),
+        "csd_status_string": (c_char_p, [c_int]),
+    }
+    for name, (res, args) in sigs.items():
+        fn = getattr(L, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = L
+    return L
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise CsdError(f"{what}: {lib().csd_status_string(rc).decode()} (status {rc})")
+
+
+def _stream_ptr(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return CSD_F32
+    if t.dtype == torch.bfloat16:
+        return CSD_BF16
+    raise CsdError(f"logits must be float32 or bfloat16, got {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def csd_scg_threshold(tau: float) -> float:
+    return float(lib().csd_scg_threshold(c_float(tau)))
+
+
+def csd_set_tuning(tile_bytes: int = 0, ctas_per_sm: int = 0):
+    _check(lib().csd_set_tuning(tile_bytes, ctas_per_sm), "csd_set_tuning")
+
+
+def csd_launch_shape(B, K, V, dtype_code):
+    g, b, te, tr = c_int(), c_int(), c_int(), c_int()
+    _check(lib().csd_launch_shape(B, K, V, dtype_code, byref(g), byref(b), byref(te), byref(tr)), "csd_launch_shape")
+    return dict(grid=g.value, block=b.value, tile_elems=te.value, tiles_per_row=tr.value)
+
+
+def csd_workspace_bytes(B, K, V, dtype_code) -> int:
+    return int(lib().csd_workspace_bytes(B, K, V, dtype_code))
+
+
+def csd_host_staging_bytes(B, K, V, dtype_code) -> int:
+    return int(lib().csd_host_staging_bytes(B, K, V, dtype_code))
+
+
+class Ocm:
+    """Owner of one csd_ocm_t (the Online Correction Memory of Sec. 4.2)."""
+
+    def __init__(self, n_slots: int, lam: int = 6, device: int = 0):
+        if not torch.cuda.is_available():
+            raise CsdError("a CUDA device is required")
+        h = c_void_p()
+        _check(lib().csd_ocm_create(byref(h), n_slots, lam, device), "csd_ocm_create")
+        self.handle = h
+        self.n_slots = n_slots
+        self.device = torch.device("cuda", device)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            torch.cuda.synchronize()
+            lib().csd_ocm_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reset(self, stream=None):
+        _check(lib().csd_ocm_reset(self.handle, _stream_ptr(stream)), "csd_ocm_reset")
+
+    def set_lambda(self, lam: int):
+        _check(lib().csd_ocm_set_lambda(self.handle, lam), "csd_ocm_set_lambda")
+
+    def update(self, rej_draft: torch.Tensor, rej_target: torch.Tensor, stream=None):
+        assert rej_draft.dtype == torch.int32 and rej_target.dtype == torch.int32
+        assert rej_draft.is_cuda and rej_target.is_cuda and rej_draft.is_contiguous() and rej_target.is_contiguous()
+        assert rej_draft.numel() == rej_target.numel()
+        _check(lib().csd_ocm_update(self.handle, _ptr(rej_draft), _ptr(rej_target), rej_draft.numel(),
+                                    _stream_ptr(stream)), "csd_ocm_update")
+
+    def import_(self, d: torch.Tensor, t: torch.Tensor, cnt: torch.Tensor, stream=None):
+        """cnt holds unsigned 32-bit counts; an int32 tensor carrying the same bits is accepted."""
+        assert d.dtype == torch.int32 and t.dtype == torch.int32 and cnt.dtype in (torch.int32, torch.uint32)
+        assert d.is_cuda and t.is_cuda and cnt.is_cuda
+        _check(lib().csd_ocm_import(self.handle, _ptr(d.contiguous()), _ptr(t.contiguous()), _ptr(cnt.contiguous()),
+                                    d.numel(), _stream_ptr(stream)), "csd_ocm_import")
+
+    def export(self, stream=None):
+        """(d, t, cnt) int64 CPU tensors of the stored pairs, sorted by (d, t).  Synchronises."""
+        st = self.stats(stream)
+        cap = max(1, st["n_keys"])
+        d = torch.empty(cap, dtype=torch.int32, device=self.device)
+        t = torch.empty(cap, dtype=torch.int32, device=self.device)
+        c = torch.empty(cap, dtype=torch.int32, device=self.device)
+        n = c_uint64()
+        _check(lib().csd_ocm_export(self.handle, _ptr(d), _ptr(t), _ptr(c), cap, byref(n), _stream_ptr(stream)),
+               "csd_ocm_export")
+        k = min(int(n.value), cap)
+        d = d[:k].cpu().to(torch.int64)
+        t = t[:k].cpu().to(torch.int64)
+        c = c[:k].cpu().to(torch.int64) & 0xFFFFFFFF
+        order = torch.argsort(d * (1 << 32) + t)
+        return d[order], t[order], c[order]
+
+    def stats(self, stream=None) -> dict:
+        s = Stats()
+        _check(lib().csd_ocm_stats(self.handle, byref(s), _stream_ptr(stream)), "csd_ocm_stats")
+        return s.as_dict()
+
+
+class StepBuffers:
+    """Caller-owned device buffers of one step shape: outputs, optional diagnostics, workspace."""
+
+    def __init__(self, B: int, K: int, V: int, dtype: torch.dtype, device="cuda", diag: bool = False):
+        self.B, self.K, self.V = B, K, V
+        self.dtype_code = CSD_F32 if dtype == torch.float32 else CSD_BF16
+        dev = torch.device(device)
+        self.accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+        self.next_token = torch.empty(B, dtype=torch.int32, device=dev)
+        self.rescued_mask = torch.empty(B, K, dtype=torch.uint8, device=dev)
+        self.rej_draft = torch.empty(B, K, dtype=torch.int32, device=dev)
+        self.rej_target = torch.empty(B, K, dtype=torch.int32, device=dev)
+        self.ws_bytes = csd_workspace_bytes(B, K, V, self.dtype_code)
+        if self.ws_bytes == 0:
+            raise CsdError(f"unsupported shape B={B} K={K} V={V}")
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        _check(lib().csd_workspace_init(_ptr(self.workspace), self.ws_bytes, _stream_ptr()), "csd_workspace_init")
+        self.diag = None
+        self._diag_struct = None
+        if diag:
+            f = dict(dtype=torch.float32, device=dev)
+            self.diag = dict(
+                m=torch.empty(B, K + 1, **f), s=torch.empty(B, K + 1, **f), lse=torch.empty(B, K + 1, **f),
+                t=torch.empty(B, K + 1, dtype=torch.int32, device=dev),
+                zd=torch.empty(B, K, **f), score=torch.empty(B, K, **f), p_d=torch.empty(B, K, **f),
+                p_t=torch.empty(B, K, **f), cnt=torch.empty(B, K, dtype=torch.int32, device=dev))
+            self._diag_struct = Diag(**{k: v.data_ptr() for k, v in self.diag.items()})
+
+
+def _step_call(fn_name, logits, draft, ocm: Ocm, tau, buf: StepBuffers, stream):
+    assert logits.is_cuda and draft.is_cuda and draft.dtype == torch.int32 and draft.is_contiguous()
+    B, K1, V = logits.shape
+    assert (B, K1 - 1, V) == (buf.B, buf.K, buf.V) and draft.shape == (B, K1 - 1)
+    assert logits.stride(2) == 1 and _dtype_code(logits) == buf.dtype_code
+    fn = getattr(lib(), fn_name)
+    rc = fn(logits.data_ptr(), buf.dtype_code, B, K1 - 1, V, logits.stride(0), logits.stride(1),
+            draft.data_ptr(), ocm.handle, c_float(tau),
+            _ptr(buf.accept_len), _ptr(buf.next_token), _ptr(buf.rescued_mask), _ptr(buf.rej_draft), _ptr(buf.rej_target),
+            byref(buf._diag_struct) if buf._diag_struct is not None else None,
+            _ptr(buf.workspace), buf.ws_bytes, _stream_ptr(stream))
+    _check(rc, fn_name)
+
+
+def csd_verify(logits, draft, ocm: Ocm, tau: float, buf: StepBuffers, stream=None):
+    """Verification loop of Algorithm 1 (greedy) for all rows; the memory is only read."""
+    _step_call("csd_verify", logits, draft, ocm, tau, buf, stream)
+
+
+def csd_step(logits, draft, ocm: Ocm, tau: float, buf: StepBuffers, stream=None):
+    """csd_verify plus the memory update with the step's rejections, in one launch."""
+    _step_call("csd_step", logits, draft, ocm, tau, buf, stream)
+
+
+class HostStep:
+    """csd_step_host: inputs and outputs in (pinned) host memory, copies inside the call."""
+
+    def __init__(self, B, K, V, dtype: torch.dtype, device="cuda"):
+        self.B, self.K, self.V = B, K, V
+        self.dtype_code = CSD_F32 if dtype == torch.float32 else CSD_BF16
+        self.bytes = csd_host_staging_bytes(B, K, V, self.dtype_code)
+        self.staging = torch.empty(self.bytes, dtype=torch.uint8, device=device)
+        assert self.staging.data_ptr() % 256 == 0
+        self.accept_len = torch.empty(B, dtype=torch.int32).pin_memory()
+        self.next_token = torch.empty(B, dtype=torch.int32).pin_memory()
+        self.rescued_mask = torch.empty(B, K, dtype=torch.uint8).pin_memory()
+
+    def __call__(self, logits_host: torch.Tensor, draft_host: torch.Tensor, ocm: Ocm, tau: float, stream=None):
+        assert not logits_host.is_cuda and logits_host.is_contiguous() and draft_host.dtype == torch.int32
+        assert tuple(logits_host.shape) == (self.B, self.K + 1, self.V) and _dtype_code(logits_host) == self.dtype_code
+        rc = lib().csd_step_host(logits_host.data_ptr(), self.dtype_code, self.B, self.K, self.V,
+                                 draft_host.data_ptr(), ocm.handle, c_float(tau),
+                                 self.accept_len.data_ptr(), self.next_token.data_ptr(), self.rescued_mask.data_ptr(),
+                                 self.staging.data_ptr(), self.bytes, _stream_ptr(stream))
+        _check(rc, "csd_step_host")
+        return self.accept_len, self.next_token, self.rescued_mask

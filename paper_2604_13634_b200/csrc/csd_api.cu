@@ -1,0 +1,455 @@
+// C ABI of the CSD verification library (see include/csd.h for the contract).
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "../../include/csd.h"
+#include "csd_common.cuh"
+#include "csd_ocm.cuh"
+#include "csd_step.cuh"
+
+using namespace csd;
+
+struct csd_ocm {
+    int device;
+    uint64_t n_slots;
+    uint32_t lambda;
+    OcmSlot *slots;
+    OcmStatsDev *stats;
+};
+
+namespace {
+
+constexpr int kDefaultSms = 148;   // B200; used only when no device can be queried
+
+int g_tile_bytes_override = 0;
+int g_ctas_per_sm_override = 0;
+
+int sm_count()
+{
+    static int cached = 0;
+    if (cached > 0) return cached;
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) {
+        cached = n;
+        return n;
+    }
+    (void)cudaGetLastError();
+    return kDefaultSms;
+}
+
+struct Shape {
+    int grid;
+    int tile_elems;
+    int n_split;
+    long long total_tiles;
+};
+
+inline int elt_bytes(csd_dtype_t dt) { return dt == CSD_F32 ? 4 : 2; }
+
+bool shape_ok(int B, int K, int V, csd_dtype_t dt)
+{
+    return B > 0 && K > 0 && V > 0 && K <= CSD_MAX_K && (dt == CSD_F32 || dt == CSD_BF16) &&
+           static_cast<long long>(B) * (K + 1) < (1ll << 31);
+}
+
+// Tiles are whole warp iterations (32 lanes x 8 x 16 bytes = 4 KiB).  Small problems
+// get 4 KiB tiles so that every warp of the machine has work; large ones get up to
+// 32 KiB so that a batch row is described by few partials.
+Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
+{
+    const int eb = elt_bytes(dt);
+    const int ctas_per_sm = g_ctas_per_sm_override > 0 ? g_ctas_per_sm_override : 4;
+    const long long workers = static_cast<long long>(sm_count()) * ctas_per_sm * kWarps;
+    const long long rows = static_cast<long long>(B) * (K + 1);
+    const long long total_bytes = rows * V * eb;
+    long long tile_bytes = 4096;
+    if (g_tile_bytes_override > 0) {
+        tile_bytes = g_tile_bytes_override;
+    } else {
+        while (tile_bytes < 32768 && total_bytes / (tile_bytes * 2) >= 4 * workers) tile_bytes *= 2;
+    }
+    Shape s;
+    s.tile_elems = static_cast<int>(tile_bytes / eb);
+    s.n_split = (V + s.tile_elems - 1) / s.tile_elems;
+    s.total_tiles = rows * s.n_split;
+    long long blocks = static_cast<long long>(sm_count()) * ctas_per_sm;
+    const long long needed = (s.total_tiles + kWarps - 1) / kWarps;
+    if (needed < blocks) blocks = needed;
+    s.grid = static_cast<int>(blocks < 1 ? 1 : blocks);
+    return s;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WorkspaceLayout {
+    size_t partials_off, b_ticket_off, g_ticket_off, total;
+};
+
+WorkspaceLayout ws_layout(int B, int K, const Shape &s)
+{
+    WorkspaceLayout w;
+    w.partials_off = 0;
+    w.b_ticket_off = align_up(static_cast<size_t>(B) * (K + 1) * s.n_split * sizeof(Partial), 256);
+    w.g_ticket_off = align_up(w.b_ticket_off + static_cast<size_t>(B) * sizeof(unsigned int), 16);
+    w.total = align_up(w.g_ticket_off + 16, 256);
+    return w;
+}
+
+OcmView view_of(const csd_ocm *o)
+{
+    OcmView v;
+    v.slots = o->slots;
+    v.mask = o->n_slots - 1;
+    v.key_limit = o->n_slots / 2;
+    v.lambda = o->lambda;
+    v.stats = o->stats;
+    return v;
+}
+
+csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b, int64_t stride_k,
+                      const int32_t *draft, const csd_ocm *ocm, float tau, int32_t *accept_len, int32_t *next_token,
+                      uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
+                      void *workspace, size_t workspace_bytes, void *stream, bool do_update)
+{
+    if (!logits || !draft || !ocm || !accept_len || !next_token || !rescued_mask || !rej_draft || !rej_target || !workspace)
+        return CSD_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || V <= 0) return CSD_ERR_INVALID_ARG;
+    if (dtype != CSD_F32 && dtype != CSD_BF16) return CSD_ERR_INVALID_ARG;
+    if (K > CSD_MAX_K) return CSD_ERR_UNSUPPORTED;
+    if (!shape_ok(B, K, V, dtype)) return CSD_ERR_UNSUPPORTED;
+    if (!(tau >= 0.0f) || std::isinf(tau)) return CSD_ERR_INVALID_ARG;   // also refuses NaN
+    if (stride_k < V || stride_b < stride_k * (K + 1)) return CSD_ERR_INVALID_ARG;
+
+    const Shape s = pick_shape(B, K, V, dtype);
+    const WorkspaceLayout w = ws_layout(B, K, s);
+    if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
+
+    StepParams p;
+    std::memset(&p, 0, sizeof p);
+    p.logits = logits;
+    p.B = B; p.K = K; p.V = V;
+    p.stride_b = stride_b; p.stride_k = stride_k;
+    p.draft = draft;
+    p.ocm = view_of(ocm);
+    p.log_tau = csd_scg_threshold(tau);
+    p.do_update = do_update ? 1 : 0;
+    p.accept_len = accept_len; p.next_token = next_token; p.rescued = rescued_mask;
+    p.rej_d = rej_draft; p.rej_t = rej_target;
+    if (diag) p.diag = *diag;
+    char *ws = static_cast<char *>(workspace);
+    p.partials = reinterpret_cast<Partial *>(ws + w.partials_off);
+    p.b_ticket = reinterpret_cast<unsigned int *>(ws + w.b_ticket_off);
+    p.g_ticket = reinterpret_cast<unsigned int *>(ws + w.g_ticket_off);
+    p.tile_elems = s.tile_elems;
+    p.n_split = s.n_split;
+    p.total_tiles = s.total_tiles;
+
+    const int eb = elt_bytes(dtype);
+    const int per_vec = 16 / eb;
+    const bool vec = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && (stride_b * eb) % 16 == 0 &&
+                     (stride_k * eb) % 16 == 0 && V % per_vec == 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dim3 grid(s.grid), block(kThreads);
+    if (dtype == CSD_F32) {
+        if (vec) csd_step_kernel<LaneF32Vec><<<grid, block, 0, st>>>(p);
+        else csd_step_kernel<LaneF32Scalar><<<grid, block, 0, st>>>(p);
+    } else {
+        if (vec) csd_step_kernel<LaneBf16Vec><<<grid, block, 0, st>>>(p);
+        else csd_step_kernel<LaneBf16Scalar><<<grid, block, 0, st>>>(p);
+    }
+    return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
+}
+
+csd_status_t run_update(csd_ocm *ocm, const int32_t *d, const int32_t *t, const uint32_t *w, int64_t n, void *stream)
+{
+    if (!ocm || n < 0 || (n > 0 && (!d || !t))) return CSD_ERR_INVALID_ARG;
+    if (n == 0) return CSD_OK;
+    long long blocks = (n + 1023) / 1024;
+    const long long cap = static_cast<long long>(sm_count()) * 2;
+    if (blocks > cap) blocks = cap;
+    ocm_update_kernel<<<static_cast<unsigned int>(blocks), 1024, 0, static_cast<cudaStream_t>(stream)>>>(
+        view_of(ocm), d, t, w, n);
+    return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+csd_status_t csd_ocm_create(csd_ocm_t **out, uint64_t n_slots, uint32_t lambda, int device)
+{
+    if (!out) return CSD_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (n_slots < 64 || (n_slots & (n_slots - 1)) != 0 || n_slots > (1ull << 40)) return CSD_ERR_INVALID_ARG;
+    if (cudaSetDevice(device) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    csd_ocm *o = new (std::nothrow) csd_ocm;
+    if (!o) return CSD_ERR_OOM;
+    o->device = device;
+    o->n_slots = n_slots;
+    o->lambda = lambda;
+    o->slots = nullptr;
+    o->stats = nullptr;
+    if (cudaMalloc(&o->slots, n_slots * sizeof(OcmSlot)) != cudaSuccess ||
+        cudaMalloc(&o->stats, sizeof(OcmStatsDev)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        if (o->slots) cudaFree(o->slots);
+        delete o;
+        return CSD_ERR_OOM;
+    }
+    csd_status_t rc = csd_ocm_reset(o, nullptr);
+    if (rc == CSD_OK && cudaDeviceSynchronize() != cudaSuccess) rc = CSD_ERR_CUDA;
+    if (rc != CSD_OK) {
+        cudaFree(o->slots);
+        cudaFree(o->stats);
+        delete o;
+        return rc;
+    }
+    *out = o;
+    return CSD_OK;
+}
+
+csd_status_t csd_ocm_reset(csd_ocm_t *ocm, void *stream)
+{
+    if (!ocm) return CSD_ERR_INVALID_ARG;
+    unsigned long long blocks = (ocm->n_slots + 255) / 256;
+    const unsigned long long cap = static_cast<unsigned long long>(sm_count()) * 8;
+    if (blocks > cap) blocks = cap;
+    ocm_reset_kernel<<<static_cast<unsigned int>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        ocm->slots, ocm->n_slots, ocm->stats);
+    return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
+}
+
+csd_status_t csd_ocm_destroy(csd_ocm_t *ocm)
+{
+    if (!ocm) return CSD_ERR_INVALID_ARG;
+    cudaError_t a = cudaFree(ocm->slots);
+    cudaError_t b = cudaFree(ocm->stats);
+    delete ocm;
+    return (a == cudaSuccess && b == cudaSuccess) ? CSD_OK : CSD_ERR_CUDA;
+}
+
+csd_status_t csd_ocm_set_lambda(csd_ocm_t *ocm, uint32_t lambda)
+{
+    if (!ocm) return CSD_ERR_INVALID_ARG;
+    ocm->lambda = lambda;
+    return CSD_OK;
+}
+
+size_t csd_workspace_bytes(int B, int K, int V, csd_dtype_t dtype)
+{
+    if (!shape_ok(B, K, V, dtype)) return 0;
+    return ws_layout(B, K, pick_shape(B, K, V, dtype)).total;
+}
+
+csd_status_t csd_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!workspace || workspace_bytes == 0) return CSD_ERR_INVALID_ARG;
+    if (cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    return CSD_OK;
+}
+
+csd_status_t csd_verify(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b, int64_t stride_k,
+                        const int32_t *draft, const csd_ocm_t *ocm, float tau, int32_t *accept_len, int32_t *next_token,
+                        uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
+                        void *workspace, size_t workspace_bytes, void *stream)
+{
+    return run_step(logits, dtype, B, K, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
+                    rej_draft, rej_target, diag, workspace, workspace_bytes, stream, false);
+}
+
+csd_status_t csd_step(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b, int64_t stride_k,
+                      const int32_t *draft, csd_ocm_t *ocm, float tau, int32_t *accept_len, int32_t *next_token,
+                      uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
+                      void *workspace, size_t workspace_bytes, void *stream)
+{
+    return run_step(logits, dtype, B, K, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
+                    rej_draft, rej_target, diag, workspace, workspace_bytes, stream, true);
+}
+
+csd_status_t csd_ocm_update(csd_ocm_t *ocm, const int32_t *rej_draft, const int32_t *rej_target, int64_t n, void *stream)
+{
+    return run_update(ocm, rej_draft, rej_target, nullptr, n, stream);
+}
+
+csd_status_t csd_ocm_import(csd_ocm_t *ocm, const int32_t *d, const int32_t *t, const uint32_t *cnt, uint64_t n,
+                            void *stream)
+{
+    if (n > 0 && !cnt) return CSD_ERR_INVALID_ARG;
+    if (n > (1ull << 62)) return CSD_ERR_INVALID_ARG;
+    return run_update(ocm, d, t, cnt, static_cast<int64_t>(n), stream);
+}
+
+// staging layout of csd_step_host: logits | draft | accept_len | next_token | rescued |
+// rej_draft | rej_target | workspace, each 256-byte aligned
+namespace {
+struct StagingLayout {
+    size_t logits, draft, accept, next, rescued, rej_d, rej_t, ws, ws_bytes, total;
+};
+StagingLayout staging_layout(int B, int K, int V, csd_dtype_t dtype)
+{
+    StagingLayout s;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    s.logits = take(static_cast<size_t>(B) * (K + 1) * V * elt_bytes(dtype));
+    s.draft = take(static_cast<size_t>(B) * K * 4);
+    s.accept = take(static_cast<size_t>(B) * 4);
+    s.next = take(static_cast<size_t>(B) * 4);
+    s.rescued = take(static_cast<size_t>(B) * K);
+    s.rej_d = take(static_cast<size_t>(B) * K * 4);
+    s.rej_t = take(static_cast<size_t>(B) * K * 4);
+    s.ws_bytes = csd_workspace_bytes(B, K, V, dtype);
+    s.ws = take(s.ws_bytes);
+    s.total = off;
+    return s;
+}
+}  // namespace
+
+size_t csd_host_staging_bytes(int B, int K, int V, csd_dtype_t dtype)
+{
+    if (!shape_ok(B, K, V, dtype)) return 0;
+    return staging_layout(B, K, V, dtype).total;
+}
+
+csd_status_t csd_step_host(const void *logits_host, csd_dtype_t dtype, int B, int K, int V, const int32_t *draft_host,
+                           csd_ocm_t *ocm, float tau, int32_t *accept_len_host, int32_t *next_token_host,
+                           uint8_t *rescued_mask_host, void *staging, size_t staging_bytes, void *stream)
+{
+    if (!logits_host || !draft_host || !ocm || !accept_len_host || !next_token_host || !rescued_mask_host || !staging)
+        return CSD_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || V <= 0 || (dtype != CSD_F32 && dtype != CSD_BF16)) return CSD_ERR_INVALID_ARG;
+    if (K > CSD_MAX_K || !shape_ok(B, K, V, dtype)) return CSD_ERR_UNSUPPORTED;
+    const StagingLayout s = staging_layout(B, K, V, dtype);
+    if (staging_bytes < s.total || (reinterpret_cast<uintptr_t>(staging) & 255u)) return CSD_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *dev = static_cast<char *>(staging);
+    const size_t lbytes = static_cast<size_t>(B) * (K + 1) * V * elt_bytes(dtype);
+    bool ok = true;
+    ok = ok && cudaMemcpyAsync(dev + s.logits, logits_host, lbytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(dev + s.draft, draft_host, static_cast<size_t>(B) * K * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    // the arrival counters sit at the end of the workspace; clearing it all keeps the staging stateless
+    ok = ok && cudaMemsetAsync(dev + s.ws, 0, s.ws_bytes, st) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    const csd_status_t rc =
+        csd_step(dev + s.logits, dtype, B, K, V, static_cast<int64_t>(K + 1) * V, V,
+                 reinterpret_cast<const int32_t *>(dev + s.draft), ocm, tau, reinterpret_cast<int32_t *>(dev + s.accept),
+                 reinterpret_cast<int32_t *>(dev + s.next), reinterpret_cast<uint8_t *>(dev + s.rescued),
+                 reinterpret_cast<int32_t *>(dev + s.rej_d), reinterpret_cast<int32_t *>(dev + s.rej_t), nullptr,
+                 dev + s.ws, s.ws_bytes, stream);
+    if (rc != CSD_OK) return rc;
+    ok = ok && cudaMemcpyAsync(accept_len_host, dev + s.accept, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(next_token_host, dev + s.next, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(rescued_mask_host, dev + s.rescued, static_cast<size_t>(B) * K, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    return CSD_OK;
+}
+
+csd_status_t csd_ocm_export(const csd_ocm_t *ocm, int32_t *d, int32_t *t, uint32_t *cnt, uint64_t cap, uint64_t *n_out,
+                            void *stream)
+{
+    if (!ocm || !n_out || (cap > 0 && (!d || !t || !cnt))) return CSD_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    bool ok = cudaMemsetAsync(&ocm->stats->export_count, 0, sizeof(unsigned long long), st) == cudaSuccess;
+    if (ok) {
+        unsigned long long blocks = (ocm->n_slots + 255) / 256;
+        const unsigned long long capb = static_cast<unsigned long long>(sm_count()) * 8;
+        if (blocks > capb) blocks = capb;
+        ocm_export_kernel<<<static_cast<unsigned int>(blocks), 256, 0, st>>>(view_of(ocm), d, t, cnt, cap);
+        ok = cudaGetLastError() == cudaSuccess;
+    }
+    unsigned long long n = 0;
+    ok = ok && cudaMemcpyAsync(&n, &ocm->stats->export_count, sizeof n, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    *n_out = n;
+    return CSD_OK;
+}
+
+csd_status_t csd_ocm_stats(const csd_ocm_t *ocm, csd_stats_t *host_out, void *stream)
+{
+    if (!ocm || !host_out) return CSD_ERR_INVALID_ARG;
+    OcmStatsDev s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&s, ocm->stats, sizeof s, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    host_out->n_slots = ocm->n_slots;
+    host_out->key_limit = ocm->n_slots / 2;
+    host_out->n_keys = s.n_keys;
+    host_out->n_dropped = s.n_dropped;
+    host_out->steps = s.steps;
+    host_out->positions = s.positions;
+    host_out->matches = s.matches;
+    host_out->rescues = s.rescues;
+    host_out->rejections = s.rejections;
+    host_out->lambda = ocm->lambda;
+    host_out->flags = s.flags;
+    return CSD_OK;
+}
+
+float csd_scg_threshold(float tau)
+{
+    if (tau == 0.0f) return -INFINITY;
+    return static_cast<float>(std::log(static_cast<double>(tau)));
+}
+
+csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype, int *grid, int *block, int *tile_elems,
+                              int *tiles_per_row)
+{
+    if (!shape_ok(B, K, V, dtype)) return CSD_ERR_INVALID_ARG;
+    const Shape s = pick_shape(B, K, V, dtype);
+    if (grid) *grid = s.grid;
+    if (block) *block = kThreads;
+    if (tile_elems) *tile_elems = s.tile_elems;
+    if (tiles_per_row) *tiles_per_row = s.n_split;
+    return CSD_OK;
+}
+
+csd_status_t csd_set_tuning(int tile_bytes, int ctas_per_sm)
+{
+    if (tile_bytes != 0 && (tile_bytes < 4096 || tile_bytes % 4096 != 0 || tile_bytes > (1 << 22))) return CSD_ERR_INVALID_ARG;
+    if (ctas_per_sm < 0 || ctas_per_sm > 4) return CSD_ERR_INVALID_ARG;
+    g_tile_bytes_override = tile_bytes;
+    g_ctas_per_sm_override = ctas_per_sm;
+    return CSD_OK;
+}
+
+const char *csd_status_string(csd_status_t status)
+{
+    switch (status) {
+        case CSD_OK: return "ok";
+        case CSD_ERR_INVALID_ARG: return "invalid argument";
+        case CSD_ERR_CUDA: return "CUDA error";
+        case CSD_ERR_OOM: return "out of memory";
+        case CSD_ERR_UNSUPPORTED: return "unsupported shape";
+        case CSD_ERR_WORKSPACE: return "workspace too small or misaligned";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

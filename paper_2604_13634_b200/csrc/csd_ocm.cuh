@@ -1,0 +1,336 @@
+// Online Correction Memory (Sec. 4.2): an open-addressed hash table in device memory
+// mapping the ordered pair (draft token, target token) to a 32-bit count.
+//
+// Layout: n_slots (power of two) 16-byte slots {key:u64, count:u32, pad:u32}, linear
+// probing from a 64-bit mix of the key.  An empty slot has key = ~0 (never a valid
+// pair: both halves would be negative).  A look-up is one 16-byte load per probe.
+//
+// Capacity rule (this library's; the paper gives none): at most key_limit =
+// n_slots / 2 distinct keys.  Present keys always count; new keys are admitted in
+// the canonical (index) order of an update while there is room; an occurrence that
+// finds no room is dropped and counted.  Because admission depends only on the set
+// of keys and on the canonical order, the table's contents never depend on the hash
+// function, on slot positions or on the order in which threads run.
+#pragma once
+
+#include "csd_common.cuh"
+
+namespace csd {
+
+struct __align__(16) OcmSlot {
+    unsigned long long key;
+    unsigned int count;
+    unsigned int pad;
+};
+
+constexpr unsigned long long kEmptyKey = ~0ull;
+
+struct OcmStatsDev {
+    unsigned long long n_keys;        // distinct keys stored (live)
+    unsigned long long n_keys_start;  // n_keys when the running update began (set between updates)
+    unsigned long long n_dropped;
+    unsigned long long steps;
+    unsigned long long positions;
+    unsigned long long matches;
+    unsigned long long rescues;
+    unsigned long long rejections;
+    unsigned int flags;
+    unsigned int ticket;              // arrival counter of multi-block update launches
+    unsigned long long export_count;  // cursor of csd_ocm_export
+};
+
+struct OcmView {
+    OcmSlot *slots;
+    unsigned long long mask;       // n_slots - 1
+    unsigned long long key_limit;  // n_slots / 2
+    unsigned int lambda;
+    OcmStatsDev *stats;
+};
+
+__device__ __forceinline__ unsigned long long make_key(int d, int t)
+{
+    return (static_cast<unsigned long long>(static_cast<unsigned int>(d)) << 32) |
+           static_cast<unsigned long long>(static_cast<unsigned int>(t));
+}
+
+// 64-bit finaliser (xor-shift-multiply rounds); any well-mixing map works because
+// the table's contents never depend on it.
+__device__ __forceinline__ unsigned long long mix64(unsigned long long x)
+{
+    x ^= x >> 31;
+    x *= 0x7fb5d329728ea185ull;
+    x ^= x >> 27;
+    x *= 0x81dadef4bc2dd44dull;
+    x ^= x >> 33;
+    return x;
+}
+
+__device__ __forceinline__ void load_slot(const OcmSlot *s, unsigned long long &key, unsigned int &count)
+{
+    const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(s));
+    key = (static_cast<unsigned long long>(v.y) << 32) | v.x;
+    count = v.z;
+}
+
+// Count stored for `key`, 0 if absent.  *slot_out = slot index or -1.
+__device__ __forceinline__ unsigned int ocm_lookup(const OcmView &tb, unsigned long long key, long long *slot_out = nullptr)
+{
+    unsigned long long slot = mix64(key) & tb.mask;
+    for (unsigned long long probe = 0; probe <= tb.mask; ++probe) {
+        unsigned long long k;
+        unsigned int c;
+        load_slot(tb.slots + slot, k, c);
+        if (k == key) {
+            if (slot_out) *slot_out = static_cast<long long>(slot);
+            return c;
+        }
+        if (k == kEmptyKey) {
+            if (slot_out) *slot_out = -1;
+            return 0;
+        }
+        slot = (slot + 1) & tb.mask;
+    }
+    atomicOr(&tb.stats->flags, 0x4u);
+    if (slot_out) *slot_out = -1;
+    return 0;
+}
+
+// count += w, saturating at 2^32 - 1.
+__device__ __forceinline__ void ocm_add(const OcmView &tb, unsigned long long slot, unsigned int w)
+{
+    unsigned int *cnt = &tb.slots[slot].count;
+    const unsigned int old = atomicAdd(cnt, w);
+    if (old + w < old) {   // wrapped: pin to the maximum (every wrapping adder does the same)
+        atomicExch(cnt, 0xffffffffu);
+        atomicOr(&tb.stats->flags, 0x8u);
+    }
+}
+
+// Insert-or-increment without a capacity check (the caller has established that there
+// is room for every new key of the batch).
+__device__ __forceinline__ void ocm_insert_or_add(const OcmView &tb, unsigned long long key, unsigned int w)
+{
+    unsigned long long slot = mix64(key) & tb.mask;
+    for (unsigned long long probe = 0; probe <= tb.mask; ++probe) {
+        unsigned long long *kp = &tb.slots[slot].key;
+        unsigned long long k = *reinterpret_cast<volatile unsigned long long *>(kp);
+        if (k == kEmptyKey) {
+            k = atomicCAS(kp, kEmptyKey, key);
+            if (k == kEmptyKey) {
+                atomicAdd(&tb.stats->n_keys, 1ull);
+                k = key;
+            }
+        }
+        if (k == key) {
+            ocm_add(tb, slot, w);
+            return;
+        }
+        slot = (slot + 1) & tb.mask;
+    }
+    atomicOr(&tb.stats->flags, 0x4u);
+}
+
+// Increment if present, else count a dropped occurrence (table full: nothing is admitted).
+__device__ __forceinline__ void ocm_add_or_drop(const OcmView &tb, unsigned long long key, unsigned int w)
+{
+    long long slot;
+    ocm_lookup(tb, key, &slot);
+    if (slot >= 0)
+        ocm_add(tb, static_cast<unsigned long long>(slot), w);
+    else
+        atomicAdd(&tb.stats->n_dropped, 1ull);
+}
+
+constexpr int kCanonChunk = 1024;   // entries handled at a time by the canonical-order path
+
+struct CanonScratch {
+    unsigned long long key[kCanonChunk];
+    unsigned short first[kCanonChunk];
+    unsigned char state[kCanonChunk];     // 0 done/skip, 1 pending first occurrence, 2 pending repeat
+    unsigned char admit[kCanonChunk];
+    unsigned long long avail;
+};
+
+__device__ __forceinline__ bool entry_key(const int *rd, const int *rt, long long j, unsigned long long &key)
+{
+    const int d = __ldcg(rd + j);
+    const int t = __ldcg(rt + j);
+    key = make_key(d, t);
+    return d >= 0 && t >= 0;
+}
+
+// Canonical-order update of entries [j0, j0 + n) (n <= kCanonChunk) by the `nthreads`
+// threads of one group (a whole block: `block_sync` true, or a single warp).  Used only
+// while the table is close to its key limit, where the order of admission matters:
+// new keys are ranked by their first occurrence and the first `avail` are admitted.
+template <bool kBlock>
+__device__ void ocm_update_canonical(const OcmView &tb, const int *rd, const int *rt, const unsigned int *w,
+                                     long long j0, int n, CanonScratch &sc, int tid, int nthreads)
+{
+    auto sync = [&]() {
+        if (kBlock) __syncthreads(); else __syncwarp();
+    };
+    if (tid == 0) {
+        const unsigned long long nk = atomicAdd(&tb.stats->n_keys, 0ull);
+        sc.avail = nk < tb.key_limit ? tb.key_limit - nk : 0ull;
+    }
+    // phase A: present keys count; absent ones become pending
+    for (int j = tid; j < n; j += nthreads) {
+        unsigned long long key;
+        const bool valid = entry_key(rd, rt, j0 + j, key);
+        sc.key[j] = key;
+        unsigned char st = 0;
+        if (valid) {
+            long long slot;
+            ocm_lookup(tb, key, &slot);
+            if (slot >= 0)
+                ocm_add(tb, static_cast<unsigned long long>(slot), w ? __ldcg(w + j0 + j) : 1u);
+            else
+                st = 1;
+        }
+        sc.state[j] = st;
+        sc.admit[j] = 0;
+    }
+    sync();
+    // phase B: mark repeats of a pending key and remember its first occurrence
+    for (int j = tid; j < n; j += nthreads) {
+        if (sc.state[j] == 0) continue;
+        const unsigned long long key = sc.key[j];
+        for (int i = 0; i < j; ++i) {
+            if (sc.state[i] != 0 && sc.key[i] == key) {
+                sc.first[j] = static_cast<unsigned short>(i);
+                sc.state[j] = 2;
+                break;
+            }
+        }
+    }
+    sync();
+    // phase C: rank first occurrences in index order; the first `avail` are admitted
+    for (int j = tid; j < n; j += nthreads) {
+        if (sc.state[j] != 1) continue;
+        unsigned long long rank = 0;
+        for (int i = 0; i < j; ++i) rank += (sc.state[i] == 1);
+        sc.admit[j] = rank < sc.avail;
+    }
+    sync();
+    // phase D: admitted keys are inserted (repeats add to them); the rest are dropped
+    for (int j = tid; j < n; j += nthreads) {
+        const unsigned char st = sc.state[j];
+        if (st == 0) continue;
+        const int f = st == 1 ? j : sc.first[j];
+        if (sc.admit[f])
+            ocm_insert_or_add(tb, sc.key[j], w ? __ldcg(w + j0 + j) : 1u);
+        else
+            atomicAdd(&tb.stats->n_dropped, 1ull);
+    }
+    sync();
+}
+
+// UpdateMemory of Algorithm 1 for entries [0, n) by one group of threads that is the
+// only writer of the table while it runs.  Three regimes, all giving the result of
+// processing the entries one by one in index order:
+//   room for everything   -> every thread inserts/increments independently
+//   table full            -> increments only; absent keys are dropped
+//   in between            -> canonical-order path, kCanonChunk entries at a time
+template <bool kBlock>
+__device__ void ocm_update_group(const OcmView &tb, const int *rd, const int *rt, const unsigned int *w,
+                                 long long n, CanonScratch &sc, int tid, int nthreads)
+{
+    auto sync = [&]() {
+        if (kBlock) __syncthreads(); else __syncwarp();
+    };
+    const unsigned long long nk = atomicAdd(&tb.stats->n_keys, 0ull);
+    if (nk + static_cast<unsigned long long>(n) <= tb.key_limit) {
+        for (long long j = tid; j < n; j += nthreads) {
+            unsigned long long key;
+            if (entry_key(rd, rt, j, key)) ocm_insert_or_add(tb, key, w ? __ldcg(w + j) : 1u);
+        }
+    } else if (nk >= tb.key_limit) {
+        for (long long j = tid; j < n; j += nthreads) {
+            unsigned long long key;
+            if (entry_key(rd, rt, j, key)) ocm_add_or_drop(tb, key, w ? __ldcg(w + j) : 1u);
+        }
+    } else {
+        for (long long j0 = 0; j0 < n; j0 += kCanonChunk) {
+            const int cn = static_cast<int>(n - j0 < kCanonChunk ? n - j0 : kCanonChunk);
+            sync();
+            ocm_update_canonical<kBlock>(tb, rd, rt, w, j0, cn, sc, tid, nthreads);
+        }
+    }
+    sync();
+}
+
+// ---- stand-alone kernels -------------------------------------------------------
+
+__global__ void ocm_reset_kernel(OcmSlot *slots, unsigned long long n_slots, OcmStatsDev *stats)
+{
+    const unsigned long long stride = static_cast<unsigned long long>(gridDim.x) * blockDim.x;
+    for (unsigned long long i = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_slots;
+         i += stride) {
+        uint4 v;
+        v.x = 0xffffffffu;
+        v.y = 0xffffffffu;
+        v.z = 0u;
+        v.w = 0u;
+        *reinterpret_cast<uint4 *>(slots + i) = v;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        OcmStatsDev z = {};
+        *stats = z;
+    }
+}
+
+// csd_ocm_update / csd_ocm_import.  Every block reads the same n_keys_start (written
+// when the previous update finished), so all blocks agree on the regime: with room
+// for all n entries each block handles its slice; otherwise block 0 alone walks the
+// whole batch in canonical order.  The last block to finish publishes n_keys_start.
+__global__ void __launch_bounds__(1024) ocm_update_kernel(OcmView tb, const int *rd, const int *rt, const unsigned int *w,
+                                                          long long n)
+{
+    __shared__ CanonScratch sc;
+    __shared__ bool last;
+    const unsigned long long nk0 = __ldcg(&tb.stats->n_keys_start);
+    if (nk0 + static_cast<unsigned long long>(n) <= tb.key_limit) {
+        const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+        for (long long j = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += stride) {
+            unsigned long long key;
+            if (entry_key(rd, rt, j, key)) ocm_insert_or_add(tb, key, w ? __ldcg(w + j) : 1u);
+        }
+    } else if (blockIdx.x == 0) {
+        ocm_update_group<true>(tb, rd, rt, w, n, sc, threadIdx.x, blockDim.x);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int old = atomicAdd(&tb.stats->ticket, 1u);
+        last = (old == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (last && threadIdx.x == 0) {
+        __threadfence();
+        const unsigned long long nk = atomicAdd(&tb.stats->n_keys, 0ull);
+        tb.stats->n_keys_start = nk;
+        tb.stats->ticket = 0u;
+    }
+}
+
+__global__ void ocm_export_kernel(OcmView tb, int *d, int *t, unsigned int *cnt, unsigned long long cap)
+{
+    const unsigned long long stride = static_cast<unsigned long long>(gridDim.x) * blockDim.x;
+    for (unsigned long long i = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x; i <= tb.mask;
+         i += stride) {
+        unsigned long long k;
+        unsigned int c;
+        load_slot(tb.slots + i, k, c);
+        if (k != kEmptyKey) {
+            const unsigned long long pos = atomicAdd(&tb.stats->export_count, 1ull);
+            if (pos < cap) {
+                d[pos] = static_cast<int>(k >> 32);
+                t[pos] = static_cast<int>(k & 0xffffffffull);
+                cnt[pos] = c;
+            }
+        }
+    }
+}
+
+}  // namespace csd

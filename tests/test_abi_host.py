@@ -1,0 +1,96 @@
+"""CPU-side checks of the C ABI: the library loads, exports what the header declares,
+and its host logic (argument checks, threshold, launch shapes) behaves as documented."""
+
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import csd_oracle as ORACLE
+from paper_2604_13634_b200 import binding, build
+
+
+@pytest.fixture(scope="module")
+def L():
+    build.build()
+    return binding.lib()
+
+
+def _declared(repo_root):
+    text = open(os.path.join(repo_root, "include", "csd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(csd_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_exports_match_header(L, repo_root):
+    names = _declared(repo_root)
+    assert len(names) >= 18
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in csd.h but not exported"
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_threshold_matches_oracle(L):
+    taus = [0.0, 1e-10, 0.001, 0.01, 0.05, 0.1, 0.2, 0.25, 0.3, 0.4, 0.5, 0.6, 0.9, 1.0, 1.5, 7.0]
+    taus += list(np.random.default_rng(0).random(2000).astype(np.float32))
+    for tau in taus:
+        assert binding.csd_scg_threshold(float(tau)) == ORACLE.scg_threshold(float(tau)), tau
+
+
+def test_status_strings(L):
+    seen = {L.csd_status_string(i) for i in range(6)}
+    assert len(seen) == 6 and b"ok" in seen
+
+
+def test_shapes_and_workspace(L):
+    for (B, K, V, dt) in ((1, 4, 32000, 0), (1, 8, 128256, 1), (32, 5, 151936, 1), (128, 8, 128256, 0),
+                          (64, 6, 152064, 1), (3, 1, 7, 0), (2, 32, 1000, 1)):
+        s = binding.csd_launch_shape(B, K, V, dt)
+        eb = 4 if dt == 0 else 2
+        assert s["block"] == 256 and s["grid"] >= 1
+        assert (s["tile_elems"] * eb) % 4096 == 0
+        assert s["tiles_per_row"] == -(-V // s["tile_elems"])
+        ws = binding.csd_workspace_bytes(B, K, V, dt)
+        assert ws >= B * (K + 1) * s["tiles_per_row"] * 16 + 4 * B + 4
+        assert binding.csd_host_staging_bytes(B, K, V, dt) >= B * (K + 1) * V * eb + ws
+    assert binding.csd_workspace_bytes(0, 4, 100, 0) == 0
+    assert binding.csd_workspace_bytes(1, 33, 100, 0) == 0
+    assert binding.csd_workspace_bytes(1, 4, 100, 7) == 0
+
+
+def test_argument_checks_refuse_before_launch(L):
+    null = None
+    one = ctypes.c_void_p(16)      # a non-null, never dereferenced, address
+    f = ctypes.c_float
+    def verify(**kw):
+        a = dict(logits=one, dt=0, B=2, K=3, V=64, sb=4 * 64, sk=64, draft=one, ocm=one, tau=0.3, acc=one, nxt=one,
+                 resc=one, rd=one, rt=one, diag=None, ws=one, wsb=1 << 20)
+        a.update(kw)
+        return L.csd_verify(a["logits"], a["dt"], a["B"], a["K"], a["V"], a["sb"], a["sk"], a["draft"], a["ocm"],
+                            f(a["tau"]), a["acc"], a["nxt"], a["resc"], a["rd"], a["rt"], a["diag"], a["ws"],
+                            a["wsb"], None)
+    assert verify(logits=null) == 1 and verify(draft=null) == 1 and verify(ocm=null) == 1 and verify(ws=null) == 1
+    assert verify(B=0) == 1 and verify(K=0) == 1 and verify(V=-5) == 1 and verify(dt=3) == 1
+    assert verify(K=33, sb=34 * 64) == 4
+    assert verify(tau=float("nan")) == 1 and verify(tau=-0.1) == 1 and verify(tau=float("inf")) == 1
+    assert verify(sk=63) == 1 and verify(sb=64) == 1
+    assert verify(wsb=16) == 5
+    assert verify(ws=ctypes.c_void_p(24)) == 5
+    assert L.csd_ocm_update(null, one, one, 4, None) == 1
+    assert L.csd_ocm_update(one, null, one, 4, None) == 1
+    assert L.csd_ocm_update(one, one, one, -1, None) == 1
+    out = ctypes.c_void_p()
+    assert L.csd_ocm_create(ctypes.byref(out), 1000, 6, 0) == 1      # not a power of two
+    assert L.csd_ocm_create(ctypes.byref(out), 32, 6, 0) == 1
+    assert L.csd_ocm_create(None, 1024, 6, 0) == 1
+    assert L.csd_set_tuning(1000, 0) == 1 and L.csd_set_tuning(0, 9) == 1 and L.csd_set_tuning(0, 0) == 0
+
+
+def test_binding_refuses_without_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("device present")
+    with pytest.raises(binding.CsdError):
+        binding.Ocm(1024)

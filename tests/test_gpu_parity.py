@@ -1,0 +1,362 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Bar: accepted lengths, next tokens, rescue masks, rejection lists, arg-max indices,
+maxima, gathered logits, look-up counts and the memory's (pair, count) set bit-exact;
+s, lse, score, p_d, p_t within 1e-5 relative (fp32 arithmetic against the fp64 oracle).
+Positions whose score lies within 1e-5 of tau are counted and reported; because the
+gate is decided exactly on both sides they are expected to agree as well.
+"""
+
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import csd_oracle as ORACLE
+from oracle import row_stats_c
+from paper_2604_13634_b200 import (CSD_BF16, CSD_F32, HostStep, Ocm, StepBuffers, csd_launch_shape, csd_set_tuning,
+                                   csd_step, csd_verify)
+from paper_2604_13634_b200.synth import WORKLOADS, Synth, logits_bits_numpy
+
+pytestmark = pytest.mark.gpu
+
+RTOL = 1e-5
+
+
+def _np_logits(z):
+    arr, is_bits = logits_bits_numpy(z)
+    if is_bits:
+        return ORACLE.bf16_bits_to_f64(arr).astype(np.float32), arr, True
+    return arr, arr, False
+
+
+def oracle_step(z, draft, mem, tau, update=True, use_c=True):
+    vals, raw, is_bits = _np_logits(z)
+    stats = None
+    if use_c and z.is_contiguous():
+        stats = row_stats_c.row_stats_batch(raw, is_bf16_bits=is_bits)
+    d = draft.cpu().numpy()
+    return ORACLE.step(vals, d, mem, tau, stats=stats) if update else ORACLE.verify(vals, d, mem, tau, stats=stats)
+
+
+def assert_close(name, got, ref, rtol=RTOL, atol=1e-37):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    both_nan = np.isnan(got) & np.isnan(ref)
+    bad = ~both_nan & ~(np.abs(got - ref) <= rtol * np.abs(ref) + atol)
+    assert not bad.any(), f"{name}: {int(bad.sum())} entries beyond {rtol}: got {got[bad][:4]} ref {ref[bad][:4]}"
+
+
+def compare(buf: StepBuffers, ref, check_diag=True):
+    g = lambda t: t.cpu().numpy()
+    for k in ("accept_len", "next_token", "rescued_mask"):
+        assert np.array_equal(g(getattr(buf, k)), ref[k]), k
+    assert np.array_equal(g(buf.rej_draft), ref["rej_draft"]), "rej_draft"
+    assert np.array_equal(g(buf.rej_target), ref["rej_target"]), "rej_target"
+    if check_diag and buf.diag is not None:
+        dg = {k: g(v) for k, v in buf.diag.items()}
+        assert np.array_equal(dg["t"], ref["t"]), "t"
+        assert np.array_equal(dg["m"].astype(np.float64), ref["m"]), "m"
+        assert np.array_equal(dg["cnt"].astype(np.int64) & 0xFFFFFFFF, ref["cnt"]), "cnt"
+        zd_ref = ref["zd"]
+        assert np.array_equal(np.isnan(dg["zd"]), np.isnan(zd_ref))
+        ok = ~np.isnan(zd_ref)
+        assert np.array_equal(dg["zd"][ok].astype(np.float64), zd_ref[ok]), "zd"
+        assert_close("s", dg["s"], ref["s"])
+        assert_close("lse", dg["lse"], ref["lse"])
+        assert_close("score", dg["score"], ref["score"])
+        assert_close("p_d", dg["p_d"], ref["p_d"])
+        assert_close("p_t", dg["p_t"], ref["p_t"])
+    return int(ref["near_tie"].sum())
+
+
+def compare_memory(ocm: Ocm, mem: ORACLE.OCM):
+    d, t, c = ocm.export()
+    rd, rt, rc = mem.export()
+    assert np.array_equal(d.numpy(), rd) and np.array_equal(t.numpy(), rt), "stored pairs differ"
+    assert np.array_equal(c.numpy(), rc), "counts differ"
+    st = ocm.stats()
+    assert st["n_keys"] == mem.n_keys and st["n_dropped"] == mem.n_dropped
+    return st
+
+
+def lockstep(wl, steps, tau, lam=None, seed=0, diag=True, prewarm_pairs=0, first_step=0, check_every=0):
+    lam = wl.lam if lam is None else lam
+    syn = Synth(wl, seed, "cuda")
+    ocm = Ocm(wl.ocm_slots, lam)
+    mem = ORACLE.OCM(wl.ocm_slots, lam)
+    if prewarm_pairs:
+        pd, pt = syn.prewarm_pairs(prewarm_pairs)
+        ocm.update(pd, pt)
+        mem.update(zip(pd.cpu().tolist(), pt.cpu().tolist()))
+        compare_memory(ocm, mem)
+    buf = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=diag)
+    near = 0
+    tot = dict(acc=0, resc=0)
+    for s in range(first_step, first_step + steps):
+        z, d = syn.step(s)
+        csd_step(z, d, ocm, tau, buf)
+        ref = oracle_step(z, d, mem, tau)
+        near += compare(buf, ref)
+        tot["acc"] += int(ref["accept_len"].sum())
+        tot["resc"] += int(ref["rescued_mask"].sum())
+        if check_every and (s + 1) % check_every == 0:
+            compare_memory(ocm, mem)
+    st = compare_memory(ocm, mem)
+    assert st["flags"] == 0
+    assert st["steps"] == steps and st["positions"] == steps * wl.B * wl.K
+    ocm.close()
+    return tot, near, st
+
+
+# ---------------------------------------------------------------------------------------
+# element-wise parity on small shapes: several tiles, ragged tails, both dtypes, both paths
+# ---------------------------------------------------------------------------------------
+SHAPES = [
+    (3, 4, 5000, torch.float32), (2, 5, 20000, torch.bfloat16), (1, 1, 1, torch.float32), (1, 1, 8, torch.bfloat16),
+    (2, 3, 4099, torch.float32),            # V not a multiple of 4: element-wise path
+    (2, 3, 4099, torch.bfloat16),
+    (4, 32, 3000, torch.bfloat16),          # K at the limit
+    (5, 2, 70001, torch.float32), (2, 2, 1024 * 33 + 8, torch.bfloat16), (1, 7, 262144, torch.float32),
+]
+
+
+def _random_inputs(B, K, V, dtype, seed, match_p=0.5):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    z = torch.randn(B, K + 1, V, generator=g, device="cuda") * 2
+    top = torch.randint(0, V, (B, K + 1), generator=g, device="cuda")
+    z.scatter_add_(2, top.unsqueeze(-1), torch.full((B, K + 1, 1), 5.0, device="cuda"))
+    z = z.to(dtype)
+    arg = z[:, :K].float().argmax(dim=2)
+    rnd = torch.randint(0, V, (B, K), generator=g, device="cuda")
+    near = (arg + torch.randint(0, 3, (B, K), generator=g, device="cuda")) % V
+    pick = torch.rand(B, K, generator=g, device="cuda")
+    draft = torch.where(pick < match_p, arg, torch.where(pick < match_p + 0.25, near, rnd)).to(torch.int32)
+    return z.contiguous(), draft.contiguous()
+
+
+@pytest.mark.parametrize("B,K,V,dtype", SHAPES)
+def test_elementwise_parity_small(B, K, V, dtype):
+    ocm = Ocm(1024, 1)
+    mem = ORACLE.OCM(1024, 1)
+    buf = StepBuffers(B, K, V, dtype, diag=True)
+    for rep in range(4):
+        z, d = _random_inputs(B, K, V, dtype, seed=100 + rep)
+        if rep >= 2:
+            d = _random_inputs(B, K, V, dtype, seed=100 + rep - 2)[1]     # revisit pairs: rescues happen
+            z = _random_inputs(B, K, V, dtype, seed=100 + rep - 2)[0]
+        csd_step(z, d, ocm, 1e-4, buf)
+        compare(buf, oracle_step(z, d, mem, 1e-4, use_c=(rep % 2 == 0)))
+    compare_memory(ocm, mem)
+    ocm.close()
+
+
+def test_strided_and_misaligned_views():
+    B, K, V = 3, 4, 6000
+    for dtype in (torch.float32, torch.bfloat16):
+        big, d = _random_inputs(B, K, V + 24, dtype, seed=7)
+        for view in (big[:, :, :V], big[:, :, 1:V + 1], big[:, :, 8:V + 8]):
+            d = d % V
+            ocm = Ocm(256, 0)
+            mem = ORACLE.OCM(256, 0)
+            buf = StepBuffers(B, K, V, dtype, diag=True)
+            csd_step(view, d, ocm, 0.05, buf)
+            ref = ORACLE.step(view.float().cpu().numpy(), d.cpu().numpy(), mem, 0.05)
+            compare(buf, ref)
+            compare_memory(ocm, mem)
+            ocm.close()
+
+
+def test_ties_infinities_and_constant_rows():
+    B, K, V = 4, 3, 9000
+    z = torch.zeros(B, K + 1, V, device="cuda", dtype=torch.bfloat16)
+    z[0] = 1.5                                   # constant rows: arg-max 0
+    z[1, :, 4000:] = 2.0                         # plateau: lowest index 4000
+    z[1, 1, 8999] = 2.0
+    z[2] = float("-inf")
+    z[2, :, 77] = -3.0                           # single finite value
+    z[2, 1, 5000] = -3.0                         # tie with 77: lowest wins
+    z[3] = torch.randn(K + 1, V, device="cuda").to(torch.bfloat16)      # real bf16 ties are likely
+    d = torch.tensor([[0, 5, 0], [4000, 8999, 3], [77, 5000, 78], [1, 2, 3]], dtype=torch.int32, device="cuda")
+    ocm = Ocm(256, 0)
+    mem = ORACLE.OCM(256, 0)
+    buf = StepBuffers(B, K, V, torch.bfloat16, diag=True)
+    csd_step(z, d, ocm, 0.9, buf)
+    ref = oracle_step(z, d, mem, 0.9)
+    compare(buf, ref)
+    assert buf.diag["t"][0].tolist() == [0, 0, 0, 0] and buf.diag["t"][1, 0].item() == 4000
+    assert buf.accept_len.tolist()[:3] == [3, 2, 2]       # score 1 at a tie passes tau = 0.9
+    compare_memory(ocm, mem)
+    assert ocm.stats()["flags"] == 0
+    ocm.close()
+
+
+def test_bad_inputs_flag_and_never_rescue():
+    B, K, V = 2, 4, 5000
+    z, d = _random_inputs(B, K, V, torch.float32, seed=3, match_p=1.0)
+    d[0, 1] = V
+    d[1, 0] = -7
+    ocm = Ocm(256, 0)
+    mem = ORACLE.OCM(256, 0)
+    buf = StepBuffers(B, K, V, torch.float32, diag=True)
+    csd_step(z, d, ocm, 0.0, buf)
+    ref = oracle_step(z, d, mem, 0.0)
+    compare(buf, ref)
+    assert buf.accept_len.tolist() == [1, 0]
+    st = compare_memory(ocm, mem)
+    assert st["flags"] == 2 and st["n_keys"] == 0
+    # a NaN logit raises the NaN flag and the launch still completes
+    z[1, 2, 17] = float("nan")
+    csd_verify(z, d.clamp(0, V - 1), ocm, 0.0, buf)
+    torch.cuda.synchronize()
+    assert ocm.stats()["flags"] & 1
+    ocm.close()
+
+
+def test_verify_leaves_memory_alone_and_is_deterministic():
+    wl = dataclasses.replace(WORKLOADS["batched_serving"], B=4)
+    syn = Synth(wl, 1, "cuda")
+    ocm = Ocm(4096, 1)
+    z, d = syn.step(0)
+    buf = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True)
+    csd_step(z, d, ocm, 0.3, buf)
+    before = [x.clone() for x in ocm.export()]
+    csd_verify(z, d, ocm, 0.3, buf)
+    first = {k: v.clone() for k, v in buf.diag.items()}
+    outs = [buf.accept_len.clone(), buf.next_token.clone(), buf.rescued_mask.clone()]
+    csd_verify(z, d, ocm, 0.3, buf)
+    after = ocm.export()
+    assert all(torch.equal(a, b) for a, b in zip(before, after))
+    for k, v in buf.diag.items():                       # bit-identical, including the sums
+        assert torch.equal(v.view(torch.int32), first[k].view(torch.int32)), k
+    assert torch.equal(outs[0], buf.accept_len) and torch.equal(outs[1], buf.next_token)
+    assert torch.equal(outs[2], buf.rescued_mask)
+    ocm.close()
+
+
+# ---------------------------------------------------------------------------------------
+# lock-step runs of the five workloads (bounded step counts; the oracle is the slow side)
+# ---------------------------------------------------------------------------------------
+def test_workload_tiny_lockstep():
+    tot, near, st = lockstep(WORKLOADS["tiny"], steps=1000, tau=0.3, check_every=250)
+    assert st["rescues"] == tot["resc"] and tot["resc"] > 0
+    print(f"tiny: accepted {tot['acc']} rescued {tot['resc']} near-ties {near} keys {st['n_keys']}")
+
+
+@pytest.mark.parametrize("tau", [0.1, 0.3, 0.5])
+def test_workload_single_stream_lockstep(tau):
+    wl = WORKLOADS["single_stream"]
+    tot, near, st = lockstep(wl, steps=150, tau=tau, prewarm_pairs=4000)
+    assert tot["resc"] > 0
+    print(f"single_stream tau={tau}: accepted {tot['acc']} rescued {tot['resc']} near-ties {near}")
+
+
+def test_workload_batched_serving_lockstep():
+    tot, near, st = lockstep(WORKLOADS["batched_serving"], steps=12, tau=0.3, lam=2)
+    assert tot["resc"] > 0
+    print(f"batched_serving: accepted {tot['acc']} rescued {tot['resc']} near-ties {near}")
+
+
+@pytest.mark.parametrize("tau", [0.2, 0.4])
+def test_workload_large_batch_lockstep(tau):
+    wl = WORKLOADS["large_batch"]
+    tot, near, st = lockstep(wl, steps=2, tau=tau, prewarm_pairs=200000, diag=True)
+    assert tot["resc"] > 0
+    print(f"large_batch tau={tau}: accepted {tot['acc']} rescued {tot['resc']} near-ties {near}")
+
+
+def test_workload_ocm_contention_lockstep():
+    wl = WORKLOADS["ocm_contention"]
+    tot, near, st = lockstep(wl, steps=16, tau=0.3, check_every=4)
+    assert tot["resc"] > 0
+    print(f"ocm_contention: accepted {tot['acc']} rescued {tot['resc']} near-ties {near} keys {st['n_keys']}")
+
+
+def test_contention_fills_the_table():
+    """The contention workload with a small table: the run crosses all three update
+    regimes (room, canonical admission, full) and the memory still matches the oracle."""
+    wl = dataclasses.replace(WORKLOADS["ocm_contention"], B=16, V=32768, ocm_slots=512)
+    tot, near, st = lockstep(wl, steps=80, tau=0.3, check_every=1, diag=False)
+    assert st["n_keys"] == 256 and st["n_dropped"] > 0
+
+
+# ---------------------------------------------------------------------------------------
+# the memory on its own
+# ---------------------------------------------------------------------------------------
+def test_update_kernel_regimes_and_import_export():
+    g = torch.Generator(device="cuda").manual_seed(5)
+    for n_slots, n, vocab in ((1 << 16, 200000, 300), (256, 5000, 40), (1024, 3000, 25), (64, 31, 1000), (64, 40, 1000)):
+        ocm = Ocm(n_slots, 6)
+        mem = ORACLE.OCM(n_slots, 6)
+        for rep in range(3):
+            d = torch.randint(0, vocab, (n,), generator=g, device="cuda", dtype=torch.int32)
+            t = torch.randint(0, vocab, (n,), generator=g, device="cuda", dtype=torch.int32)
+            d[::17] = -1                                    # placeholders are skipped
+            ocm.update(d, t)
+            mem.update(zip(d.cpu().tolist(), t.cpu().tolist()))
+            compare_memory(ocm, mem)
+        # export -> fresh table -> import reproduces the contents
+        d, t, c = ocm.export()
+        other = Ocm(n_slots, 6)
+        other.import_(d.to(torch.int32).cuda(), t.to(torch.int32).cuda(), c.to(torch.int32).cuda())
+        d2, t2, c2 = other.export()
+        assert torch.equal(d, d2) and torch.equal(t, t2) and torch.equal(c, c2)
+        # saturation
+        one = torch.tensor([int(d[0])], dtype=torch.int32, device="cuda")
+        two = torch.tensor([int(t[0])], dtype=torch.int32, device="cuda")
+        big = torch.tensor([-2], dtype=torch.int32, device="cuda")          # 2^32 - 2 as bits
+        other.import_(one, two, big)
+        other.import_(one, two, big)
+        d3, t3, c3 = other.export()
+        assert int(c3[0]) == 2**32 - 1 and other.stats()["flags"] & 8
+        other.reset()
+        assert other.stats()["n_keys"] == 0 and other.export()[0].numel() == 0
+        ocm.close(); other.close()
+
+
+def test_host_entry_point_matches_device_entry_point():
+    wl = dataclasses.replace(WORKLOADS["batched_serving"], B=6)
+    syn = Synth(wl, 2, "cuda")
+    a, b = Ocm(4096, 1), Ocm(4096, 1)
+    buf = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype)
+    host = HostStep(wl.B, wl.K, wl.V, wl.torch_dtype)
+    for s in range(5):
+        z, d = syn.step(s)
+        csd_step(z, d, a, 0.3, buf)
+        acc, nxt, resc = host(z.cpu().pin_memory(), d.cpu().pin_memory(), b, 0.3)
+        assert torch.equal(acc, buf.accept_len.cpu()) and torch.equal(nxt, buf.next_token.cpu())
+        assert torch.equal(resc, buf.rescued_mask.cpu())
+    assert all(torch.equal(x, y) for x, y in zip(a.export(), b.export()))
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("tile_bytes,ctas", [(4096, 1), (8192, 2), (32768, 4), (65536, 3)])
+def test_parity_under_other_tilings(tile_bytes, ctas):
+    try:
+        csd_set_tuning(tile_bytes, ctas)
+        wl = dataclasses.replace(WORKLOADS["ocm_contention"], B=8)
+        assert csd_launch_shape(wl.B, wl.K, wl.V, CSD_BF16)["tile_elems"] == tile_bytes // 2
+        lockstep(wl, steps=3, tau=0.3, lam=1)
+        wl = dataclasses.replace(WORKLOADS["large_batch"], B=4)
+        assert csd_launch_shape(wl.B, wl.K, wl.V, CSD_F32)["tile_elems"] == tile_bytes // 4
+        lockstep(wl, steps=2, tau=0.2, lam=1)
+    finally:
+        csd_set_tuning(0, 0)
+
+
+def test_long_row_many_tiles_per_warp():
+    """One row far longer than the machine has warps x tiles: exercises the 32-tile batches."""
+    try:
+        csd_set_tuning(4096, 1)
+        B, K, V = 48, 1, 1 << 20            # 96 rows x 1024 tiles = 98304 tiles > 32 x 1184 warps
+        z, d = _random_inputs(B, K, V, torch.float32, seed=11)
+        ocm = Ocm(256, 0)
+        mem = ORACLE.OCM(256, 0)
+        buf = StepBuffers(B, K, V, torch.float32, diag=True)
+        csd_step(z, d, ocm, 0.01, buf)
+        compare(buf, oracle_step(z, d, mem, 0.01))
+        compare_memory(ocm, mem)
+        ocm.close()
+    finally:
+        csd_set_tuning(0, 0)
