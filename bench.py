@@ -1,0 +1,426 @@
+#!/usr/bin/env python
+"""Benchmark of the CSD verification step (csd_step: verify + memory update, one launch).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one pass of the whole hot path over one synthetic batch: the streaming
+max/arg-max/sum-exp over logits[B,K+1,V], the match test, the OCM look-up, the gate of
+Eq. 3, the prefix scan, and the memory update.  Rank 0 prints ONE JSON line:
+
+  value     verified draft positions per second (B*K*steps / time), inputs resident in HBM,
+            timed with CUDA events on the launching stream, max over ranks;
+  e2e       the same metric through csd_step_host: logits and draft in pinned host memory,
+            host->device and device->host copies inside the timed region;
+  roofline  achieved logit bytes per second of the step kernel against the measured HBM copy
+            bandwidth of this machine;
+  cpu_baseline  the CPU oracle timed on this machine's cores on a bounded sample of the workload.
+
+With N > 1 every rank runs an independent replica (own batch, own memory): the path has no
+exchange step, so there is no data-path collective; torch.distributed only carries the
+barrier and the max over ranks of the elapsed time.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verified_draft_positions_per_sec"
+UNIT = "positions/s"
+FALLBACK_HBM_GBS = 6650.0            # earlier measurement on this machine, used when no measured file exists
+DEFAULT_WORKLOAD = "large_batch"
+# DRAM bytes per launch of the step kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum); a workload is absent where no capture of the current kernel exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def workload_config(wl, tau, extra=None):
+    cfg = {"workload": f"{wl.name}: B={wl.B} K={wl.K} V={wl.V} {wl.dtype} logits, OCM {wl.ocm_slots} slots, "
+                       f"lambda={wl.lam}, tau={tau}",
+           "B": wl.B, "K": wl.K, "V": wl.V, "ocm_slots": wl.ocm_slots, "tau": tau, "lambda": wl.lam,
+           "logit_bytes_per_step": wl.logit_bytes}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+def reduce_over_ranks(seconds: float, units: float, dist=None, device=None):
+    """Whole-job figures from per-rank ones: elapsed = max over ranks, units = sum over ranks."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return seconds, units
+    import torch
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ---------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# ---------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self._nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+        self.period = period_s
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------------------
+# the CPU oracle leg (also the whole of --impl reference)
+# ---------------------------------------------------------------------------------------
+class OracleRunner:
+    """The CPU oracle on `rows_b` batch rows of the workload (CPU-generated inputs, seed 0)."""
+
+    def __init__(self, wl, tau, rows_b):
+        import dataclasses
+        from oracle import csd_oracle, row_stats_c
+        from paper_2604_13634_b200.synth import Synth, logits_bits_numpy
+        self.o, self.rs = csd_oracle, row_stats_c
+        self.wl = dataclasses.replace(wl, B=rows_b)
+        self.tau = tau
+        self.cores = row_stats_c.max_threads()
+        syn = Synth(self.wl, 0, "cpu")
+        self.mem = csd_oracle.OCM(wl.ocm_slots, wl.lam)
+        self.inputs = []
+        for s in range(2):
+            z, d = syn.step(s)
+            raw, is_bits = logits_bits_numpy(z)
+            vals = csd_oracle.bf16_bits_to_f64(raw).astype("float32") if is_bits else raw
+            self.inputs.append((vals, raw, is_bits, d.numpy()))
+        self.done = 0
+
+    def step(self):
+        vals, raw, is_bits, d = self.inputs[self.done % 2]
+        stats = self.rs.row_stats_batch(raw, is_bf16_bits=is_bits)
+        self.o.step(vals, d, self.mem, self.tau, stats=stats)
+        self.done += 1
+
+    def timed(self, n):
+        t0 = time.perf_counter()
+        for _ in range(n):
+            self.step()
+        return time.perf_counter() - t0
+
+
+def oracle_row_seconds(wl, tau):
+    """Seconds the oracle needs per batch row of this workload (calibration on a few rows)."""
+    rows = min(wl.B, 4)
+    r = OracleRunner(wl, tau, rows)
+    r.timed(1)
+    return r.timed(2) / (2 * rows)
+
+
+def time_oracle(wl, tau, budget_s=15.0):
+    """Oracle positions/s on the host cores over a bounded sample of the workload."""
+    t_row = oracle_row_seconds(wl, tau)
+    rows_b = wl.B if t_row * wl.B <= budget_s / 3 else max(1, int(budget_s / 3 / t_row))
+    n = max(2, min(200, int(budget_s / (t_row * rows_b))))
+    r = OracleRunner(wl, tau, rows_b)
+    sec = r.timed(n)
+    return {"steps": n, "rows_b": rows_b, "seconds": sec, "positions_per_s": rows_b * wl.K * n / sec, "cores": r.cores}
+
+
+def run_reference(args, wl, tau):
+    """--impl reference: the oracle as it stands, timed on the host cores.  Each bench step
+    is one oracle step over a bounded number of batch rows, sized so that the whole run
+    (warm-up included) stays near two minutes."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    t_row = oracle_row_seconds(wl, tau)
+    total = args.steps + args.warmup
+    rows_b = max(1, min(wl.B, int(120.0 / (total * t_row))))
+    r = OracleRunner(wl, tau, rows_b)
+    r.timed(args.warmup)
+    sec = r.timed(args.steps)
+    value = rows_b * wl.K * args.steps / sec
+    sample = f"each step = the oracle on {rows_b} of the workload's {wl.B} batch rows (K+1 logit rows each)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(wl, tau),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": r.cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------
+# the GPU leg
+# ---------------------------------------------------------------------------------------
+class Bench:
+    def __init__(self, wl, tau, device, seed=0):
+        import torch
+        import paper_2604_13634_b200 as pkg
+        from paper_2604_13634_b200.synth import Synth
+        self.torch, self.pkg, self.wl, self.tau = torch, pkg, wl, tau
+        self.device = device
+        l2 = torch.cuda.get_device_properties(device).L2_cache_size
+        self.ring_len = max(2, math.ceil(2 * l2 / wl.logit_bytes) + 1)
+        syn = Synth(wl, seed, device)
+        self.ring = [syn.step(s) for s in range(self.ring_len)]
+        self.ocm = pkg.Ocm(wl.ocm_slots, wl.lam, device.index)
+        kind, n = wl.prewarm
+        if kind == "pairs":
+            self.ocm.update(*syn.prewarm_pairs(n))
+        self.buf = pkg.StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, device=device)
+        if kind == "steps":
+            for s in range(n):
+                z, d = self.ring[s % self.ring_len]
+                pkg.csd_step(z, d, self.ocm, tau, self.buf)
+        torch.cuda.synchronize(device)
+        self.graph = None
+
+    def step(self, i):
+        z, d = self.ring[i % self.ring_len]
+        self.pkg.csd_step(z, d, self.ocm, self.tau, self.buf)
+
+    def capture(self):
+        """A CUDA graph of ring_len consecutive steps (the launches are captured, not changed)."""
+        torch = self.torch
+        side = torch.cuda.Stream(self.device)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.step(0)
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(self.ring_len):
+                self.step(i)
+        self.graph = g
+
+    def run(self, steps):
+        """Enqueue `steps` steps: whole-graph replays, then the remainder eagerly."""
+        if self.graph is not None:
+            while steps >= self.ring_len:
+                self.graph.replay()
+                steps -= self.ring_len
+        for i in range(steps):
+            self.step(i)
+
+    def timed(self, steps):
+        torch = self.torch
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        self.run(steps)
+        b.record()
+        b.synchronize()
+        return a.elapsed_time(b) * 1e-3
+
+
+def time_e2e(wl, tau, device, steps):
+    """csd_step_host: pinned host inputs, copies inside the timed region."""
+    import torch
+    import paper_2604_13634_b200 as pkg
+    from paper_2604_13634_b200.synth import Synth
+    syn = Synth(wl, 0, device)
+    host = []
+    for s in range(2):
+        z, d = syn.step(s)
+        host.append((z.cpu().pin_memory(), d.cpu().pin_memory()))
+    del z, d
+    ocm = pkg.Ocm(wl.ocm_slots, wl.lam, device.index)
+    hs = pkg.HostStep(wl.B, wl.K, wl.V, wl.torch_dtype, device=device)
+    for i in range(2):
+        hs(*host[i % 2], ocm, tau)
+    torch.cuda.synchronize(device)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(steps):
+        hs(*host[i % 2], ocm, tau)
+    b.record()
+    b.synchronize()
+    sec = a.elapsed_time(b) * 1e-3
+    ocm.close()
+    h2d = wl.logit_bytes + wl.B * wl.K * 4
+    d2h = wl.B * 8 + wl.B * wl.K
+    return {"value": wl.B * wl.K * steps / sec, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "steps": steps, "ms_per_step": 1e3 * sec / steps}
+
+
+def run_ours(args, wl, tau):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2604_13634_b200 as pkg
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    pkg.lib()
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    bench = Bench(wl, tau, device, seed=rank)
+    use_graph = not args.eager
+    if use_graph:
+        bench.capture()
+    warm = max(args.warmup, 3)
+    bench.run(warm)
+    torch.cuda.synchronize(device)
+
+    sampler = ClockSampler(local)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize(device)
+    sampler.start()
+    sec = bench.timed(args.steps)
+    torch.cuda.synchronize(device)
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    sec, positions = reduce_over_ranks(sec, wl.B * wl.K * args.steps, dist if world > 1 else None, device)
+
+    st = bench.ocm.stats()
+    e2e = time_e2e(wl, tau, device, steps=max(3, min(args.steps, args.e2e_steps)))
+    if world > 1:
+        _, e2e["value"] = reduce_over_ranks(0.0, e2e["value"], dist, device)
+
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        per_launch_s = sec / args.steps
+        achieved = wl.logit_bytes / per_launch_s / 1e9
+        shape = pkg.csd_launch_shape(wl.B, wl.K, wl.V, 0 if wl.dtype == "f32" else 1)
+        line = {
+            "metric": METRIC, "value": positions / sec, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warm, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": workload_config(wl, tau, {
+                "steps_per_s": args.steps * world / sec, "parallelism": f"replicas x{world}",
+                "l2_policy": f"ring of {bench.ring_len} distinct step inputs "
+                             f"({bench.ring_len * wl.logit_bytes / 1e6:.0f} MB, > 2x L2)",
+                "launch": ("CUDA graph of %d steps replayed" % bench.ring_len) if use_graph else "eager",
+                "kernel_shape": shape}),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_source": f"of {peak_kind}",
+                         "kernel": "csd_step_kernel", "bytes_per_launch": wl.logit_bytes,
+                         "frac_of_nominal_8TBs": achieved / 8000.0},
+            "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks,
+            "ocm": {k: st[k] for k in ("n_keys", "n_dropped", "steps", "matches", "rescues", "rejections", "flags")},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            r = time_oracle(wl, tau)
+            line["cpu_baseline"] = {"value": r["positions_per_s"], "unit": UNIT, "cores": r["cores"], "kind": "oracle",
+                                    "sample": f"{r['steps']} oracle steps over {r['rows_b']} of the workload's {wl.B} "
+                                              f"batch rows (CPU-generated inputs, same recipe) in {r['seconds']:.1f} s"}
+        if args.extras and world == 1:
+            line["other_workloads"] = run_extras(device, wl.name, peak)
+        print(json.dumps(line), flush=True)
+    bench.ocm.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_extras(device, skip, peak):
+    """Short device-resident runs of the other workloads (extra keys, not bench lines)."""
+    import torch
+    from paper_2604_13634_b200.synth import WORKLOADS
+    out = {}
+    for name in ("batched_serving", "large_batch", "ocm_contention", "single_stream", "tiny"):
+        if name == skip:
+            continue
+        wl = WORKLOADS[name]
+        b = Bench(wl, wl.taus[0], device)
+        b.capture()
+        b.run(50)
+        torch.cuda.synchronize(device)
+        steps = 4000 if wl.logit_bytes > 100e6 else 20000
+        steps -= steps % b.ring_len
+        sec = b.timed(steps)
+        out[name] = {"positions_per_s": wl.B * wl.K * steps / sec, "us_per_step": 1e6 * sec / steps,
+                     "achieved_GBs": wl.logit_bytes * steps / sec / 1e9,
+                     "frac_of_measured_peak": wl.logit_bytes * steps / sec / 1e9 / peak, "steps": steps}
+        b.ocm.close()
+        del b
+        torch.cuda.empty_cache()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--tau", type=float, default=None)
+    ap.add_argument("--eager", action="store_true", help="launch every step from Python instead of replaying a graph")
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--extras", action="store_true", help="also time the other workloads (extra keys, same line)")
+    args = ap.parse_args()
+
+    from paper_2604_13634_b200.synth import WORKLOADS
+    wl = WORKLOADS[args.workload]
+    tau = wl.taus[0] if args.tau is None else args.tau
+    if args.impl == "reference":
+        run_reference(args, wl, tau)
+    else:
+        run_ours(args, wl, tau)
+
+
+if __name__ == "__main__":
+    main()
