@@ -45,37 +45,42 @@ struct Shape {
     int grid;
     int tile_elems;
     int n_split;
-    long long total_tiles;
+    int total_tiles;
 };
 
 inline int elt_bytes(csd_dtype_t dt) { return dt == CSD_F32 ? 4 : 2; }
 
 bool shape_ok(int B, int K, int V, csd_dtype_t dt)
 {
-    return B > 0 && K > 0 && V > 0 && K <= CSD_MAX_K && (dt == CSD_F32 || dt == CSD_BF16) &&
-           static_cast<long long>(B) * (K + 1) < (1ll << 31);
+    if (!(B > 0 && K > 0 && V > 0 && K <= CSD_MAX_K && (dt == CSD_F32 || dt == CSD_BF16))) return false;
+    // tile and position indices are 32-bit: the smallest tile is 4 KiB
+    const long long rows = static_cast<long long>(B) * (K + 1);
+    const long long tiles_max = rows * ((static_cast<long long>(V) * elt_bytes(dt) + 4095) / 4096);
+    return tiles_max < (1ll << 31) && static_cast<long long>(B) * K < (1ll << 31);
 }
 
-// Tiles are whole warp iterations (32 lanes x 8 x 16 bytes = 4 KiB).  Small problems
-// get 4 KiB tiles so that every warp of the machine has work; large ones get up to
-// 32 KiB so that a batch row is described by few partials.
+// Tiles are whole warp iterations (32 lanes x 8 x 16 bytes = 4 KiB).  A logit row is cut
+// into at most 32 tiles, so that a batch row is described by few partials; when that
+// leaves more than 8 tiles per warp of the persistent grid the tiles are doubled (up to
+// 64 KiB), which amortises the per-tile publication.
 Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
 {
     const int eb = elt_bytes(dt);
     const int ctas_per_sm = g_ctas_per_sm_override > 0 ? g_ctas_per_sm_override : 4;
     const long long workers = static_cast<long long>(sm_count()) * ctas_per_sm * kWarps;
     const long long rows = static_cast<long long>(B) * (K + 1);
-    const long long total_bytes = rows * V * eb;
-    long long tile_bytes = 4096;
+    const long long row_bytes = static_cast<long long>(V) * eb;
+    long long tile_bytes;
     if (g_tile_bytes_override > 0) {
         tile_bytes = g_tile_bytes_override;
     } else {
-        while (tile_bytes < 32768 && total_bytes / (tile_bytes * 2) >= 4 * workers) tile_bytes *= 2;
+        tile_bytes = ((row_bytes + 31) / 32 + 4095) / 4096 * 4096;
+        while (tile_bytes < 65536 && rows * ((row_bytes + tile_bytes - 1) / tile_bytes) > 8 * workers) tile_bytes *= 2;
     }
     Shape s;
     s.tile_elems = static_cast<int>(tile_bytes / eb);
     s.n_split = (V + s.tile_elems - 1) / s.tile_elems;
-    s.total_tiles = rows * s.n_split;
+    s.total_tiles = static_cast<int>(rows * s.n_split);
     long long blocks = static_cast<long long>(sm_count()) * ctas_per_sm;
     const long long needed = (s.total_tiles + kWarps - 1) / kWarps;
     if (needed < blocks) blocks = needed;
@@ -86,14 +91,15 @@ Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t partials_off, b_ticket_off, g_ticket_off, total;
+    size_t partials_off, hint_off, b_ticket_off, g_ticket_off, total;
 };
 
 WorkspaceLayout ws_layout(int B, int K, const Shape &s)
 {
     WorkspaceLayout w;
     w.partials_off = 0;
-    w.b_ticket_off = align_up(static_cast<size_t>(B) * (K + 1) * s.n_split * sizeof(Partial), 256);
+    w.hint_off = align_up(static_cast<size_t>(B) * (K + 1) * s.n_split * sizeof(Partial), 256);
+    w.b_ticket_off = align_up(w.hint_off + static_cast<size_t>(B) * K * sizeof(long long), 256);
     w.g_ticket_off = align_up(w.b_ticket_off + static_cast<size_t>(B) * sizeof(unsigned int), 16);
     w.total = align_up(w.g_ticket_off + 16, 256);
     return w;
@@ -142,6 +148,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     if (diag) p.diag = *diag;
     char *ws = static_cast<char *>(workspace);
     p.partials = reinterpret_cast<Partial *>(ws + w.partials_off);
+    p.slot_hint = reinterpret_cast<long long *>(ws + w.hint_off);
     p.b_ticket = reinterpret_cast<unsigned int *>(ws + w.b_ticket_off);
     p.g_ticket = reinterpret_cast<unsigned int *>(ws + w.g_ticket_off);
     p.tile_elems = s.tile_elems;

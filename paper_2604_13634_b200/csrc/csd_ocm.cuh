@@ -130,6 +130,30 @@ __device__ __forceinline__ void ocm_insert_or_add(const OcmView &tb, unsigned lo
     atomicOr(&tb.stats->flags, 0x4u);
 }
 
+// Slot of `key`, claiming an empty slot (count 0) if the key is absent.  A slot with
+// count 0 reads as "absent" to every look-up, so a reservation is invisible until the
+// count is raised.  The caller has established that there is room.  -1 only if the
+// probe wrapped around (flagged).
+__device__ __forceinline__ long long ocm_reserve(const OcmView &tb, unsigned long long key)
+{
+    unsigned long long slot = mix64(key) & tb.mask;
+    for (unsigned long long probe = 0; probe <= tb.mask; ++probe) {
+        unsigned long long *kp = &tb.slots[slot].key;
+        unsigned long long k = *reinterpret_cast<volatile unsigned long long *>(kp);
+        if (k == kEmptyKey) {
+            k = atomicCAS(kp, kEmptyKey, key);
+            if (k == kEmptyKey) {
+                atomicAdd(&tb.stats->n_keys, 1ull);
+                k = key;
+            }
+        }
+        if (k == key) return static_cast<long long>(slot);
+        slot = (slot + 1) & tb.mask;
+    }
+    atomicOr(&tb.stats->flags, 0x4u);
+    return -1;
+}
+
 // Increment if present, else count a dropped occurrence (table full: nothing is admitted).
 __device__ __forceinline__ void ocm_add_or_drop(const OcmView &tb, unsigned long long key, unsigned int w)
 {

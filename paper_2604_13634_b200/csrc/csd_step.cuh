@@ -4,21 +4,25 @@
 //
 // Work decomposition
 //   * The R = B*(K+1) logit rows are cut into tiles of `tile_elems` contiguous
-//     elements; a tile is reduced by ONE WARP on its own (no block barrier anywhere in
-//     the streaming phase).  Warps are persistent workers: tile t goes to block
-//     t mod G, warp (t / G) mod 8, so every SM gets the same number of tiles +-1.
+//     elements (at most ~32 tiles per row); a tile is reduced by ONE WARP on its own:
+//     there is no block barrier anywhere.  Warps are persistent workers: tile t goes to
+//     block t mod G, warp (t / G) mod 8, so every SM gets the same number of tiles +-1
+//     and batch rows complete in index order while later ones are still streaming.
 //   * A lane keeps 8 x 16 bytes in flight; a tile is reduced with a running maximum,
 //     an integer reference exponent and four independent sum accumulators; only the
 //     iteration in which the maximum last improved is remembered, and the exact
 //     lowest arg-max index is recovered by re-reading that one iteration (an L2 hit).
-//   * A warp keeps the partial results of up to 32 tiles in registers (lane j holds
-//     tile j), then publishes them together: one store per lane, ONE fence per warp,
-//     one ticket atomic per tile on its batch row's arrival counter.
-//   * Whichever warp delivers the last tile of a batch row finalises that row: a
-//     segmented warp scan folds the row's partials in a fixed order (bit-reproducible
-//     sums), lanes 0..K-1 take the per-position decisions, a ballot gives the
-//     accepted prefix.  The warp finalising the last batch row applies the step's
-//     rejections to the memory, so every look-up of the step saw the step-start table.
+//   * After each tile lane 0 stores the partial, fences, and takes a ticket on the
+//     batch row's arrival counter.  Whichever warp delivers the last tile of a batch
+//     row finalises it: the row's partials are prefetched together and folded by a
+//     segmented warp scan in a fixed order (bit-reproducible sums), lanes 0..K-1 take
+//     the per-position decisions, a ballot gives the accepted prefix.
+//   * Memory update without a second probe: the look-up already found each recorded
+//     pair's slot (absent pairs get an empty slot reserved with count 0, which no
+//     look-up can tell from "absent"), and leaves it as a hint.  The warp finalising
+//     the LAST batch row then only adds 1 to the hinted slots, so every look-up of the
+//     step saw the step-start counts.  Near the key limit, where admission order
+//     matters, that warp falls back to the canonical-order path.
 //   * Nothing ever waits for another block: arrival counters only, so no launch can hang.
 #pragma once
 
@@ -45,12 +49,17 @@ struct StepParams {
     int *rej_t;
     csd_diag_t diag;
     Partial *partials;       // [R * n_split]
+    long long *slot_hint;    // [B * K] slot of each recorded pair (see kHint*)
     unsigned int *b_ticket;  // [B]
     unsigned int *g_ticket;  // [1]
     int tile_elems;
     int n_split;             // tiles per logit row
-    long long total_tiles;
+    int total_tiles;
 };
+
+constexpr long long kHintNone = -1;          // nothing to record at this position
+constexpr long long kHintAbsent = -2;        // recorded pair not in the table and no slot reserved
+constexpr long long kHintCareful = 1ll << 62; // count close to saturation: add with the wrap check
 
 // ---- element access policies ---------------------------------------------------------
 
@@ -199,7 +208,7 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
     U v[kUnroll];
 
-    auto consume = [&](int it) {
+    auto consume = [&](const U (&v)[kUnroll], int it) {
         U mx = L::vmax(L::vmax(L::vmax(v[0], v[1]), L::vmax(v[2], v[3])),
                        L::vmax(L::vmax(v[4], v[5]), L::vmax(v[6], v[7])));
         const float bmax = L::hmax(mx);
@@ -224,7 +233,7 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
     for (int it = 0; it < nfull; ++it) {
 #pragma unroll
         for (int k = 0; k < kUnroll; ++k) v[k] = L::load(base, (it * kUnroll + k) * 32 + lane);
-        consume(it);
+        consume(v, it);
     }
     if (nfull * kPerIter < nunits) {
 #pragma unroll
@@ -232,7 +241,7 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
             const int u = (nfull * kUnroll + k) * 32 + lane;
             v[k] = u < nunits ? L::load(base, u) : L::neg_inf();
         }
-        consume(nfull);
+        consume(v, nfull);
     }
 
     // warp maximum, then everything is rescaled to the warp's reference exponent
@@ -275,6 +284,19 @@ struct RowScratch {
     int t[CSD_MAX_K + 1];
 };
 
+enum UpdateRegime { kRegimeRoom = 0, kRegimeFull = 1, kRegimeTransition = 2 };
+
+// Which of the three update regimes this step is in.  n_keys_start is written when the
+// previous update finished, so every warp of the launch computes the same answer.
+__device__ __forceinline__ int update_regime(const StepParams &p)
+{
+    const unsigned long long nk = __ldcg(&p.ocm.stats->n_keys_start);
+    const unsigned long long n = static_cast<unsigned long long>(p.B) * p.K;
+    if (nk + n <= p.ocm.key_limit) return kRegimeRoom;
+    if (nk >= p.ocm.key_limit) return kRegimeFull;
+    return kRegimeTransition;
+}
+
 template <typename L>
 __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScratch &rs)
 {
@@ -299,49 +321,61 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
     }
 
     // S1 (second half): fold the K+1 rows' partials with a segmented inclusive scan,
-    // 32 partials at a time, always in the same order.
+    // 32 partials at a time, always in the same order; up to 256 are fetched at once.
     Partial carry = partial_identity();
     int carry_row = -1;
-    for (int base = 0; base < n; base += 32) {
-        const int e = base + lane;
-        const bool in = e < n;
-        const int row = in ? e / p.n_split : 0x7ffffff0 + lane;
-        Partial v = in ? ld_partial_cg(part + e) : partial_identity();
-        if (lane == 0 && carry_row == row) v = combine(carry, v);
+    for (int g0 = 0; g0 < n; g0 += 256) {
+        Partial pre[8];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const Partial up = shfl_up_partial(v, o);
-            const int up_row = __shfl_up_sync(kFull, row, o);
-            if (lane >= o && up_row == row) v = combine(up, v);
+        for (int q = 0; q < 8; ++q) {
+            const int e = g0 + q * 32 + lane;
+            pre[q] = e < n ? ld_partial_cg(part + e) : partial_identity();
         }
-        if (in && (e + 1) % p.n_split == 0) {
-            // last partial of a row: v is the row's total.  sum exp(x - m) = s * 2^(c - m log2 e)
-            const float r = fmaf(-v.m, kLog2e, v.c);
-            const float s_m = v.s * exp2f(r);
-            rs.m[row] = v.m;
-            rs.s[row] = s_m;
-            rs.t[row] = v.idx;
-            if (!(s_m == s_m) || s_m == INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
-            if (p.diag.m) p.diag.m[row0 + row] = v.m;
-            if (p.diag.s) p.diag.s[row0 + row] = s_m;
-            if (p.diag.lse) p.diag.lse[row0 + row] = v.m + logf(s_m);
-            if (p.diag.t) p.diag.t[row0 + row] = v.idx;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int base = g0 + q * 32;
+            if (base >= n) break;
+            const int e = base + lane;
+            const bool in = e < n;
+            const int row = in ? e / p.n_split : 0x7ffffff0 + lane;
+            Partial v = pre[q];
+            if (lane == 0 && carry_row == row) v = combine(carry, v);
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const Partial up = shfl_up_partial(v, o);
+                const int up_row = __shfl_up_sync(kFull, row, o);
+                if (lane >= o && up_row == row) v = combine(up, v);
+            }
+            if (in && (e + 1) % p.n_split == 0) {
+                // last partial of a row: v is the row's total.  sum exp(x - m) = s * 2^(c - m log2 e)
+                const float r = fmaf(-v.m, kLog2e, v.c);
+                const float s_m = v.s * exp2f(r);
+                rs.m[row] = v.m;
+                rs.s[row] = s_m;
+                rs.t[row] = v.idx;
+                if (!(s_m == s_m) || s_m == INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
+                if (p.diag.m) p.diag.m[row0 + row] = v.m;
+                if (p.diag.s) p.diag.s[row0 + row] = s_m;
+                if (p.diag.lse) p.diag.lse[row0 + row] = v.m + logf(s_m);
+                if (p.diag.t) p.diag.t[row0 + row] = v.idx;
+            }
+            carry = shfl_partial(v, 31);
+            carry_row = __shfl_sync(kFull, row, 31);
         }
-        carry = shfl_partial(v, 31);
-        carry_row = __shfl_sync(kFull, row, 31);
     }
     __syncwarp();
 
     // S2 (second half), S3, S4 per position; S5 across the warp.
     bool match = false, ok = false;
     int t = -1;
+    unsigned int cnt = 0;
+    long long slot = -1;
     if (lane < K) {
         t = rs.t[lane];
         const float m = rs.m[lane];
         const float s_m = rs.s[lane];
         match = (d == t);
-        unsigned int cnt = 0;
-        if (valid) cnt = ocm_lookup(p.ocm, make_key(d, t));                           // S3
+        if (valid) cnt = ocm_lookup(p.ocm, make_key(d, t), &slot);                     // S3
         const bool is_freq = cnt >= p.ocm.lambda;
         const bool is_safe = (static_cast<double>(zd) - static_cast<double>(m)) >= static_cast<double>(p.log_tau);  // S4, Eq. 3
         ok = match || (valid && is_freq && is_safe);
@@ -366,6 +400,17 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
         p.rescued[pos] = (lane < n_acc && !match) ? 1 : 0;
         p.rej_d[pos] = record ? d : -1;
         p.rej_t[pos] = record ? t : -1;
+        if (p.do_update) {
+            // S6, first half: leave the slot of every recorded pair for the final adder
+            long long hint = kHintNone;
+            if (record) {
+                if (slot < 0 && update_regime(p) == kRegimeRoom) slot = ocm_reserve(p.ocm, make_key(d, t));
+                hint = slot < 0 ? kHintAbsent : slot;
+                const unsigned int room = 0xffffffffu - static_cast<unsigned int>(p.B * p.K);
+                if (slot >= 0 && cnt > room) hint |= kHintCareful;
+            }
+            __stcg(p.slot_hint + pos, hint);
+        }
     }
     const unsigned int m_match = __ballot_sync(kFull, reached && match);
     const unsigned int m_resc = __ballot_sync(kFull, lane < n_acc && !match && lane < K);
@@ -384,6 +429,35 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
     __syncwarp();
 }
 
+// S6, second half, by the warp that finalised the last batch row: every look-up of the
+// step is done, so the counts may change now.
+__device__ void apply_step_update(const StepParams &p, int lane, CanonScratch &canon)
+{
+    const int n = p.B * p.K;
+    const int regime = update_regime(p);
+    if (regime == kRegimeTransition) {
+        ocm_update_group<false>(p.ocm, p.rej_d, p.rej_t, nullptr, n, canon, lane, 32);
+        return;
+    }
+    unsigned int dropped = 0;
+    for (int j = lane; j < n; j += 32) {
+        const long long h = __ldcg(p.slot_hint + j);
+        if (h >= 0) {
+            const unsigned long long s = static_cast<unsigned long long>(h & ~kHintCareful);
+            if (h & kHintCareful)
+                ocm_add(p.ocm, s, 1u);
+            else
+                atomicAdd(&p.ocm.slots[s].count, 1u);
+        } else if (h == kHintAbsent) {
+            ++dropped;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dropped += __shfl_xor_sync(kFull, dropped, o);
+    if (lane == 0 && dropped) atomicAdd(&p.ocm.stats->n_dropped, static_cast<unsigned long long>(dropped));
+    __syncwarp();
+}
+
 // ---- the kernel ------------------------------------------------------------------------
 
 template <typename L>
@@ -396,67 +470,51 @@ __global__ void __launch_bounds__(kThreads, 4) csd_step_kernel(const __grid_cons
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int K1 = p.K + 1;
-    const long long G = gridDim.x;
-    const long long W = G * kWarps;
-    const long long first_tile = static_cast<long long>(warp) * G + blockIdx.x;
+    const int G = gridDim.x;
+    const int W = G * kWarps;
     const unsigned int tiles_per_b = static_cast<unsigned int>(K1 * p.n_split);
 
-    for (long long tile0 = first_tile; tile0 < p.total_tiles; tile0 += 32 * W) {
-        // ---- S1: reduce up to 32 tiles, lane j keeping the result of the j-th ----
-        Partial mine = partial_identity();
-        int n_mine = 0;
-        for (long long tile = tile0; tile < p.total_tiles && n_mine < 32; tile += W, ++n_mine) {
-            const long long row = tile / p.n_split;
-            const int chunk = static_cast<int>(tile - row * p.n_split);
-            const long long b = row / K1;
-            const int i = static_cast<int>(row - b * K1);
-            const E *rp = reinterpret_cast<const E *>(p.logits) + b * p.stride_b + i * p.stride_k;
-            const int e0 = chunk * p.tile_elems;
-            const int e1 = min(p.V, e0 + p.tile_elems);
-            const Partial r = warp_tile<L>(rp, e0, e1, lane);
-            if (lane == n_mine) mine = r;
-        }
+    for (int tile = warp * G + blockIdx.x; tile < p.total_tiles; tile += W) {
+        // ---- S1: this warp reduces one tile ----
+        const int row = tile / p.n_split;
+        const int chunk = tile - row * p.n_split;
+        const int b = row / K1;
+        const int i = row - b * K1;
+        const E *rp = reinterpret_cast<const E *>(p.logits) + (size_t)b * p.stride_b + (size_t)i * p.stride_k;
+        const int e0 = chunk * p.tile_elems;
+        const int e1 = min(p.V, e0 + p.tile_elems);
+        const Partial r = warp_tile<L>(rp, e0, e1, lane);
 
-        // ---- publish: one store per lane, one fence per warp, one ticket per tile ----
-        int my_b = -1;
-        if (lane < n_mine) {
-            const long long tile = tile0 + lane * W;
-            st_partial_cg(p.partials + tile, mine);
-            my_b = static_cast<int>((tile / p.n_split) / K1);
+        // ---- publish it and take a ticket on the batch row's arrival counter ----
+        bool completes = false;
+        if (lane == 0) {
+            st_partial_cg(p.partials + tile, r);
+            __threadfence();
+            completes = atomicAdd(p.b_ticket + b, 1u) == tiles_per_b - 1;
         }
+        completes = __shfl_sync(kFull, completes, 0);
+        if (!completes) continue;
+
+        // ---- this warp delivered the batch row's last tile: S2..S5 ----
+        __threadfence();
+        finalize_batch_row<L>(p, b, lane, row_scratch[warp]);
+        bool last = false;
+        if (lane == 0) p.b_ticket[b] = 0u;               // ready for the next launch
         __threadfence();
         __syncwarp();
-        bool completes = false;
-        if (lane < n_mine) completes = atomicAdd(p.b_ticket + my_b, 1u) == tiles_per_b - 1;
-        unsigned int todo = __ballot_sync(kFull, completes);
+        if (lane == 0) last = atomicAdd(p.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
+        last = __shfl_sync(kFull, last, 0);
+        if (!last) continue;
 
-        // ---- the warp that delivered a batch row's last tile finalises that row ----
-        while (todo) {
-            const int src = __ffs(todo) - 1;
-            todo &= todo - 1;
-            const int b = __shfl_sync(kFull, my_b, src);
+        // ---- every batch row is final: S6 ----
+        __threadfence();
+        if (p.do_update) apply_step_update(p, lane, canon);
+        if (lane == 0) {
+            OcmStatsDev *st = p.ocm.stats;
             __threadfence();
-            finalize_batch_row<L>(p, b, lane, row_scratch[warp]);
-            bool last = false;
-            if (lane == 0) {
-                p.b_ticket[b] = 0u;                       // ready for the next launch
-                __threadfence();
-                last = atomicAdd(p.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
-            }
-            last = __shfl_sync(kFull, last, 0);
-            if (last) {
-                // every batch row is final: S6, the step's UpdateMemory calls in (b, i) order
-                __threadfence();
-                if (p.do_update)
-                    ocm_update_group<false>(p.ocm, p.rej_d, p.rej_t, nullptr, static_cast<long long>(p.B) * p.K, canon, lane, 32);
-                if (lane == 0) {
-                    OcmStatsDev *st = p.ocm.stats;
-                    __threadfence();
-                    st->n_keys_start = atomicAdd(&st->n_keys, 0ull);
-                    atomicAdd(&st->steps, 1ull);
-                    *p.g_ticket = 0u;
-                }
-            }
+            st->n_keys_start = atomicAdd(&st->n_keys, 0ull);
+            atomicAdd(&st->steps, 1ull);
+            *p.g_ticket = 0u;
         }
     }
 }
