@@ -314,6 +314,7 @@ def run_ours(args, wl, tau):
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
 
+    pkg.csd_set_overlap(not args.no_overlap)
     bench = Bench(wl, tau, device, seed=rank)
     use_graph = not args.eager
     if use_graph:
@@ -353,6 +354,8 @@ def run_ours(args, wl, tau):
                 "l2_policy": f"ring of {bench.ring_len} distinct step inputs "
                              f"({bench.ring_len * wl.logit_bytes / 1e6:.0f} MB, > 2x L2)",
                 "launch": ("CUDA graph of %d steps replayed" % bench.ring_len) if use_graph else "eager",
+                "step_overlap": "off" if args.no_overlap else
+                                "programmatic dependent launch: a step streams its logits while the previous step drains",
                 "kernel_shape": shape}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_source": f"of {peak_kind}",
@@ -408,6 +411,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--tau", type=float, default=None)
     ap.add_argument("--eager", action="store_true", help="launch every step from Python instead of replaying a graph")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="plain stream-ordered launches (no programmatic dependent launch between steps)")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extras", action="store_true", help="also time the other workloads (extra keys, same line)")

@@ -225,18 +225,30 @@ csd_status_t csd_ocm_stats(const csd_ocm_t *ocm, csd_stats_t *host_out, void *st
  * -inf for tau == 0.  Host function. */
 float csd_scg_threshold(float tau);
 
-/* Launch shape a step of this size uses: grid blocks, threads per block, elements
- * per tile and tiles per logit row.  Host function; for reports and tests. */
+/* Launch shape a step of this size uses: grid blocks, threads per block, warps that
+ * own a span of the logits, and partial-result slots reserved per logit row.  Host
+ * function; for reports and tests. */
 csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype,
-                              int *grid, int *block, int *tile_elems, int *tiles_per_row);
+                              int *grid, int *block, int *workers, int *parts_per_row);
 
-/* Expert knob, process-wide: override the automatic tiling.  tile_bytes: bytes of
- * logits reduced by one warp at a time (multiple of 4096; 0 = automatic);
- * ctas_per_sm: resident blocks per SM of the persistent grid (1..4; 0 = automatic,
- * which is 4).  Changes csd_workspace_bytes: size workspaces after calling it.
- * Results stay bit-reproducible for a fixed setting; the low-order bits of the
- * sums s may differ between settings (different summation trees).  Host function. */
-csd_status_t csd_set_tuning(int tile_bytes, int ctas_per_sm);
+/* Expert knob, process-wide: override the automatic work split.  parts_per_row: cap
+ * on the number of warps that share one logit row (0 = automatic, which is 32; small
+ * values mean fewer, longer spans); ctas_per_sm: resident blocks per SM of the
+ * persistent grid (1..4; 0 = automatic, which is 4).  Changes csd_workspace_bytes:
+ * size workspaces after calling it.  Results stay bit-reproducible for a fixed
+ * setting; the low-order bits of the sums s may differ between settings (different
+ * summation trees).  Host function. */
+csd_status_t csd_set_tuning(int parts_per_row, int ctas_per_sm);
+
+/* Process-wide, off by default.  When on, csd_verify / csd_step launch with
+ * programmatic stream serialization: the kernel may start, and stream logits, while
+ * the previous kernel on the stream is still draining; it waits for that kernel to
+ * complete before it first touches the workspace, the memory or any output.  Turn it
+ * on only if the logits and draft of a step are never written by the kernel launched
+ * directly before that step on the same stream (back-to-back steps over inputs that
+ * are already resident qualify; a producer kernel launched right before the step
+ * does too as long as it does not itself signal early completion).  Host function. */
+csd_status_t csd_set_overlap(int enable);
 
 const char *csd_status_string(csd_status_t status);
 

@@ -25,7 +25,7 @@ EXPORTS = [
     "csd_ocm_create", "csd_ocm_reset", "csd_ocm_destroy", "csd_ocm_set_lambda",
     "csd_workspace_bytes", "csd_workspace_init", "csd_verify", "csd_ocm_update", "csd_step",
     "csd_host_staging_bytes", "csd_step_host", "csd_ocm_export", "csd_ocm_import", "csd_ocm_stats",
-    "csd_scg_threshold", "csd_launch_shape", "csd_set_tuning", "csd_status_string",
+    "csd_scg_threshold", "csd_launch_shape", "csd_set_tuning", "csd_set_overlap", "csd_status_string",
 ]
 
 
@@ -79,6 +79,7 @@ def lib():
         "csd_scg_threshold": (c_float, [c_float]),
         "csd_launch_shape": (c_int, [c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
         "csd_set_tuning": (c_int, [c_int, c_int]),
+        "csd_set_overlap": (c_int, [c_int]),
         "csd_status_string": (c_char_p, [c_int]),
     }
     for name, (res, args) in sigs.items():
@@ -115,14 +116,18 @@ def csd_scg_threshold(tau: float) -> float:
     return float(lib().csd_scg_threshold(c_float(tau)))
 
 
-def csd_set_tuning(tile_bytes: int = 0, ctas_per_sm: int = 0):
-    _check(lib().csd_set_tuning(tile_bytes, ctas_per_sm), "csd_set_tuning")
+def csd_set_tuning(parts_per_row: int = 0, ctas_per_sm: int = 0):
+    _check(lib().csd_set_tuning(parts_per_row, ctas_per_sm), "csd_set_tuning")
+
+
+def csd_set_overlap(enable: bool):
+    _check(lib().csd_set_overlap(1 if enable else 0), "csd_set_overlap")
 
 
 def csd_launch_shape(B, K, V, dtype_code):
     g, b, te, tr = c_int(), c_int(), c_int(), c_int()
     _check(lib().csd_launch_shape(B, K, V, dtype_code, byref(g), byref(b), byref(te), byref(tr)), "csd_launch_shape")
-    return dict(grid=g.value, block=b.value, tile_elems=te.value, tiles_per_row=tr.value)
+    return dict(grid=g.value, block=b.value, workers=te.value, parts_per_row=tr.value)
 
 
 def csd_workspace_bytes(B, K, V, dtype_code) -> int:

@@ -24,8 +24,9 @@ namespace {
 
 constexpr int kDefaultSms = 148;   // B200; used only when no device can be queried
 
-int g_tile_bytes_override = 0;
+int g_parts_per_row_override = 0;
 int g_ctas_per_sm_override = 0;
+int g_overlap_steps = 0;
 
 int sm_count()
 {
@@ -43,48 +44,46 @@ int sm_count()
 
 struct Shape {
     int grid;
-    int tile_elems;
-    int n_split;
-    int total_tiles;
+    int n_workers;         // warps owning a span
+    int unit_elems;        // elements per 512-byte unit
+    int units_per_row;
+    int slots_per_row;     // partial slots reserved per logit row
+    long long total_units;
 };
 
 inline int elt_bytes(csd_dtype_t dt) { return dt == CSD_F32 ? 4 : 2; }
 
+constexpr int kUnitBytes = 512;   // one 16-byte vector per lane
+
 bool shape_ok(int B, int K, int V, csd_dtype_t dt)
 {
     if (!(B > 0 && K > 0 && V > 0 && K <= CSD_MAX_K && (dt == CSD_F32 || dt == CSD_BF16))) return false;
-    // tile and position indices are 32-bit: the smallest tile is 4 KiB
-    const long long rows = static_cast<long long>(B) * (K + 1);
-    const long long tiles_max = rows * ((static_cast<long long>(V) * elt_bytes(dt) + 4095) / 4096);
-    return tiles_max < (1ll << 31) && static_cast<long long>(B) * K < (1ll << 31);
+    // row and position indices are 32-bit
+    return static_cast<long long>(B) * (K + 1) < (1ll << 31) && static_cast<long long>(B) * K < (1ll << 31);
 }
 
-// Tiles are whole warp iterations (32 lanes x 8 x 16 bytes = 4 KiB).  A logit row is cut
-// into at most 32 tiles, so that a batch row is described by few partials; when that
-// leaves more than 8 tiles per warp of the persistent grid the tiles are doubled (up to
-// 64 KiB), which amortises the per-tile publication.
+// The unit space (R rows x U units of 512 bytes) is split evenly over W warps.  W is the
+// persistent grid's warp count, capped so that a row is touched by at most ~33 warps
+// (few partials per row keeps the per-row fold short) and never above the unit count.
 Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
 {
     const int eb = elt_bytes(dt);
     const int ctas_per_sm = g_ctas_per_sm_override > 0 ? g_ctas_per_sm_override : 4;
-    const long long workers = static_cast<long long>(sm_count()) * ctas_per_sm * kWarps;
+    const int parts_cap = g_parts_per_row_override > 0 ? g_parts_per_row_override : 32;
     const long long rows = static_cast<long long>(B) * (K + 1);
-    const long long row_bytes = static_cast<long long>(V) * eb;
-    long long tile_bytes;
-    if (g_tile_bytes_override > 0) {
-        tile_bytes = g_tile_bytes_override;
-    } else {
-        tile_bytes = ((row_bytes + 31) / 32 + 4095) / 4096 * 4096;
-        while (tile_bytes < 65536 && rows * ((row_bytes + tile_bytes - 1) / tile_bytes) > 8 * workers) tile_bytes *= 2;
-    }
     Shape s;
-    s.tile_elems = static_cast<int>(tile_bytes / eb);
-    s.n_split = (V + s.tile_elems - 1) / s.tile_elems;
-    s.total_tiles = static_cast<int>(rows * s.n_split);
-    long long blocks = static_cast<long long>(sm_count()) * ctas_per_sm;
-    const long long needed = (s.total_tiles + kWarps - 1) / kWarps;
-    if (needed < blocks) blocks = needed;
-    s.grid = static_cast<int>(blocks < 1 ? 1 : blocks);
+    s.unit_elems = kUnitBytes / eb;
+    s.units_per_row = (V + s.unit_elems - 1) / s.unit_elems;
+    s.total_units = rows * s.units_per_row;
+    long long workers = static_cast<long long>(sm_count()) * ctas_per_sm * kWarps;
+    if (workers > rows * parts_cap) workers = rows * parts_cap;
+    if (workers > s.total_units) workers = s.total_units;
+    s.n_workers = static_cast<int>(workers);
+    s.grid = static_cast<int>((workers + kWarps - 1) / kWarps);
+    // span boundaries lie at floor(w*T/W): at most ceil((U-1)*W/T) of them fall inside a row
+    long long slots = ((s.units_per_row - 1) * workers + s.total_units - 1) / s.total_units + 1;
+    if (slots > s.units_per_row) slots = s.units_per_row;
+    s.slots_per_row = static_cast<int>(slots < 1 ? 1 : slots);
     return s;
 }
 
@@ -98,7 +97,7 @@ WorkspaceLayout ws_layout(int B, int K, const Shape &s)
 {
     WorkspaceLayout w;
     w.partials_off = 0;
-    w.hint_off = align_up(static_cast<size_t>(B) * (K + 1) * s.n_split * sizeof(Partial), 256);
+    w.hint_off = align_up(static_cast<size_t>(B) * (K + 1) * s.slots_per_row * sizeof(Partial), 256);
     w.b_ticket_off = align_up(w.hint_off + static_cast<size_t>(B) * K * sizeof(long long), 256);
     w.g_ticket_off = align_up(w.b_ticket_off + static_cast<size_t>(B) * sizeof(unsigned int), 16);
     w.total = align_up(w.g_ticket_off + 16, 256);
@@ -151,22 +150,41 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.slot_hint = reinterpret_cast<long long *>(ws + w.hint_off);
     p.b_ticket = reinterpret_cast<unsigned int *>(ws + w.b_ticket_off);
     p.g_ticket = reinterpret_cast<unsigned int *>(ws + w.g_ticket_off);
-    p.tile_elems = s.tile_elems;
-    p.n_split = s.n_split;
-    p.total_tiles = s.total_tiles;
+    p.n_workers = s.n_workers;
+    p.unit_elems = s.unit_elems;
+    p.units_per_row = s.units_per_row;
+    p.slots_per_row = s.slots_per_row;
+    p.total_units = s.total_units;
 
     const int eb = elt_bytes(dtype);
     const int per_vec = 16 / eb;
     const bool vec = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && (stride_b * eb) % 16 == 0 &&
                      (stride_k * eb) % 16 == 0 && V % per_vec == 0;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const dim3 grid(s.grid), block(kThreads);
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(s.grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    if (g_overlap_steps) {
+        // let this launch begin while the previous kernel on the stream drains; the kernel
+        // itself waits for that kernel before its first write
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    cudaError_t err;
     if (dtype == CSD_F32) {
-        if (vec) csd_step_kernel<LaneF32Vec><<<grid, block, 0, st>>>(p);
-        else csd_step_kernel<LaneF32Scalar><<<grid, block, 0, st>>>(p);
+        err = vec ? cudaLaunchKernelEx(&cfg, csd_step_kernel<LaneF32Vec>, p)
+                  : cudaLaunchKernelEx(&cfg, csd_step_kernel<LaneF32Scalar>, p);
     } else {
-        if (vec) csd_step_kernel<LaneBf16Vec><<<grid, block, 0, st>>>(p);
-        else csd_step_kernel<LaneBf16Scalar><<<grid, block, 0, st>>>(p);
+        err = vec ? cudaLaunchKernelEx(&cfg, csd_step_kernel<LaneBf16Vec>, p)
+                  : cudaLaunchKernelEx(&cfg, csd_step_kernel<LaneBf16Scalar>, p);
+    }
+    if (err != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
     }
     return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
 }
@@ -425,24 +443,30 @@ float csd_scg_threshold(float tau)
     return static_cast<float>(std::log(static_cast<double>(tau)));
 }
 
-csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype, int *grid, int *block, int *tile_elems,
-                              int *tiles_per_row)
+csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype, int *grid, int *block, int *workers,
+                              int *parts_per_row)
 {
     if (!shape_ok(B, K, V, dtype)) return CSD_ERR_INVALID_ARG;
     const Shape s = pick_shape(B, K, V, dtype);
     if (grid) *grid = s.grid;
     if (block) *block = kThreads;
-    if (tile_elems) *tile_elems = s.tile_elems;
-    if (tiles_per_row) *tiles_per_row = s.n_split;
+    if (workers) *workers = s.n_workers;
+    if (parts_per_row) *parts_per_row = s.slots_per_row;
     return CSD_OK;
 }
 
-csd_status_t csd_set_tuning(int tile_bytes, int ctas_per_sm)
+csd_status_t csd_set_tuning(int parts_per_row, int ctas_per_sm)
 {
-    if (tile_bytes != 0 && (tile_bytes < 4096 || tile_bytes % 4096 != 0 || tile_bytes > (1 << 22))) return CSD_ERR_INVALID_ARG;
+    if (parts_per_row < 0 || parts_per_row > 4096) return CSD_ERR_INVALID_ARG;
     if (ctas_per_sm < 0 || ctas_per_sm > 4) return CSD_ERR_INVALID_ARG;
-    g_tile_bytes_override = tile_bytes;
+    g_parts_per_row_override = parts_per_row;
     g_ctas_per_sm_override = ctas_per_sm;
+    return CSD_OK;
+}
+
+csd_status_t csd_set_overlap(int enable)
+{
+    g_overlap_steps = enable ? 1 : 0;
     return CSD_OK;
 }
 

@@ -3,27 +3,33 @@
 // Algorithm 1's verification loop, and finally the memory update -- one launch.
 //
 // Work decomposition
-//   * The R = B*(K+1) logit rows are cut into tiles of `tile_elems` contiguous
-//     elements (at most ~32 tiles per row); a tile is reduced by ONE WARP on its own:
-//     there is no block barrier anywhere.  Warps are persistent workers: tile t goes to
-//     block t mod G, warp (t / G) mod 8, so every SM gets the same number of tiles +-1
-//     and batch rows complete in index order while later ones are still streaming.
-//   * A lane keeps 8 x 16 bytes in flight; a tile is reduced with a running maximum,
-//     an integer reference exponent and four independent sum accumulators; only the
-//     iteration in which the maximum last improved is remembered, and the exact
-//     lowest arg-max index is recovered by re-reading that one iteration (an L2 hit).
-//   * After each tile lane 0 stores the partial, fences, and takes a ticket on the
-//     batch row's arrival counter.  Whichever warp delivers the last tile of a batch
-//     row finalises it: the row's partials are prefetched together and folded by a
-//     segmented warp scan in a fixed order (bit-reproducible sums), lanes 0..K-1 take
-//     the per-position decisions, a ballot gives the accepted prefix.
+//   * The R = B*(K+1) logit rows, each cut into 512-byte units, form one long unit
+//     space that is split EVENLY and contiguously over the W warps of a persistent
+//     grid (warp w owns units [w*T/W, (w+1)*T/W)).  Every warp streams the same number
+//     of bytes +-512, a warp touches one or two rows, and a row is described by about
+//     W/R + 1 partial results (the host caps W so that this stays <= ~33).
+//   * A warp reduces its part of a row on its own: a lane keeps 8 x 16 bytes in flight,
+//     carries a running maximum, an integer reference exponent and four independent
+//     sum accumulators; only the iteration in which the maximum last improved is
+//     remembered, and the exact lowest arg-max index is recovered by re-reading that
+//     one iteration (an L2 hit).  No block barrier anywhere.
+//   * Partials stay in registers (lane j holds the j-th row part) until the warp's span
+//     is done; then one store per lane, ONE fence per warp, and one ticket per batch
+//     row touched.  Everything before that point reads only the logits, so with
+//     programmatic dependent launch the streaming phase of step n+1 overlaps the tail
+//     of step n: the only wait on the previous launch sits just before the first
+//     workspace write.
+//   * Whichever warp delivers a batch row's last part finalises it: the row's partials
+//     are fetched together and folded by a segmented warp scan in a fixed order
+//     (bit-reproducible sums), lanes 0..K-1 take the per-position decisions, a ballot
+//     gives the accepted prefix.
 //   * Memory update without a second probe: the look-up already found each recorded
 //     pair's slot (absent pairs get an empty slot reserved with count 0, which no
 //     look-up can tell from "absent"), and leaves it as a hint.  The warp finalising
 //     the LAST batch row then only adds 1 to the hinted slots, so every look-up of the
 //     step saw the step-start counts.  Near the key limit, where admission order
 //     matters, that warp falls back to the canonical-order path.
-//   * Nothing ever waits for another block: arrival counters only, so no launch can hang.
+//   * Nothing ever spins on another block: arrival counters only, so no launch can hang.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -48,13 +54,15 @@ struct StepParams {
     int *rej_d;
     int *rej_t;
     csd_diag_t diag;
-    Partial *partials;       // [R * n_split]
+    Partial *partials;       // [R * slots_per_row]
     long long *slot_hint;    // [B * K] slot of each recorded pair (see kHint*)
     unsigned int *b_ticket;  // [B]
     unsigned int *g_ticket;  // [1]
-    int tile_elems;
-    int n_split;             // tiles per logit row
-    int total_tiles;
+    int n_workers;           // W: warps that own a span of the unit space
+    int unit_elems;          // elements per 512-byte unit
+    int units_per_row;       // U = ceil(V / unit_elems)
+    int slots_per_row;       // S >= most warps that can touch one row
+    long long total_units;   // T = R * U
 };
 
 constexpr long long kHintNone = -1;          // nothing to record at this position
@@ -276,12 +284,30 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
     return p;
 }
 
+// ---- the even split of the unit space ---------------------------------------------------
+
+__device__ __forceinline__ long long span_begin(const StepParams &p, int w)
+{
+    return static_cast<long long>(w) * p.total_units / p.n_workers;
+}
+
+// The warp whose span holds global unit g: the largest w with span_begin(w) <= g.
+__device__ __forceinline__ int owner_of(const StepParams &p, long long g)
+{
+    return static_cast<int>(((g + 1) * p.n_workers - 1) / p.total_units);
+}
+
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- S2..S5 for one batch row, by one warp ------------------------------------------
 
 struct RowScratch {
     float m[CSD_MAX_K + 1];
     float s[CSD_MAX_K + 1];
     int t[CSD_MAX_K + 1];
+    int first[CSD_MAX_K + 1];   // first warp touching the row
+    int parts[CSD_MAX_K + 1];   // number of warps touching the row
 };
 
 enum UpdateRegime { kRegimeRoom = 0, kRegimeFull = 1, kRegimeTransition = 2 };
@@ -301,10 +327,10 @@ template <typename L>
 __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScratch &rs)
 {
     using E = typename L::elem;
-    const int K = p.K, K1 = p.K + 1;
-    const int n = K1 * p.n_split;
-    const Partial *part = p.partials + (size_t)b * n;
+    const int K = p.K, K1 = p.K + 1, S = p.slots_per_row;
+    const int n = K1 * S;
     const size_t row0 = (size_t)b * K1;
+    const Partial *part = p.partials + row0 * S;
 
     // S2 (first half): the draft tokens and their logits do not depend on the
     // reduction, so their loads are issued before the partials are folded.
@@ -319,9 +345,17 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
             zd = L::load_elem(rowp, d);
         }
     }
+    const int regime = p.do_update ? update_regime(p) : kRegimeFull;
+    for (int r = lane; r < K1; r += 32) {
+        const long long u0 = static_cast<long long>(row0 + r) * p.units_per_row;
+        const int wf = owner_of(p, u0);
+        rs.first[r] = wf;
+        rs.parts[r] = owner_of(p, u0 + p.units_per_row - 1) - wf + 1;
+    }
+    __syncwarp();
 
     // S1 (second half): fold the K+1 rows' partials with a segmented inclusive scan,
-    // 32 partials at a time, always in the same order; up to 256 are fetched at once.
+    // 32 slots at a time, always in the same order; up to 256 slots are fetched at once.
     Partial carry = partial_identity();
     int carry_row = -1;
     for (int g0 = 0; g0 < n; g0 += 256) {
@@ -329,7 +363,11 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             const int e = g0 + q * 32 + lane;
-            pre[q] = e < n ? ld_partial_cg(part + e) : partial_identity();
+            pre[q] = partial_identity();
+            if (e < n) {
+                const int row = e / S;
+                if (e - row * S < rs.parts[row]) pre[q] = ld_partial_cg(part + e);
+            }
         }
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -337,7 +375,7 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
             if (base >= n) break;
             const int e = base + lane;
             const bool in = e < n;
-            const int row = in ? e / p.n_split : 0x7ffffff0 + lane;
+            const int row = in ? e / S : 0x7ffffff0 + lane;
             Partial v = pre[q];
             if (lane == 0 && carry_row == row) v = combine(carry, v);
 #pragma unroll
@@ -346,8 +384,8 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
                 const int up_row = __shfl_up_sync(kFull, row, o);
                 if (lane >= o && up_row == row) v = combine(up, v);
             }
-            if (in && (e + 1) % p.n_split == 0) {
-                // last partial of a row: v is the row's total.  sum exp(x - m) = s * 2^(c - m log2 e)
+            if (in && e - row * S == rs.parts[row] - 1) {
+                // last part of a row: v is the row's total.  sum exp(x - m) = s * 2^(c - m log2 e)
                 const float r = fmaf(-v.m, kLog2e, v.c);
                 const float s_m = v.s * exp2f(r);
                 rs.m[row] = v.m;
@@ -404,7 +442,7 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
             // S6, first half: leave the slot of every recorded pair for the final adder
             long long hint = kHintNone;
             if (record) {
-                if (slot < 0 && update_regime(p) == kRegimeRoom) slot = ocm_reserve(p.ocm, make_key(d, t));
+                if (slot < 0 && regime == kRegimeRoom) slot = ocm_reserve(p.ocm, make_key(d, t));
                 hint = slot < 0 ? kHintAbsent : slot;
                 const unsigned int room = 0xffffffffu - static_cast<unsigned int>(p.B * p.K);
                 if (slot >= 0 && cnt > room) hint |= kHintCareful;
@@ -440,16 +478,24 @@ __device__ void apply_step_update(const StepParams &p, int lane, CanonScratch &c
         return;
     }
     unsigned int dropped = 0;
-    for (int j = lane; j < n; j += 32) {
-        const long long h = __ldcg(p.slot_hint + j);
-        if (h >= 0) {
-            const unsigned long long s = static_cast<unsigned long long>(h & ~kHintCareful);
-            if (h & kHintCareful)
-                ocm_add(p.ocm, s, 1u);
-            else
-                atomicAdd(&p.ocm.slots[s].count, 1u);
-        } else if (h == kHintAbsent) {
-            ++dropped;
+    for (int j0 = 0; j0 < n; j0 += 256) {
+        long long h[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int j = j0 + q * 32 + lane;
+            h[q] = j < n ? __ldcg(p.slot_hint + j) : kHintNone;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            if (h[q] >= 0) {
+                const unsigned long long s = static_cast<unsigned long long>(h[q] & ~kHintCareful);
+                if (h[q] & kHintCareful)
+                    ocm_add(p.ocm, s, 1u);
+                else
+                    atomicAdd(&p.ocm.slots[s].count, 1u);
+            } else if (h[q] == kHintAbsent) {
+                ++dropped;
+            }
         }
     }
 #pragma unroll
@@ -467,54 +513,92 @@ __global__ void __launch_bounds__(kThreads, 4) csd_step_kernel(const __grid_cons
     __shared__ CanonScratch canon;
 
     using E = typename L::elem;
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
+    const int w = blockIdx.x * kWarps + warp;
+    if (w >= p.n_workers) return;
     const int K1 = p.K + 1;
-    const int G = gridDim.x;
-    const int W = G * kWarps;
-    const unsigned int tiles_per_b = static_cast<unsigned int>(K1 * p.n_split);
+    const int U = p.units_per_row;
+    long long g = span_begin(p, w);
+    const long long g_end = span_begin(p, w + 1);
 
-    for (int tile = warp * G + blockIdx.x; tile < p.total_tiles; tile += W) {
-        // ---- S1: this warp reduces one tile ----
-        const int row = tile / p.n_split;
-        const int chunk = tile - row * p.n_split;
-        const int b = row / K1;
-        const int i = row - b * K1;
-        const E *rp = reinterpret_cast<const E *>(p.logits) + (size_t)b * p.stride_b + (size_t)i * p.stride_k;
-        const int e0 = chunk * p.tile_elems;
-        const int e1 = min(p.V, e0 + p.tile_elems);
-        const Partial r = warp_tile<L>(rp, e0, e1, lane);
-
-        // ---- publish it and take a ticket on the batch row's arrival counter ----
-        bool completes = false;
-        if (lane == 0) {
-            st_partial_cg(p.partials + tile, r);
-            __threadfence();
-            completes = atomicAdd(p.b_ticket + b, 1u) == tiles_per_b - 1;
+    while (g < g_end) {
+        // ---- S1: reduce this warp's part of up to 32 rows, lane j keeping the j-th ----
+        Partial mine = partial_identity();
+        int my_row = -1;
+        int n_held = 0;
+        while (g < g_end && n_held < 32) {
+            const long long row = g / U;
+            const int o0 = static_cast<int>(g - row * U);
+            const long long left = g_end - row * U;
+            const int o1 = left < U ? static_cast<int>(left) : U;
+            const long long b = row / K1;
+            const int i = static_cast<int>(row - b * K1);
+            const E *rp = reinterpret_cast<const E *>(p.logits) + b * p.stride_b + i * p.stride_k;
+            const int e0 = o0 * p.unit_elems;
+            const long long e1l = static_cast<long long>(o1) * p.unit_elems;
+            const int e1 = e1l < p.V ? static_cast<int>(e1l) : p.V;
+            const Partial r = warp_tile<L>(rp, e0, e1, lane);
+            if (lane == n_held) {
+                mine = r;
+                my_row = static_cast<int>(row);
+            }
+            ++n_held;
+            g = (row + 1) * U;
         }
-        completes = __shfl_sync(kFull, completes, 0);
-        if (!completes) continue;
+        const int next_b = g < g_end ? static_cast<int>((g / U) / K1) : -1;
 
-        // ---- this warp delivered the batch row's last tile: S2..S5 ----
-        __threadfence();
-        finalize_batch_row<L>(p, b, lane, row_scratch[warp]);
-        bool last = false;
-        if (lane == 0) p.b_ticket[b] = 0u;               // ready for the next launch
+        // ---- publish: one store per lane, one fence per warp, one ticket per batch row.
+        //      This is the first access to memory another launch may still be using. ----
+        pdl_wait();
+        int my_b = -1;
+        if (lane < n_held) {
+            const int slot = w - owner_of(p, static_cast<long long>(my_row) * U);
+            if (slot < p.slots_per_row) st_partial_cg(p.partials + (size_t)my_row * p.slots_per_row + slot, mine);
+            else atomicOr(&p.ocm.stats->flags, CSD_FLAG_PROBE_EXHAUSTED);
+            my_b = my_row / K1;
+        }
         __threadfence();
         __syncwarp();
-        if (lane == 0) last = atomicAdd(p.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
-        last = __shfl_sync(kFull, last, 0);
-        if (!last) continue;
+        const int below_b = __shfl_down_sync(kFull, my_b, 1);
+        bool completes = false;
+        if (lane < n_held) {
+            // the lane holding this warp's last part of a batch row takes that row's ticket
+            const bool closes = (lane == n_held - 1) ? (my_b != next_b) : (below_b != my_b);
+            if (closes) {
+                const long long u0 = static_cast<long long>(my_b) * K1 * U;
+                const unsigned int expected = owner_of(p, u0 + static_cast<long long>(K1) * U - 1) - owner_of(p, u0) + 1;
+                completes = atomicAdd(p.b_ticket + my_b, 1u) == expected - 1;
+            }
+        }
+        unsigned int todo = __ballot_sync(kFull, completes);
 
-        // ---- every batch row is final: S6 ----
-        __threadfence();
-        if (p.do_update) apply_step_update(p, lane, canon);
-        if (lane == 0) {
-            OcmStatsDev *st = p.ocm.stats;
+        // ---- the warp that delivered a batch row's last part finalises it: S2..S5 ----
+        while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const int b = __shfl_sync(kFull, my_b, src);
             __threadfence();
-            st->n_keys_start = atomicAdd(&st->n_keys, 0ull);
-            atomicAdd(&st->steps, 1ull);
-            *p.g_ticket = 0u;
+            finalize_batch_row<L>(p, b, lane, row_scratch[warp]);
+            bool last = false;
+            if (lane == 0) p.b_ticket[b] = 0u;               // ready for the next launch
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) last = atomicAdd(p.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
+            last = __shfl_sync(kFull, last, 0);
+            if (!last) continue;
+
+            // ---- every batch row is final: S6 ----
+            __threadfence();
+            if (p.do_update) apply_step_update(p, lane, canon);
+            if (lane == 0) {
+                OcmStatsDev *st = p.ocm.stats;
+                __threadfence();
+                st->n_keys_start = atomicAdd(&st->n_keys, 0ull);
+                atomicAdd(&st->steps, 1ull);
+                *p.g_ticket = 0u;
+            }
         }
     }
 }

@@ -331,32 +331,81 @@ def test_host_entry_point_matches_device_entry_point():
     a.close(); b.close()
 
 
-@pytest.mark.parametrize("tile_bytes,ctas", [(4096, 1), (8192, 2), (32768, 4), (65536, 3)])
-def test_parity_under_other_tilings(tile_bytes, ctas):
+@pytest.mark.parametrize("parts,ctas", [(1, 1), (2, 2), (8, 4), (300, 3)])
+def test_parity_under_other_splits(parts, ctas):
     try:
-        csd_set_tuning(tile_bytes, ctas)
+        csd_set_tuning(parts, ctas)
         wl = dataclasses.replace(WORKLOADS["ocm_contention"], B=8)
-        assert csd_launch_shape(wl.B, wl.K, wl.V, CSD_BF16)["tile_elems"] == tile_bytes // 2
+        assert csd_launch_shape(wl.B, wl.K, wl.V, CSD_BF16)["workers"] <= min(148 * ctas * 8, parts * wl.rows)
         lockstep(wl, steps=3, tau=0.3, lam=1)
         wl = dataclasses.replace(WORKLOADS["large_batch"], B=4)
-        assert csd_launch_shape(wl.B, wl.K, wl.V, CSD_F32)["tile_elems"] == tile_bytes // 4
         lockstep(wl, steps=2, tau=0.2, lam=1)
     finally:
         csd_set_tuning(0, 0)
 
 
-def test_long_row_many_tiles_per_warp():
-    """One row far longer than the machine has warps x tiles: exercises the 32-tile batches."""
-    try:
-        csd_set_tuning(4096, 1)
-        B, K, V = 48, 1, 1 << 20            # 96 rows x 1024 tiles = 98304 tiles > 32 x 1184 warps
-        z, d = _random_inputs(B, K, V, torch.float32, seed=11)
-        ocm = Ocm(256, 0)
-        mem = ORACLE.OCM(256, 0)
-        buf = StepBuffers(B, K, V, torch.float32, diag=True)
-        csd_step(z, d, ocm, 0.01, buf)
-        compare(buf, oracle_step(z, d, mem, 0.01))
-        compare_memory(ocm, mem)
-        ocm.close()
-    finally:
-        csd_set_tuning(0, 0)
+def test_many_short_rows_per_warp():
+    """Rows far shorter than a warp's span: a warp holds parts of many rows and of several
+    batch rows (more than 32 row parts per warp with the single-block setting)."""
+    for (B, K, V, dtype) in ((600, 3, 160, torch.float32), (97, 32, 520, torch.bfloat16), (3000, 1, 24, torch.bfloat16)):
+        for tuning in ((0, 0), (1, 1)):
+            try:
+                csd_set_tuning(*tuning)
+                z, d = _random_inputs(B, K, V, dtype, seed=21)
+                ocm = Ocm(1 << 14, 0)
+                mem = ORACLE.OCM(1 << 14, 0)
+                buf = StepBuffers(B, K, V, dtype, diag=True)
+                csd_step(z, d, ocm, 0.02, buf)
+                compare(buf, oracle_step(z, d, mem, 0.02))
+                compare_memory(ocm, mem)
+                ocm.close()
+            finally:
+                csd_set_tuning(0, 0)
+
+
+def test_overlapped_launches_match():
+    """Back-to-back steps launched with programmatic stream serialization (the setting the
+    benchmark times) give the same results as plain launches."""
+    from paper_2604_13634_b200 import csd_set_overlap
+    wl = dataclasses.replace(WORKLOADS["batched_serving"], B=8)
+    syn = Synth(wl, 4, "cuda")
+    inputs = [syn.step(s) for s in range(6)]
+    results = []
+    for overlap in (False, True):
+        try:
+            csd_set_overlap(overlap)
+            ocm = Ocm(4096, 1)
+            bufs = [StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True) for _ in inputs]
+            for rep in range(3):
+                for (z, d), buf in zip(inputs, bufs):        # 18 launches with nothing between them
+                    csd_step(z, d, ocm, 0.3, buf)
+            torch.cuda.synchronize()
+            results.append(([(b.accept_len.clone(), b.next_token.clone(), b.rescued_mask.clone(),
+                              b.diag["s"].clone(), b.diag["cnt"].clone()) for b in bufs], ocm.export(), ocm.stats()))
+            ocm.close()
+        finally:
+            csd_set_overlap(False)
+    (ra, ea, sa), (rb, eb, sb) = results
+    for x, y in zip(ra, rb):
+        assert all(torch.equal(p, q) for p, q in zip(x, y))
+    assert all(torch.equal(p, q) for p, q in zip(ea, eb)) and sa == sb
+    # and the plain run itself is pinned to the oracle
+    mem = ORACLE.OCM(4096, 1)
+    for rep in range(3):
+        for z, d in inputs:
+            ref = oracle_step(z, d, mem, 0.3)
+    assert np.array_equal(ra[-1][0].cpu().numpy(), ref["accept_len"])
+    assert np.array_equal(ea[2].numpy(), mem.export()[2])
+
+
+def test_long_rows():
+    """Rows far longer than one warp's share: many warps per row, parts capped by the split."""
+    B, K, V = 48, 1, 1 << 20
+    z, d = _random_inputs(B, K, V, torch.float32, seed=11)
+    ocm = Ocm(256, 0)
+    mem = ORACLE.OCM(256, 0)
+    buf = StepBuffers(B, K, V, torch.float32, diag=True)
+    csd_step(z, d, ocm, 0.01, buf)
+    compare(buf, oracle_step(z, d, mem, 0.01))
+    compare_memory(ocm, mem)
+    ocm.close()
