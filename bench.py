@@ -315,6 +315,7 @@ def run_ours(args, wl, tau):
         dist.init_process_group("nccl", device_id=device)
 
     pkg.csd_set_overlap(not args.no_overlap)
+    pkg.csd_set_tuning(args.chunk_bytes, args.ctas_per_sm, args.block_threads)
     bench = Bench(wl, tau, device, seed=rank)
     use_graph = not args.eager
     if use_graph:
@@ -413,6 +414,9 @@ def main():
     ap.add_argument("--eager", action="store_true", help="launch every step from Python instead of replaying a graph")
     ap.add_argument("--no-overlap", action="store_true",
                     help="plain stream-ordered launches (no programmatic dependent launch between steps)")
+    ap.add_argument("--chunk-bytes", type=int, default=0, help="override the automatic chunk size (0 = automatic)")
+    ap.add_argument("--ctas-per-sm", type=int, default=0, help="override the resident blocks per SM (0 = automatic)")
+    ap.add_argument("--block-threads", type=int, default=0, help="override the threads per block (0 = automatic)")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extras", action="store_true", help="also time the other workloads (extra keys, same line)")

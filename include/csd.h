@@ -101,7 +101,7 @@ typedef struct {
  */
 
 /* Allocate an empty table on `device` (cudaSetDevice is called and left set).
- * n_slots: power of two, >= 64.  lambda: frequency threshold of the candidate
+ * n_slots: power of two, 64 .. 2^30.  lambda: frequency threshold of the candidate
  * proposal test T[(d,t*)] >= lambda (the paper's main protocol uses 6; 0 makes
  * every divergence a candidate).  Synchronises the device once.
  * Errors: INVALID_ARG (null out, bad n_slots), OOM, CUDA. */
@@ -125,7 +125,8 @@ size_t csd_workspace_bytes(int B, int K, int V, csd_dtype_t dtype);
 /* Zero a workspace.  Required once before its first use (and after any aborted
  * launch); the kernels leave the counters zeroed again on completion, so the
  * same workspace can be reused step after step without further clearing.  One
- * workspace serves one step at a time. */
+ * workspace serves one step at a time, and all steps that use it are issued on
+ * one stream. */
 csd_status_t csd_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 
 /* The verification loop of Algorithm 1 (greedy) for all B rows, read-only on the
@@ -225,20 +226,21 @@ csd_status_t csd_ocm_stats(const csd_ocm_t *ocm, csd_stats_t *host_out, void *st
  * -inf for tau == 0.  Host function. */
 float csd_scg_threshold(float tau);
 
-/* Launch shape a step of this size uses: grid blocks, threads per block, warps that
- * own a span of the logits, and partial-result slots reserved per logit row.  Host
- * function; for reports and tests. */
+/* Launch shape a step of this size uses: grid blocks (each owns an equal contiguous
+ * share of the logits), threads per block, elements per chunk (the run of one logit row
+ * that a warp reduces at a time) and partial results kept per logit row.  Host function;
+ * for reports and tests. */
 csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype,
-                              int *grid, int *block, int *workers, int *parts_per_row);
+                              int *grid, int *block, int *chunk_elems, int *parts_per_row);
 
-/* Expert knob, process-wide: override the automatic work split.  parts_per_row: cap
- * on the number of warps that share one logit row (0 = automatic, which is 32; small
- * values mean fewer, longer spans); ctas_per_sm: resident blocks per SM of the
- * persistent grid (1..4; 0 = automatic, which is 4).  Changes csd_workspace_bytes:
- * size workspaces after calling it.  Results stay bit-reproducible for a fixed
- * setting; the low-order bits of the sums s may differ between settings (different
- * summation trees).  Host function. */
-csd_status_t csd_set_tuning(int parts_per_row, int ctas_per_sm);
+/* Expert knob, process-wide: override the automatic work split.  chunk_bytes: bytes of
+ * one logit row reduced by a warp at a time (multiple of 512; 0 = automatic, 8192);
+ * ctas_per_sm: blocks of the persistent grid per SM (0 = automatic, 4); block_threads:
+ * threads per block (multiple of 32, at most 1024; 0 = automatic, 256).  Changes
+ * csd_workspace_bytes: size workspaces after calling it.  Results stay
+ * bit-reproducible for a fixed setting; the low-order bits of the sums s may differ
+ * between settings (different summation trees).  Host function. */
+csd_status_t csd_set_tuning(int chunk_bytes, int ctas_per_sm, int block_threads);
 
 /* Process-wide, off by default.  When on, csd_verify / csd_step launch with
  * programmatic stream serialization: the kernel may start, and stream logits, while

@@ -78,7 +78,7 @@ def lib():
         "csd_ocm_stats": (c_int, [c_void_p, POINTER(Stats), c_void_p]),
         "csd_scg_threshold": (c_float, [c_float]),
         "csd_launch_shape": (c_int, [c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
-        "csd_set_tuning": (c_int, [c_int, c_int]),
+        "csd_set_tuning": (c_int, [c_int, c_int, c_int]),
         "csd_set_overlap": (c_int, [c_int]),
         "csd_status_string": (c_char_p, [c_int]),
     }
@@ -116,8 +116,8 @@ def csd_scg_threshold(tau: float) -> float:
     return float(lib().csd_scg_threshold(c_float(tau)))
 
 
-def csd_set_tuning(parts_per_row: int = 0, ctas_per_sm: int = 0):
-    _check(lib().csd_set_tuning(parts_per_row, ctas_per_sm), "csd_set_tuning")
+def csd_set_tuning(chunk_bytes: int = 0, ctas_per_sm: int = 0, block_threads: int = 0):
+    _check(lib().csd_set_tuning(chunk_bytes, ctas_per_sm, block_threads), "csd_set_tuning")
 
 
 def csd_set_overlap(enable: bool):
@@ -127,7 +127,7 @@ def csd_set_overlap(enable: bool):
 def csd_launch_shape(B, K, V, dtype_code):
     g, b, te, tr = c_int(), c_int(), c_int(), c_int()
     _check(lib().csd_launch_shape(B, K, V, dtype_code, byref(g), byref(b), byref(te), byref(tr)), "csd_launch_shape")
-    return dict(grid=g.value, block=b.value, workers=te.value, parts_per_row=tr.value)
+    return dict(grid=g.value, block=b.value, chunk_elems=te.value, parts_per_row=tr.value)
 
 
 def csd_workspace_bytes(B, K, V, dtype_code) -> int:

@@ -24,8 +24,9 @@ namespace {
 
 constexpr int kDefaultSms = 148;   // B200; used only when no device can be queried
 
-int g_parts_per_row_override = 0;
+int g_chunk_bytes_override = 0;
 int g_ctas_per_sm_override = 0;
+int g_block_threads_override = 0;
 int g_overlap_steps = 0;
 
 int sm_count()
@@ -43,11 +44,12 @@ int sm_count()
 }
 
 struct Shape {
-    int grid;
-    int n_workers;         // warps owning a span
+    int grid;              // blocks = spans of the unit space
+    int block;             // threads per block
     int unit_elems;        // elements per 512-byte unit
     int units_per_row;
     int slots_per_row;     // partial slots reserved per logit row
+    int chunk_units;       // units per chunk of the in-block hand-out
     long long total_units;
 };
 
@@ -62,28 +64,34 @@ bool shape_ok(int B, int K, int V, csd_dtype_t dt)
     return static_cast<long long>(B) * (K + 1) < (1ll << 31) && static_cast<long long>(B) * K < (1ll << 31);
 }
 
-// The unit space (R rows x U units of 512 bytes) is split evenly over W warps.  W is the
-// persistent grid's warp count, capped so that a row is touched by at most ~33 warps
-// (few partials per row keeps the per-row fold short) and never above the unit count.
+// The unit space (R rows x U units of 512 bytes) is split evenly over the blocks of a
+// persistent grid: as many blocks as fit the machine, but no more than 64 per row (few
+// partials per row keep the last fold short), at least ~8 KiB each, never more than units.
 Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
 {
     const int eb = elt_bytes(dt);
     const int ctas_per_sm = g_ctas_per_sm_override > 0 ? g_ctas_per_sm_override : 4;
-    const int parts_cap = g_parts_per_row_override > 0 ? g_parts_per_row_override : 32;
     const long long rows = static_cast<long long>(B) * (K + 1);
     Shape s;
+    s.block = g_block_threads_override > 0 ? g_block_threads_override : kThreads;
     s.unit_elems = kUnitBytes / eb;
     s.units_per_row = (V + s.unit_elems - 1) / s.unit_elems;
     s.total_units = rows * s.units_per_row;
-    long long workers = static_cast<long long>(sm_count()) * ctas_per_sm * kWarps;
-    if (workers > rows * parts_cap) workers = rows * parts_cap;
-    if (workers > s.total_units) workers = s.total_units;
-    s.n_workers = static_cast<int>(workers);
-    s.grid = static_cast<int>((workers + kWarps - 1) / kWarps);
-    // span boundaries lie at floor(w*T/W): at most ceil((U-1)*W/T) of them fall inside a row
-    long long slots = ((s.units_per_row - 1) * workers + s.total_units - 1) / s.total_units + 1;
+    long long blocks = static_cast<long long>(sm_count()) * ctas_per_sm;
+    if (blocks > rows * 64) blocks = rows * 64;
+    if (blocks > (s.total_units + 15) / 16) blocks = (s.total_units + 15) / 16;
+    if (blocks < 1) blocks = 1;
+    s.grid = static_cast<int>(blocks);
+    // span boundaries lie at floor(c*T/G): at most ceil((U-1)*G/T) of them fall inside a row
+    long long slots = ((s.units_per_row - 1) * blocks + s.total_units - 1) / s.total_units + 1;
     if (slots > s.units_per_row) slots = s.units_per_row;
     s.slots_per_row = static_cast<int>(slots < 1 ? 1 : slots);
+    // chunks: 8 KiB unless overridden, grown so that a block's span fits its chunk table
+    long long chunk_units = (g_chunk_bytes_override > 0 ? g_chunk_bytes_override : 8192) / kUnitBytes;
+    const long long span_max = (s.total_units + blocks - 1) / blocks;
+    const long long need = (span_max + (kMaxChunks - kMaxSegs - 2) - 1) / (kMaxChunks - kMaxSegs - 2);
+    if (chunk_units < need) chunk_units = (need + 7) / 8 * 8;
+    s.chunk_units = static_cast<int>(chunk_units);
     return s;
 }
 
@@ -98,7 +106,7 @@ WorkspaceLayout ws_layout(int B, int K, const Shape &s)
     WorkspaceLayout w;
     w.partials_off = 0;
     w.hint_off = align_up(static_cast<size_t>(B) * (K + 1) * s.slots_per_row * sizeof(Partial), 256);
-    w.b_ticket_off = align_up(w.hint_off + static_cast<size_t>(B) * K * sizeof(long long), 256);
+    w.b_ticket_off = align_up(w.hint_off + static_cast<size_t>(B) * K * sizeof(int), 256);
     w.g_ticket_off = align_up(w.b_ticket_off + static_cast<size_t>(B) * sizeof(unsigned int), 16);
     w.total = align_up(w.g_ticket_off + 16, 256);
     return w;
@@ -147,13 +155,14 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     if (diag) p.diag = *diag;
     char *ws = static_cast<char *>(workspace);
     p.partials = reinterpret_cast<Partial *>(ws + w.partials_off);
-    p.slot_hint = reinterpret_cast<long long *>(ws + w.hint_off);
+    p.slot_hint = reinterpret_cast<int *>(ws + w.hint_off);
     p.b_ticket = reinterpret_cast<unsigned int *>(ws + w.b_ticket_off);
     p.g_ticket = reinterpret_cast<unsigned int *>(ws + w.g_ticket_off);
-    p.n_workers = s.n_workers;
+    p.n_spans = s.grid;
     p.unit_elems = s.unit_elems;
     p.units_per_row = s.units_per_row;
     p.slots_per_row = s.slots_per_row;
+    p.chunk_units = s.chunk_units;
     p.total_units = s.total_units;
 
     const int eb = elt_bytes(dtype);
@@ -163,7 +172,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(s.grid);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(s.block);
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     if (g_overlap_steps) {
@@ -209,7 +218,7 @@ csd_status_t csd_ocm_create(csd_ocm_t **out, uint64_t n_slots, uint32_t lambda, 
 {
     if (!out) return CSD_ERR_INVALID_ARG;
     *out = nullptr;
-    if (n_slots < 64 || (n_slots & (n_slots - 1)) != 0 || n_slots > (1ull << 40)) return CSD_ERR_INVALID_ARG;
+    if (n_slots < 64 || (n_slots & (n_slots - 1)) != 0 || n_slots > (1ull << 30)) return CSD_ERR_INVALID_ARG;
     if (cudaSetDevice(device) != cudaSuccess) {
         (void)cudaGetLastError();
         return CSD_ERR_CUDA;
@@ -443,24 +452,26 @@ float csd_scg_threshold(float tau)
     return static_cast<float>(std::log(static_cast<double>(tau)));
 }
 
-csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype, int *grid, int *block, int *workers,
+csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype, int *grid, int *block, int *chunk_elems,
                               int *parts_per_row)
 {
     if (!shape_ok(B, K, V, dtype)) return CSD_ERR_INVALID_ARG;
     const Shape s = pick_shape(B, K, V, dtype);
     if (grid) *grid = s.grid;
-    if (block) *block = kThreads;
-    if (workers) *workers = s.n_workers;
+    if (block) *block = s.block;
+    if (chunk_elems) *chunk_elems = s.chunk_units * s.unit_elems;
     if (parts_per_row) *parts_per_row = s.slots_per_row;
     return CSD_OK;
 }
 
-csd_status_t csd_set_tuning(int parts_per_row, int ctas_per_sm)
+csd_status_t csd_set_tuning(int chunk_bytes, int ctas_per_sm, int block_threads)
 {
-    if (parts_per_row < 0 || parts_per_row > 4096) return CSD_ERR_INVALID_ARG;
-    if (ctas_per_sm < 0 || ctas_per_sm > 4) return CSD_ERR_INVALID_ARG;
-    g_parts_per_row_override = parts_per_row;
+    if (chunk_bytes != 0 && (chunk_bytes < 512 || chunk_bytes % 512 != 0 || chunk_bytes > (1 << 22))) return CSD_ERR_INVALID_ARG;
+    if (ctas_per_sm < 0 || ctas_per_sm > 8) return CSD_ERR_INVALID_ARG;
+    if (block_threads != 0 && (block_threads < 32 || block_threads > 1024 || block_threads % 32 != 0)) return CSD_ERR_INVALID_ARG;
+    g_chunk_bytes_override = chunk_bytes;
     g_ctas_per_sm_override = ctas_per_sm;
+    g_block_threads_override = block_threads;
     return CSD_OK;
 }
 

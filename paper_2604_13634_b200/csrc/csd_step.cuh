@@ -4,25 +4,30 @@
 //
 // Work decomposition
 //   * The R = B*(K+1) logit rows, each cut into 512-byte units, form one long unit
-//     space that is split EVENLY and contiguously over the W warps of a persistent
-//     grid (warp w owns units [w*T/W, (w+1)*T/W)).  Every warp streams the same number
-//     of bytes +-512, a warp touches one or two rows, and a row is described by about
-//     W/R + 1 partial results (the host caps W so that this stays <= ~33).
-//   * A warp reduces its part of a row on its own: a lane keeps 8 x 16 bytes in flight,
-//     carries a running maximum, an integer reference exponent and four independent
-//     sum accumulators; only the iteration in which the maximum last improved is
+//     space that is split EVENLY and contiguously over the G blocks of a persistent
+//     grid (block c owns units [c*T/G, (c+1)*T/G)); a block touches one or a few rows.
+//   * Inside a block the span is cut into fixed chunks (8 KiB by default, never across
+//     a row) that the block's warps pull from a shared-memory counter.  Shared-memory
+//     atomics cost next to nothing, so the hand-out can be this fine, and it evens out
+//     the large warp-to-warp differences in memory latency: a block is done when its
+//     bytes are done, not when its unluckiest warp is.  The chunk geometry is fixed,
+//     so which warp reduces a chunk has no effect on any result bit.
+//   * A warp reduces a chunk on its own: a lane keeps 8 x 16 bytes in flight, carries a
+//     running maximum, an integer reference exponent and four independent sum
+//     accumulators; only the iteration in which the maximum last improved is
 //     remembered, and the exact lowest arg-max index is recovered by re-reading that
-//     one iteration (an L2 hit).  No block barrier anywhere.
-//   * Partials stay in registers (lane j holds the j-th row part) until the warp's span
-//     is done; then one store per lane, ONE fence per warp, and one ticket per batch
-//     row touched.  Everything before that point reads only the logits, so with
-//     programmatic dependent launch the streaming phase of step n+1 overlaps the tail
-//     of step n: the only wait on the previous launch sits just before the first
-//     workspace write.
-//   * Whichever warp delivers a batch row's last part finalises it: the row's partials
-//     are fetched together and folded by a segmented warp scan in a fixed order
-//     (bit-reproducible sums), lanes 0..K-1 take the per-position decisions, a ballot
-//     gives the accepted prefix.
+//     one iteration (an L2 hit).  Chunk results go to a shared-memory table.
+//   * The warp that delivers the last chunk of a row's part folds that part (fixed
+//     order) while the others keep streaming; the warp that completes the block's last
+//     fold publishes one partial per (block, row) to global memory: one fence and one
+//     ticket per batch row touched, per BLOCK.  Everything before that reads only the
+//     logits, so with programmatic dependent launch the streaming of step n+1 overlaps
+//     the tail of step n: the only wait on the previous launch sits just before the
+//     first global write.
+//   * Whichever block delivers a batch row's last part finalises it (one warp): the
+//     few partials per row are folded by fixed-shape butterflies (maximum first, then
+//     the sums rescaled to the row's reference: bit-reproducible), lanes 0..K-1 take
+//     the per-position decisions, a ballot gives the accepted prefix.
 //   * Memory update without a second probe: the look-up already found each recorded
 //     pair's slot (absent pairs get an empty slot reserved with count 0, which no
 //     look-up can tell from "absent"), and leaves it as a hint.  The warp finalising
@@ -54,20 +59,21 @@ struct StepParams {
     int *rej_d;
     int *rej_t;
     csd_diag_t diag;
-    Partial *partials;       // [R * slots_per_row]
-    long long *slot_hint;    // [B * K] slot of each recorded pair (see kHint*)
+    Partial *partials;       // [R * slots_per_row]: one slot per (row, block touching it)
+    int *slot_hint;          // [B * K] slot of each recorded pair (see kHint*)
     unsigned int *b_ticket;  // [B]
     unsigned int *g_ticket;  // [1]
-    int n_workers;           // W: warps that own a span of the unit space
+    int n_spans;             // G: blocks that own a span of the unit space
     int unit_elems;          // elements per 512-byte unit
     int units_per_row;       // U = ceil(V / unit_elems)
-    int slots_per_row;       // S >= most warps that can touch one row
+    int slots_per_row;       // S >= most blocks that can touch one row
+    int chunk_units;         // units per chunk
     long long total_units;   // T = R * U
 };
 
-constexpr long long kHintNone = -1;          // nothing to record at this position
-constexpr long long kHintAbsent = -2;        // recorded pair not in the table and no slot reserved
-constexpr long long kHintCareful = 1ll << 62; // count close to saturation: add with the wrap check
+constexpr int kHintNone = -1;          // nothing to record at this position
+constexpr int kHintAbsent = -2;        // recorded pair not in the table and no slot reserved
+constexpr int kHintCareful = 1 << 30;  // count close to saturation: add with the wrap check
 
 // ---- element access policies ---------------------------------------------------------
 
@@ -284,21 +290,32 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
     return p;
 }
 
-// ---- the even split of the unit space ---------------------------------------------------
-
-__device__ __forceinline__ long long span_begin(const StepParams &p, int w)
-{
-    return static_cast<long long>(w) * p.total_units / p.n_workers;
-}
-
-// The warp whose span holds global unit g: the largest w with span_begin(w) <= g.
-__device__ __forceinline__ int owner_of(const StepParams &p, long long g)
-{
-    return static_cast<int>(((g + 1) * p.n_workers - 1) / p.total_units);
-}
-
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ---- the even split of the unit space over blocks -----------------------------------------
+
+__device__ __forceinline__ long long span_begin(const StepParams &p, int c)
+{
+    return static_cast<long long>(c) * p.total_units / p.n_spans;
+}
+
+// The block whose span holds global unit g: the largest c with span_begin(c) <= g.
+__device__ __forceinline__ int owner_of(const StepParams &p, long long g)
+{
+    return static_cast<int>(((g + 1) * p.n_spans - 1) / p.total_units);
+}
+
+constexpr int kMaxSegs = 32;       // row parts a block handles between two block barriers
+constexpr int kMaxChunks = 1024;   // chunk results held in shared memory at a time
+
+struct BlockState {
+    unsigned int next_chunk;            // hand-out counter
+    unsigned int segs_folded;           // row parts folded so far
+    unsigned int seg_done[kMaxSegs];    // chunks delivered per row part
+    Partial seg_result[kMaxSegs];
+    Partial chunk_part[kMaxChunks];
+};
 
 // ---- S2..S5 for one batch row, by one warp ------------------------------------------
 
@@ -306,8 +323,7 @@ struct RowScratch {
     float m[CSD_MAX_K + 1];
     float s[CSD_MAX_K + 1];
     int t[CSD_MAX_K + 1];
-    int first[CSD_MAX_K + 1];   // first warp touching the row
-    int parts[CSD_MAX_K + 1];   // number of warps touching the row
+    int parts[CSD_MAX_K + 1];   // number of blocks touching the row
 };
 
 enum UpdateRegime { kRegimeRoom = 0, kRegimeFull = 1, kRegimeTransition = 2 };
@@ -323,14 +339,92 @@ __device__ __forceinline__ int update_regime(const StepParams &p)
     return kRegimeTransition;
 }
 
+// Butterfly fold of one value per lane inside aligned groups of `width` lanes: maximum and
+// its lowest index first, then the sums rescaled (exactly) to the group's reference.
+// Every lane of a group ends with the group's total.
+__device__ __forceinline__ Partial butterfly_fold(Partial v, int width)
+{
+    float m = v.m;
+    int idx = v.idx;
+    for (int o = 1; o < width; o <<= 1) {
+        const float om = __shfl_xor_sync(kFull, m, o);
+        const int oi = __shfl_xor_sync(kFull, idx, o);
+        const bool take = (om > m) || (om == m && oi < idx);
+        m = take ? om : m;
+        idx = take ? oi : idx;
+    }
+    const float c = (m == -INFINITY) ? kNoRef : rintf(m * kLog2e);
+    float s = v.s * pow2_nonpos(v.c - c);
+    for (int o = 1; o < width; o <<= 1) s += __shfl_xor_sync(kFull, s, o);
+    Partial r;
+    r.m = m;
+    r.idx = idx;
+    r.c = c;
+    r.s = s;
+    return r;
+}
+
+// Fold the per-block partials of the K+1 logit rows of batch row b (S1, last level).  The
+// lanes are arranged as (32 / width) rows x width slots, width = the power of two >= the
+// slots per row (at most 32; more slots are pre-folded in lane order).
+__device__ __forceinline__ void fold_rows(const StepParams &p, int b, int lane, RowScratch &rs)
+{
+    const int K1 = p.K + 1, S = p.slots_per_row;
+    int width = 1;
+    while (width < S && width < 32) width <<= 1;
+    const int rows_per_pass = 32 / width;
+    const int sub = lane / width;          // which row of the pass
+    const int k0 = lane - sub * width;     // first slot this lane folds
+    const size_t row0 = (size_t)b * K1;
+    const Partial *part = p.partials + row0 * S;
+
+    for (int r = lane; r < K1; r += 32) {
+        const long long u0 = static_cast<long long>(row0 + r) * p.units_per_row;
+        rs.parts[r] = owner_of(p, u0 + p.units_per_row - 1) - owner_of(p, u0) + 1;
+    }
+    __syncwarp();
+
+    for (int r0 = 0; r0 < K1; r0 += rows_per_pass * 4) {
+        Partial v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int row = r0 + q * rows_per_pass + sub;
+            v[q] = partial_identity();
+            if (row < K1) {
+                const int np = rs.parts[row];
+                for (int k = k0; k < np; k += width) {       // one trip unless a row has > 32 parts
+                    const Partial x = ld_partial_cg(part + (size_t)row * S + k);
+                    v[q] = (k == k0) ? x : combine(v[q], x);
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int row = r0 + q * rows_per_pass + sub;
+            if (r0 + q * rows_per_pass >= K1) break;
+            const Partial t = butterfly_fold(v[q], width);
+            if (k0 == 0 && row < K1) {
+                // sum exp(x - m) = s * 2^(c - m log2 e)
+                const float s_m = t.s * exp2f(fmaf(-t.m, kLog2e, t.c));
+                rs.m[row] = t.m;
+                rs.s[row] = s_m;
+                rs.t[row] = t.idx;
+                if (!(s_m == s_m) || s_m == INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
+                if (p.diag.m) p.diag.m[row0 + row] = t.m;
+                if (p.diag.s) p.diag.s[row0 + row] = s_m;
+                if (p.diag.lse) p.diag.lse[row0 + row] = t.m + logf(s_m);
+                if (p.diag.t) p.diag.t[row0 + row] = t.idx;
+            }
+        }
+    }
+    __syncwarp();
+}
+
 template <typename L>
 __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScratch &rs)
 {
     using E = typename L::elem;
-    const int K = p.K, K1 = p.K + 1, S = p.slots_per_row;
-    const int n = K1 * S;
-    const size_t row0 = (size_t)b * K1;
-    const Partial *part = p.partials + row0 * S;
+    const int K = p.K;
 
     // S2 (first half): the draft tokens and their logits do not depend on the
     // reduction, so their loads are issued before the partials are folded.
@@ -346,62 +440,8 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
         }
     }
     const int regime = p.do_update ? update_regime(p) : kRegimeFull;
-    for (int r = lane; r < K1; r += 32) {
-        const long long u0 = static_cast<long long>(row0 + r) * p.units_per_row;
-        const int wf = owner_of(p, u0);
-        rs.first[r] = wf;
-        rs.parts[r] = owner_of(p, u0 + p.units_per_row - 1) - wf + 1;
-    }
-    __syncwarp();
 
-    // S1 (second half): fold the K+1 rows' partials with a segmented inclusive scan,
-    // 32 slots at a time, always in the same order; up to 256 slots are fetched at once.
-    Partial carry = partial_identity();
-    int carry_row = -1;
-    for (int g0 = 0; g0 < n; g0 += 256) {
-        Partial pre[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int e = g0 + q * 32 + lane;
-            pre[q] = partial_identity();
-            if (e < n) {
-                const int row = e / S;
-                if (e - row * S < rs.parts[row]) pre[q] = ld_partial_cg(part + e);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int base = g0 + q * 32;
-            if (base >= n) break;
-            const int e = base + lane;
-            const bool in = e < n;
-            const int row = in ? e / S : 0x7ffffff0 + lane;
-            Partial v = pre[q];
-            if (lane == 0 && carry_row == row) v = combine(carry, v);
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const Partial up = shfl_up_partial(v, o);
-                const int up_row = __shfl_up_sync(kFull, row, o);
-                if (lane >= o && up_row == row) v = combine(up, v);
-            }
-            if (in && e - row * S == rs.parts[row] - 1) {
-                // last part of a row: v is the row's total.  sum exp(x - m) = s * 2^(c - m log2 e)
-                const float r = fmaf(-v.m, kLog2e, v.c);
-                const float s_m = v.s * exp2f(r);
-                rs.m[row] = v.m;
-                rs.s[row] = s_m;
-                rs.t[row] = v.idx;
-                if (!(s_m == s_m) || s_m == INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
-                if (p.diag.m) p.diag.m[row0 + row] = v.m;
-                if (p.diag.s) p.diag.s[row0 + row] = s_m;
-                if (p.diag.lse) p.diag.lse[row0 + row] = v.m + logf(s_m);
-                if (p.diag.t) p.diag.t[row0 + row] = v.idx;
-            }
-            carry = shfl_partial(v, 31);
-            carry_row = __shfl_sync(kFull, row, 31);
-        }
-    }
-    __syncwarp();
+    fold_rows(p, b, lane, rs);
 
     // S2 (second half), S3, S4 per position; S5 across the warp.
     bool match = false, ok = false;
@@ -440,10 +480,10 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
         p.rej_t[pos] = record ? t : -1;
         if (p.do_update) {
             // S6, first half: leave the slot of every recorded pair for the final adder
-            long long hint = kHintNone;
+            int hint = kHintNone;
             if (record) {
                 if (slot < 0 && regime == kRegimeRoom) slot = ocm_reserve(p.ocm, make_key(d, t));
-                hint = slot < 0 ? kHintAbsent : slot;
+                hint = slot < 0 ? kHintAbsent : static_cast<int>(slot);
                 const unsigned int room = 0xffffffffu - static_cast<unsigned int>(p.B * p.K);
                 if (slot >= 0 && cnt > room) hint |= kHintCareful;
             }
@@ -478,15 +518,15 @@ __device__ void apply_step_update(const StepParams &p, int lane, CanonScratch &c
         return;
     }
     unsigned int dropped = 0;
-    for (int j0 = 0; j0 < n; j0 += 256) {
-        long long h[8];
+    for (int j0 = 0; j0 < n; j0 += 32 * 16) {
+        int h[16];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < 16; ++q) {
             const int j = j0 + q * 32 + lane;
             h[q] = j < n ? __ldcg(p.slot_hint + j) : kHintNone;
         }
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < 16; ++q) {
             if (h[q] >= 0) {
                 const unsigned long long s = static_cast<unsigned long long>(h[q] & ~kHintCareful);
                 if (h[q] & kHintCareful)
@@ -504,102 +544,166 @@ __device__ void apply_step_update(const StepParams &p, int lane, CanonScratch &c
     __syncwarp();
 }
 
+// Publication of a block's row parts and everything that may follow from it: tickets,
+// batch-row finalisation, the memory update.  Executed by ONE warp of the block.
+//   nseg row parts, rows first_row .. first_row + nseg - 1, results in bs.seg_result;
+//   next_b: batch row of the next row this block will still publish, or -1.
+template <typename L>
+__device__ void publish_and_finalize(const StepParams &p, BlockState &bs, RowScratch &rs, CanonScratch &canon,
+                                     int first_row, int nseg, int next_b, int lane)
+{
+    const int K1 = p.K + 1;
+    const int U = p.units_per_row;
+    // the first access to memory that the previous launch on the stream may still be using
+    pdl_wait();
+    int my_b = -1;
+    if (lane < nseg) {
+        const int row = first_row + lane;
+        const int slot = static_cast<int>(blockIdx.x) - owner_of(p, static_cast<long long>(row) * U);
+        if (slot < p.slots_per_row) st_partial_cg(p.partials + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
+        else atomicOr(&p.ocm.stats->flags, CSD_FLAG_PROBE_EXHAUSTED);
+        my_b = row / K1;
+    }
+    __threadfence();
+    __syncwarp();
+    const int below_b = __shfl_down_sync(kFull, my_b, 1);
+    bool completes = false;
+    if (lane < nseg) {
+        // the lane holding this block's last part of a batch row takes that row's ticket
+        const bool closes = (lane == nseg - 1) ? (my_b != next_b) : (below_b != my_b);
+        if (closes) {
+            const long long u0 = static_cast<long long>(my_b) * K1 * U;
+            const unsigned int expected = owner_of(p, u0 + static_cast<long long>(K1) * U - 1) - owner_of(p, u0) + 1;
+            completes = atomicAdd(p.b_ticket + my_b, 1u) == expected - 1;
+        }
+    }
+    unsigned int todo = __ballot_sync(kFull, completes);
+
+    // ---- this block delivered a batch row's last part: S2..S5 ----
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int b = __shfl_sync(kFull, my_b, src);
+        __threadfence();
+        finalize_batch_row<L>(p, b, lane, rs);
+        bool last = false;
+        if (lane == 0) p.b_ticket[b] = 0u;               // ready for the next launch
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) last = atomicAdd(p.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
+        last = __shfl_sync(kFull, last, 0);
+        if (!last) continue;
+
+        // ---- every batch row is final: S6 ----
+        __threadfence();
+        if (p.do_update) apply_step_update(p, lane, canon);
+        if (lane == 0) {
+            OcmStatsDev *st = p.ocm.stats;
+            __threadfence();
+            st->n_keys_start = atomicAdd(&st->n_keys, 0ull);
+            atomicAdd(&st->steps, 1ull);
+            *p.g_ticket = 0u;
+        }
+    }
+}
+
 // ---- the kernel ------------------------------------------------------------------------
 
 template <typename L>
-__global__ void __launch_bounds__(kThreads, 4) csd_step_kernel(const __grid_constant__ StepParams p)
+__global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ StepParams p)
 {
-    __shared__ RowScratch row_scratch[kWarps];
+    __shared__ BlockState bs;
+    __shared__ RowScratch row_scratch;
     __shared__ CanonScratch canon;
 
     using E = typename L::elem;
     pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    const int w = blockIdx.x * kWarps + warp;
-    if (w >= p.n_workers) return;
     const int K1 = p.K + 1;
     const int U = p.units_per_row;
-    long long g = span_begin(p, w);
-    const long long g_end = span_begin(p, w + 1);
+    const int CH = p.chunk_units;
+    const int cpr = (U + CH - 1) / CH;                       // chunks of a whole row
+    long long g = span_begin(p, blockIdx.x);
+    const long long g_end = span_begin(p, blockIdx.x + 1);
 
     while (g < g_end) {
-        // ---- S1: reduce this warp's part of up to 32 rows, lane j keeping the j-th ----
-        Partial mine = partial_identity();
-        int my_row = -1;
-        int n_held = 0;
-        while (g < g_end && n_held < 32) {
-            const long long row = g / U;
-            const int o0 = static_cast<int>(g - row * U);
-            const long long left = g_end - row * U;
-            const int o1 = left < U ? static_cast<int>(left) : U;
+        // ---- a window: up to kMaxSegs consecutive row parts of this block's span ----
+        const long long row0 = g / U;
+        const int o0 = static_cast<int>(g - row0 * U);
+        long long w_end = (row0 + kMaxSegs) * U;
+        if (w_end > g_end) w_end = g_end;
+        const int nseg = static_cast<int>((w_end - row0 * U + U - 1) / U);
+        const long long first_len = w_end - row0 * U;        // units from row0's start to the window end
+        const int b0 = first_len < U ? static_cast<int>(first_len) : U;
+        const int n0 = (b0 - o0 + CH - 1) / CH;               // chunks of the first row part
+        const int last_units = static_cast<int>(w_end - (row0 + nseg - 1) * U);
+        const int n_last = (last_units + CH - 1) / CH;
+        const int nchunks = nseg == 1 ? n0 : n0 + (nseg - 2) * cpr + n_last;
+
+        if (threadIdx.x == 0) {
+            bs.next_chunk = 0u;
+            bs.segs_folded = 0u;
+        }
+        if (threadIdx.x < kMaxSegs) bs.seg_done[threadIdx.x] = 0u;
+        __syncthreads();
+
+        while (true) {
+            unsigned int q = 0;
+            if (lane == 0) q = atomicAdd(&bs.next_chunk, 1u);
+            q = __shfl_sync(kFull, q, 0);
+            if (q >= static_cast<unsigned int>(nchunks)) break;
+
+            // ---- S1: which row part and which chunk of it ----
+            int seg, k, seg_first, seg_n, ua, ub;
+            if (static_cast<int>(q) < n0) {
+                seg = 0; k = q; seg_first = 0; seg_n = n0; ua = o0; ub = b0;
+            } else {
+                const int r = static_cast<int>(q) - n0;
+                seg = 1 + r / cpr;
+                k = r - (seg - 1) * cpr;
+                seg_first = n0 + (seg - 1) * cpr;
+                ua = 0;
+                if (seg == nseg - 1) { seg_n = n_last; ub = last_units; } else { seg_n = cpr; ub = U; }
+            }
+            const long long row = row0 + seg;
             const long long b = row / K1;
             const int i = static_cast<int>(row - b * K1);
             const E *rp = reinterpret_cast<const E *>(p.logits) + b * p.stride_b + i * p.stride_k;
-            const int e0 = o0 * p.unit_elems;
-            const long long e1l = static_cast<long long>(o1) * p.unit_elems;
+            const int u0 = ua + k * CH;
+            const int u1 = min(ub, u0 + CH);
+            const int e0 = u0 * p.unit_elems;
+            const long long e1l = static_cast<long long>(u1) * p.unit_elems;
             const int e1 = e1l < p.V ? static_cast<int>(e1l) : p.V;
             const Partial r = warp_tile<L>(rp, e0, e1, lane);
-            if (lane == n_held) {
-                mine = r;
-                my_row = static_cast<int>(row);
-            }
-            ++n_held;
-            g = (row + 1) * U;
-        }
-        const int next_b = g < g_end ? static_cast<int>((g / U) / K1) : -1;
 
-        // ---- publish: one store per lane, one fence per warp, one ticket per batch row.
-        //      This is the first access to memory another launch may still be using. ----
-        pdl_wait();
-        int my_b = -1;
-        if (lane < n_held) {
-            const int slot = w - owner_of(p, static_cast<long long>(my_row) * U);
-            if (slot < p.slots_per_row) st_partial_cg(p.partials + (size_t)my_row * p.slots_per_row + slot, mine);
-            else atomicOr(&p.ocm.stats->flags, CSD_FLAG_PROBE_EXHAUSTED);
-            my_b = my_row / K1;
-        }
-        __threadfence();
-        __syncwarp();
-        const int below_b = __shfl_down_sync(kFull, my_b, 1);
-        bool completes = false;
-        if (lane < n_held) {
-            // the lane holding this warp's last part of a batch row takes that row's ticket
-            const bool closes = (lane == n_held - 1) ? (my_b != next_b) : (below_b != my_b);
-            if (closes) {
-                const long long u0 = static_cast<long long>(my_b) * K1 * U;
-                const unsigned int expected = owner_of(p, u0 + static_cast<long long>(K1) * U - 1) - owner_of(p, u0) + 1;
-                completes = atomicAdd(p.b_ticket + my_b, 1u) == expected - 1;
-            }
-        }
-        unsigned int todo = __ballot_sync(kFull, completes);
-
-        // ---- the warp that delivered a batch row's last part finalises it: S2..S5 ----
-        while (todo) {
-            const int src = __ffs(todo) - 1;
-            todo &= todo - 1;
-            const int b = __shfl_sync(kFull, my_b, src);
-            __threadfence();
-            finalize_batch_row<L>(p, b, lane, row_scratch[warp]);
-            bool last = false;
-            if (lane == 0) p.b_ticket[b] = 0u;               // ready for the next launch
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) last = atomicAdd(p.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
-            last = __shfl_sync(kFull, last, 0);
-            if (!last) continue;
-
-            // ---- every batch row is final: S6 ----
-            __threadfence();
-            if (p.do_update) apply_step_update(p, lane, canon);
+            // ---- deliver it; the warp bringing a row part's last chunk folds that part ----
+            bool seg_complete = false;
             if (lane == 0) {
-                OcmStatsDev *st = p.ocm.stats;
-                __threadfence();
-                st->n_keys_start = atomicAdd(&st->n_keys, 0ull);
-                atomicAdd(&st->steps, 1ull);
-                *p.g_ticket = 0u;
+                bs.chunk_part[q] = r;
+                __threadfence_block();
+                seg_complete = atomicAdd(&bs.seg_done[seg], 1u) == static_cast<unsigned int>(seg_n) - 1u;
             }
+            if (!__shfl_sync(kFull, seg_complete, 0)) continue;
+            __threadfence_block();
+            Partial v = partial_identity();
+            for (int j = lane; j < seg_n; j += 32) {
+                const Partial x = bs.chunk_part[seg_first + j];
+                v = (j == lane) ? x : combine(v, x);
+            }
+            v = butterfly_fold(v, 32);
+            bool block_complete = false;
+            if (lane == 0) {
+                bs.seg_result[seg] = v;
+                __threadfence_block();
+                block_complete = atomicAdd(&bs.segs_folded, 1u) == static_cast<unsigned int>(nseg) - 1u;
+            }
+            if (!__shfl_sync(kFull, block_complete, 0)) continue;
+            __threadfence_block();
+            const int next_b = w_end < g_end ? static_cast<int>((w_end / U) / K1) : -1;
+            publish_and_finalize<L>(p, bs, row_scratch, canon, static_cast<int>(row0), nseg, next_b, lane);
         }
+        g = w_end;
+        if (g < g_end) __syncthreads();       // the next window reuses the shared-memory tables
     }
 }
 

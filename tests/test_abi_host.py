@@ -44,37 +44,41 @@ def test_status_strings(L):
     assert len(seen) == 6 and b"ok" in seen
 
 
+SHAPES = ((1, 4, 32000, 0), (1, 8, 128256, 1), (32, 5, 151936, 1), (128, 8, 128256, 0), (64, 6, 152064, 1),
+          (3, 1, 7, 0), (2, 32, 1000, 1), (1, 1, 1 << 22, 0), (5, 2, 70001, 0), (48, 1, 1 << 20, 0), (30000, 1, 24, 1))
+
+
 def test_shapes_and_workspace(L):
-    for (B, K, V, dt) in ((1, 4, 32000, 0), (1, 8, 128256, 1), (32, 5, 151936, 1), (128, 8, 128256, 0),
-                          (64, 6, 152064, 1), (3, 1, 7, 0), (2, 32, 1000, 1), (1, 1, 1 << 22, 0)):
+    for (B, K, V, dt) in SHAPES:
         s = binding.csd_launch_shape(B, K, V, dt)
         eb = 4 if dt == 0 else 2
         rows = B * (K + 1)
         units = rows * -(-V * eb // 512)
-        assert s["block"] == 256 and s["grid"] == -(-s["workers"] // 8)
-        assert 1 <= s["workers"] <= min(units, 32 * rows, 148 * 4 * 8)
-        assert 1 <= s["parts_per_row"] <= 34
+        assert s["block"] == 256 and 1 <= s["grid"] <= min(148 * 4, units, 64 * rows)
+        assert (s["chunk_elems"] * eb) % 512 == 0 and 1 <= s["parts_per_row"] <= 66
         ws = binding.csd_workspace_bytes(B, K, V, dt)
-        assert ws >= rows * s["parts_per_row"] * 16 + 8 * B * K + 4 * B + 4
+        assert ws >= rows * s["parts_per_row"] * 16 + 4 * B * K + 4 * B + 4
         assert binding.csd_host_staging_bytes(B, K, V, dt) >= rows * V * eb + ws
     assert binding.csd_workspace_bytes(0, 4, 100, 0) == 0
     assert binding.csd_workspace_bytes(1, 33, 100, 0) == 0
     assert binding.csd_workspace_bytes(1, 4, 100, 7) == 0
 
 
-def test_even_split_covers_every_row_within_its_slots():
-    """Host replay of the kernels' span arithmetic: every unit has exactly one owner, owners
-    of a row are consecutive, and no row is touched by more warps than it has slots."""
-    for (B, K, V, dt) in ((1, 4, 32000, 0), (32, 5, 151936, 1), (128, 8, 128256, 0), (64, 6, 152064, 1),
-                          (3, 1, 7, 0), (2, 32, 1000, 1), (5, 2, 70001, 0), (48, 1, 1 << 20, 0)):
+def test_even_split_geometry():
+    """Host replay of the kernels' span arithmetic: every span is non-empty, the blocks touching
+    a row are consecutive and fit the row's slots, and a span never needs more chunk results
+    than a block can hold."""
+    for (B, K, V, dt) in SHAPES:
         s = binding.csd_launch_shape(B, K, V, dt)
         eb = 4 if dt == 0 else 2
         U = -(-V * eb // 512)
         rows = B * (K + 1)
-        T, W = rows * U, s["workers"]
-        begin = [w * T // W for w in range(W + 1)]
-        assert all(begin[w + 1] > begin[w] for w in range(W))          # no empty span
-        owner = lambda g: ((g + 1) * W - 1) // T
+        T, G = rows * U, s["grid"]
+        CH = s["chunk_elems"] * eb // 512
+        begin = [c * T // G for c in range(G + 1)]
+        assert all(begin[c + 1] > begin[c] for c in range(G))
+        assert max(begin[c + 1] - begin[c] for c in range(G)) // CH + 34 <= 1024
+        owner = lambda g: ((g + 1) * G - 1) // T
         for r in list(range(min(rows, 40))) + [rows - 1]:
             first, last = owner(r * U), owner((r + 1) * U - 1)
             assert begin[first] <= r * U < begin[first + 1] and begin[last] <= (r + 1) * U - 1 < begin[last + 1]
@@ -106,7 +110,9 @@ def test_argument_checks_refuse_before_launch(L):
     assert L.csd_ocm_create(ctypes.byref(out), 1000, 6, 0) == 1      # not a power of two
     assert L.csd_ocm_create(ctypes.byref(out), 32, 6, 0) == 1
     assert L.csd_ocm_create(None, 1024, 6, 0) == 1
-    assert L.csd_set_tuning(-1, 0) == 1 and L.csd_set_tuning(0, 9) == 1 and L.csd_set_tuning(0, 0) == 0
+    assert L.csd_ocm_create(ctypes.byref(out), 1 << 31, 6, 0) == 1
+    assert L.csd_set_tuning(1000, 0, 0) == 1 and L.csd_set_tuning(0, 9, 0) == 1 and L.csd_set_tuning(0, 0, 48) == 1
+    assert L.csd_set_tuning(0, 0, 0) == 0
 
 
 def test_binding_refuses_without_device():

@@ -331,24 +331,26 @@ def test_host_entry_point_matches_device_entry_point():
     a.close(); b.close()
 
 
-@pytest.mark.parametrize("parts,ctas", [(1, 1), (2, 2), (8, 4), (300, 3)])
-def test_parity_under_other_splits(parts, ctas):
+@pytest.mark.parametrize("chunk_bytes,ctas,threads", [(512, 4, 256), (4096, 1, 1024), (8192, 2, 512), (36864, 3, 96),
+                                                        (1 << 20, 4, 32), (16384, 8, 128)])
+def test_parity_under_other_splits(chunk_bytes, ctas, threads):
     try:
-        csd_set_tuning(parts, ctas)
+        csd_set_tuning(chunk_bytes, ctas, threads)
         wl = dataclasses.replace(WORKLOADS["ocm_contention"], B=8)
-        assert csd_launch_shape(wl.B, wl.K, wl.V, CSD_BF16)["workers"] <= min(148 * ctas * 8, parts * wl.rows)
+        shape = csd_launch_shape(wl.B, wl.K, wl.V, CSD_BF16)
+        assert shape["block"] == threads and shape["grid"] <= 148 * ctas and shape["chunk_elems"] * 2 >= chunk_bytes
         lockstep(wl, steps=3, tau=0.3, lam=1)
         wl = dataclasses.replace(WORKLOADS["large_batch"], B=4)
         lockstep(wl, steps=2, tau=0.2, lam=1)
     finally:
-        csd_set_tuning(0, 0)
+        csd_set_tuning(0, 0, 0)
 
 
 def test_many_short_rows_per_warp():
-    """Rows far shorter than a warp's span: a warp holds parts of many rows and of several
-    batch rows (more than 32 row parts per warp with the single-block setting)."""
-    for (B, K, V, dtype) in ((600, 3, 160, torch.float32), (97, 32, 520, torch.bfloat16), (3000, 1, 24, torch.bfloat16)):
-        for tuning in ((0, 0), (1, 1)):
+    """Many short rows: a block's span covers far more than 32 rows and several batch rows, so
+    it works through several windows, publishing after each."""
+    for (B, K, V, dtype) in ((600, 3, 160, torch.float32), (97, 32, 520, torch.bfloat16), (30000, 1, 24, torch.bfloat16)):
+        for tuning in ((0, 0, 0), (512, 1, 64)):
             try:
                 csd_set_tuning(*tuning)
                 z, d = _random_inputs(B, K, V, dtype, seed=21)
@@ -360,46 +362,73 @@ def test_many_short_rows_per_warp():
                 compare_memory(ocm, mem)
                 ocm.close()
             finally:
-                csd_set_tuning(0, 0)
+                csd_set_tuning(0, 0, 0)
 
 
 def test_overlapped_launches_match():
-    """Back-to-back steps launched with programmatic stream serialization (the setting the
-    benchmark times) give the same results as plain launches."""
+    """Hundreds of back-to-back steps launched with programmatic stream serialization (the
+    setting the benchmark times), eagerly and as a replayed CUDA graph, give the same
+    results as plain launches; the plain run is pinned to the oracle."""
     from paper_2604_13634_b200 import csd_set_overlap
-    wl = dataclasses.replace(WORKLOADS["batched_serving"], B=8)
+    wl = WORKLOADS["batched_serving"]
     syn = Synth(wl, 4, "cuda")
-    inputs = [syn.step(s) for s in range(6)]
-    results = []
-    for overlap in (False, True):
+    inputs = [syn.step(s) for s in range(5)]         # an odd ring: replays follow each other out of phase
+    reps = 41
+
+    def run(overlap, graph):
         try:
             csd_set_overlap(overlap)
-            ocm = Ocm(4096, 1)
+            ocm = Ocm(wl.ocm_slots, 2)
             bufs = [StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True) for _ in inputs]
-            for rep in range(3):
-                for (z, d), buf in zip(inputs, bufs):        # 18 launches with nothing between them
+            ws = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype)         # one shared workspace, as the benchmark has
+            for b in bufs:
+                b.workspace, b.ws_bytes = ws.workspace, ws.ws_bytes
+
+            def ring():
+                for (z, d), buf in zip(inputs, bufs):
                     csd_step(z, d, ocm, 0.3, buf)
+            if graph:
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    ring()
+                torch.cuda.current_stream().wait_stream(side)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    ring()
+                for _ in range(reps - 1):        # the capture itself runs nothing
+                    g.replay()
+            else:
+                for _ in range(reps):
+                    ring()
             torch.cuda.synchronize()
-            results.append(([(b.accept_len.clone(), b.next_token.clone(), b.rescued_mask.clone(),
-                              b.diag["s"].clone(), b.diag["cnt"].clone()) for b in bufs], ocm.export(), ocm.stats()))
+            out = ([(b.accept_len.clone(), b.next_token.clone(), b.rescued_mask.clone(), b.diag["s"].clone(),
+                     b.diag["cnt"].clone()) for b in bufs], ocm.export(), ocm.stats())
             ocm.close()
+            return out
         finally:
             csd_set_overlap(False)
-    (ra, ea, sa), (rb, eb, sb) = results
-    for x, y in zip(ra, rb):
-        assert all(torch.equal(p, q) for p, q in zip(x, y))
-    assert all(torch.equal(p, q) for p, q in zip(ea, eb)) and sa == sb
-    # and the plain run itself is pinned to the oracle
-    mem = ORACLE.OCM(4096, 1)
-    for rep in range(3):
+
+    ref_out, ref_exp, ref_st = run(False, False)
+    assert ref_st["steps"] == reps * len(inputs) and ref_st["flags"] == 0
+    for overlap, graph in ((True, False), (True, True), (False, True)):
+        out, exp, st = run(overlap, graph)
+        assert st == ref_st, (overlap, graph, st, ref_st)
+        assert all(torch.equal(p, q) for p, q in zip(exp, ref_exp)), (overlap, graph)
+        for x, y in zip(out, ref_out):
+            assert all(torch.equal(p, q) for p, q in zip(x, y)), (overlap, graph)
+    mem = ORACLE.OCM(wl.ocm_slots, 2)
+    for rep in range(reps):
         for z, d in inputs:
             ref = oracle_step(z, d, mem, 0.3)
-    assert np.array_equal(ra[-1][0].cpu().numpy(), ref["accept_len"])
-    assert np.array_equal(ea[2].numpy(), mem.export()[2])
+    assert np.array_equal(ref_out[-1][0].cpu().numpy(), ref["accept_len"])
+    assert np.array_equal(ref_out[-1][2].cpu().numpy(), ref["rescued_mask"])
+    rd, rt, rc = mem.export()
+    assert np.array_equal(ref_exp[0].numpy(), rd) and np.array_equal(ref_exp[2].numpy(), rc)
 
 
 def test_long_rows():
-    """Rows far longer than one warp's share: many warps per row, parts capped by the split."""
+    """Rows of 4 MiB: each is shared by several blocks, and a block's span needs larger chunks."""
     B, K, V = 48, 1, 1 << 20
     z, d = _random_inputs(B, K, V, torch.float32, seed=11)
     ocm = Ocm(256, 0)
