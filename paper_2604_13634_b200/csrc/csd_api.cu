@@ -86,8 +86,8 @@ Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
     long long slots = ((s.units_per_row - 1) * blocks + s.total_units - 1) / s.total_units + 1;
     if (slots > s.units_per_row) slots = s.units_per_row;
     s.slots_per_row = static_cast<int>(slots < 1 ? 1 : slots);
-    // chunks: 8 KiB unless overridden, grown so that a block's span fits its chunk table
-    long long chunk_units = (g_chunk_bytes_override > 0 ? g_chunk_bytes_override : 8192) / kUnitBytes;
+    // chunks: 16 KiB unless overridden, grown so that a block's span fits its chunk table
+    long long chunk_units = (g_chunk_bytes_override > 0 ? g_chunk_bytes_override : 16384) / kUnitBytes;
     const long long span_max = (s.total_units + blocks - 1) / blocks;
     const long long need = (span_max + (kMaxChunks - kMaxSegs - 2) - 1) / (kMaxChunks - kMaxSegs - 2);
     if (chunk_units < need) chunk_units = (need + 7) / 8 * 8;
@@ -98,17 +98,24 @@ Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t partials_off, hint_off, b_ticket_off, g_ticket_off, total;
+    size_t seq_off, half_bytes, partials_off, hint_off, b_ticket_off, g_ticket_off, total;   // *_off within a half
+    size_t half_off[2];
 };
 
+// header {launch sequence, blocks counted in, launches completed} followed by two halves,
+// each {partials | slot hints | per-batch-row tickets | global ticket}
 WorkspaceLayout ws_layout(int B, int K, const Shape &s)
 {
     WorkspaceLayout w;
+    w.seq_off = 0;
     w.partials_off = 0;
     w.hint_off = align_up(static_cast<size_t>(B) * (K + 1) * s.slots_per_row * sizeof(Partial), 256);
     w.b_ticket_off = align_up(w.hint_off + static_cast<size_t>(B) * K * sizeof(int), 256);
     w.g_ticket_off = align_up(w.b_ticket_off + static_cast<size_t>(B) * sizeof(unsigned int), 16);
-    w.total = align_up(w.g_ticket_off + 16, 256);
+    w.half_bytes = align_up(w.g_ticket_off + 16, 256);
+    w.half_off[0] = 256;
+    w.half_off[1] = 256 + w.half_bytes;
+    w.total = 256 + 2 * w.half_bytes;
     return w;
 }
 
@@ -154,10 +161,15 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.rej_d = rej_draft; p.rej_t = rej_target;
     if (diag) p.diag = *diag;
     char *ws = static_cast<char *>(workspace);
-    p.partials = reinterpret_cast<Partial *>(ws + w.partials_off);
-    p.slot_hint = reinterpret_cast<int *>(ws + w.hint_off);
-    p.b_ticket = reinterpret_cast<unsigned int *>(ws + w.b_ticket_off);
-    p.g_ticket = reinterpret_cast<unsigned int *>(ws + w.g_ticket_off);
+    for (int h = 0; h < 2; ++h) {
+        char *half = ws + w.half_off[h];
+        p.partials[h] = reinterpret_cast<Partial *>(half + w.partials_off);
+        p.slot_hint[h] = reinterpret_cast<int *>(half + w.hint_off);
+        p.b_ticket[h] = reinterpret_cast<unsigned int *>(half + w.b_ticket_off);
+        p.g_ticket[h] = reinterpret_cast<unsigned int *>(half + w.g_ticket_off);
+    }
+    p.launch_seq = reinterpret_cast<unsigned long long *>(ws + w.seq_off);
+    p.completed = reinterpret_cast<unsigned int *>(ws + w.seq_off + 8);
     p.n_spans = s.grid;
     p.unit_elems = s.unit_elems;
     p.units_per_row = s.units_per_row;
@@ -467,7 +479,7 @@ csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype, int *grid,
 csd_status_t csd_set_tuning(int chunk_bytes, int ctas_per_sm, int block_threads)
 {
     if (chunk_bytes != 0 && (chunk_bytes < 512 || chunk_bytes % 512 != 0 || chunk_bytes > (1 << 22))) return CSD_ERR_INVALID_ARG;
-    if (ctas_per_sm < 0 || ctas_per_sm > 8) return CSD_ERR_INVALID_ARG;
+    if (ctas_per_sm < 0 || ctas_per_sm > 32) return CSD_ERR_INVALID_ARG;
     if (block_threads != 0 && (block_threads < 32 || block_threads > 1024 || block_threads % 32 != 0)) return CSD_ERR_INVALID_ARG;
     g_chunk_bytes_override = chunk_bytes;
     g_ctas_per_sm_override = ctas_per_sm;

@@ -6,7 +6,7 @@
 //   * The R = B*(K+1) logit rows, each cut into 512-byte units, form one long unit
 //     space that is split EVENLY and contiguously over the G blocks of a persistent
 //     grid (block c owns units [c*T/G, (c+1)*T/G)); a block touches one or a few rows.
-//   * Inside a block the span is cut into fixed chunks (8 KiB by default, never across
+//   * Inside a block the span is cut into fixed chunks (16 KiB by default, never across
 //     a row) that the block's warps pull from a shared-memory counter.  Shared-memory
 //     atomics cost next to nothing, so the hand-out can be this fine, and it evens out
 //     the large warp-to-warp differences in memory latency: a block is done when its
@@ -22,8 +22,12 @@
 //     fold publishes one partial per (block, row) to global memory: one fence and one
 //     ticket per batch row touched, per BLOCK.  Everything before that reads only the
 //     logits, so with programmatic dependent launch the streaming of step n+1 overlaps
-//     the tail of step n: the only wait on the previous launch sits just before the
-//     first global write.
+//     the tail of step n.  The scratch exists twice and launches alternate between the
+//     copies by a sequence number kept in the workspace itself (every block reads it,
+//     the last block to do so advances it, and only then can the next launch begin), so
+//     publication, tickets and the per-row fold of step n+1 also happen while step n is
+//     still finishing; step n+1 waits for step n only before its first OCM look-up and
+//     its first write to an output buffer.
 //   * Whichever block delivers a batch row's last part finalises it (one warp): the
 //     few partials per row are folded by fixed-shape butterflies (maximum first, then
 //     the sums rescaled to the row's reference: bit-reproducible), lanes 0..K-1 take
@@ -59,10 +63,14 @@ struct StepParams {
     int *rej_d;
     int *rej_t;
     csd_diag_t diag;
-    Partial *partials;       // [R * slots_per_row]: one slot per (row, block touching it)
-    int *slot_hint;          // [B * K] slot of each recorded pair (see kHint*)
-    unsigned int *b_ticket;  // [B]
-    unsigned int *g_ticket;  // [1]
+    // Two copies of the scratch ("halves"), used by consecutive launches in turn, so that
+    // a launch can publish and fold while the previous one is still finishing.
+    Partial *partials[2];       // [R * slots_per_row]: one slot per (row, block touching it)
+    int *slot_hint[2];          // [B * K] slot of each recorded pair (see kHint*)
+    unsigned int *b_ticket[2];  // [B]
+    unsigned int *g_ticket[2];  // [1]
+    unsigned long long *launch_seq;  // (sequence number of the launch now starting << 32) | blocks counted in
+    unsigned int *completed;         // launches completed on this workspace
     int n_spans;             // G: blocks that own a span of the unit space
     int unit_elems;          // elements per 512-byte unit
     int units_per_row;       // U = ceil(V / unit_elems)
@@ -310,6 +318,7 @@ constexpr int kMaxSegs = 32;       // row parts a block handles between two bloc
 constexpr int kMaxChunks = 1024;   // chunk results held in shared memory at a time
 
 struct BlockState {
+    unsigned int seq;                   // this launch's sequence number on the workspace
     unsigned int next_chunk;            // hand-out counter
     unsigned int segs_folded;           // row parts folded so far
     unsigned int seg_done[kMaxSegs];    // chunks delivered per row part
@@ -367,7 +376,7 @@ __device__ __forceinline__ Partial butterfly_fold(Partial v, int width)
 // Fold the per-block partials of the K+1 logit rows of batch row b (S1, last level).  The
 // lanes are arranged as (32 / width) rows x width slots, width = the power of two >= the
 // slots per row (at most 32; more slots are pre-folded in lane order).
-__device__ __forceinline__ void fold_rows(const StepParams &p, int b, int lane, RowScratch &rs)
+__device__ __forceinline__ void fold_rows(const StepParams &p, int half, int b, int lane, RowScratch &rs)
 {
     const int K1 = p.K + 1, S = p.slots_per_row;
     int width = 1;
@@ -376,7 +385,7 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, int b, int lane, 
     const int sub = lane / width;          // which row of the pass
     const int k0 = lane - sub * width;     // first slot this lane folds
     const size_t row0 = (size_t)b * K1;
-    const Partial *part = p.partials + row0 * S;
+    const Partial *part = p.partials[half] + row0 * S;
 
     for (int r = lane; r < K1; r += 32) {
         const long long u0 = static_cast<long long>(row0 + r) * p.units_per_row;
@@ -409,11 +418,6 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, int b, int lane, 
                 rs.m[row] = t.m;
                 rs.s[row] = s_m;
                 rs.t[row] = t.idx;
-                if (!(s_m == s_m) || s_m == INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
-                if (p.diag.m) p.diag.m[row0 + row] = t.m;
-                if (p.diag.s) p.diag.s[row0 + row] = s_m;
-                if (p.diag.lse) p.diag.lse[row0 + row] = t.m + logf(s_m);
-                if (p.diag.t) p.diag.t[row0 + row] = t.idx;
             }
         }
     }
@@ -421,7 +425,7 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, int b, int lane, 
 }
 
 template <typename L>
-__device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScratch &rs)
+__device__ void finalize_batch_row(const StepParams &p, int half, int b, int lane, RowScratch &rs)
 {
     using E = typename L::elem;
     const int K = p.K;
@@ -439,9 +443,22 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
             zd = L::load_elem(rowp, d);
         }
     }
-    const int regime = p.do_update ? update_regime(p) : kRegimeFull;
+    fold_rows(p, half, b, lane, rs);
 
-    fold_rows(p, b, lane, rs);
+    // Everything above read only this launch's inputs and its own half of the scratch.
+    // From here on the previous launch must be complete: the memory, its statistics and
+    // the output buffers come into play.
+    pdl_wait();
+    const int regime = p.do_update ? update_regime(p) : kRegimeFull;
+    for (int row = lane; row <= K; row += 32) {
+        const size_t at = (size_t)b * (K + 1) + row;
+        const float s_m = rs.s[row];
+        if (!(s_m == s_m) || s_m == INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
+        if (p.diag.m) p.diag.m[at] = rs.m[row];
+        if (p.diag.s) p.diag.s[at] = s_m;
+        if (p.diag.lse) p.diag.lse[at] = rs.m[row] + logf(s_m);
+        if (p.diag.t) p.diag.t[at] = rs.t[row];
+    }
 
     // S2 (second half), S3, S4 per position; S5 across the warp.
     bool match = false, ok = false;
@@ -487,7 +504,7 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
                 const unsigned int room = 0xffffffffu - static_cast<unsigned int>(p.B * p.K);
                 if (slot >= 0 && cnt > room) hint |= kHintCareful;
             }
-            __stcg(p.slot_hint + pos, hint);
+            __stcg(p.slot_hint[half] + pos, hint);
         }
     }
     const unsigned int m_match = __ballot_sync(kFull, reached && match);
@@ -509,7 +526,7 @@ __device__ void finalize_batch_row(const StepParams &p, int b, int lane, RowScra
 
 // S6, second half, by the warp that finalised the last batch row: every look-up of the
 // step is done, so the counts may change now.
-__device__ void apply_step_update(const StepParams &p, int lane, CanonScratch &canon)
+__device__ void apply_step_update(const StepParams &p, int half, int lane, CanonScratch &canon)
 {
     const int n = p.B * p.K;
     const int regime = update_regime(p);
@@ -523,7 +540,7 @@ __device__ void apply_step_update(const StepParams &p, int lane, CanonScratch &c
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             const int j = j0 + q * 32 + lane;
-            h[q] = j < n ? __ldcg(p.slot_hint + j) : kHintNone;
+            h[q] = j < n ? __ldcg(p.slot_hint[half] + j) : kHintNone;
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
@@ -554,14 +571,18 @@ __device__ void publish_and_finalize(const StepParams &p, BlockState &bs, RowScr
 {
     const int K1 = p.K + 1;
     const int U = p.units_per_row;
-    // the first access to memory that the previous launch on the stream may still be using
-    pdl_wait();
+    const unsigned int seq = bs.seq;
+    const int half = static_cast<int>(seq & 1u);
+    // This half was last used by launch seq-2.  If that launch is known to be complete the
+    // scratch can be written right away; otherwise wait for the previous launch first
+    // (launches complete in order, so that covers seq-2 as well).
+    const unsigned int completed = __ldcg(p.completed);
+    if (static_cast<int>(completed - (seq - 1u)) < 0) pdl_wait();
     int my_b = -1;
     if (lane < nseg) {
         const int row = first_row + lane;
         const int slot = static_cast<int>(blockIdx.x) - owner_of(p, static_cast<long long>(row) * U);
-        if (slot < p.slots_per_row) st_partial_cg(p.partials + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
-        else atomicOr(&p.ocm.stats->flags, CSD_FLAG_PROBE_EXHAUSTED);
+        if (slot < p.slots_per_row) st_partial_cg(p.partials[half] + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
         my_b = row / K1;
     }
     __threadfence();
@@ -574,7 +595,7 @@ __device__ void publish_and_finalize(const StepParams &p, BlockState &bs, RowScr
         if (closes) {
             const long long u0 = static_cast<long long>(my_b) * K1 * U;
             const unsigned int expected = owner_of(p, u0 + static_cast<long long>(K1) * U - 1) - owner_of(p, u0) + 1;
-            completes = atomicAdd(p.b_ticket + my_b, 1u) == expected - 1;
+            completes = atomicAdd(p.b_ticket[half] + my_b, 1u) == expected - 1;
         }
     }
     unsigned int todo = __ballot_sync(kFull, completes);
@@ -585,24 +606,25 @@ __device__ void publish_and_finalize(const StepParams &p, BlockState &bs, RowScr
         todo &= todo - 1;
         const int b = __shfl_sync(kFull, my_b, src);
         __threadfence();
-        finalize_batch_row<L>(p, b, lane, rs);
+        finalize_batch_row<L>(p, half, b, lane, rs);
         bool last = false;
-        if (lane == 0) p.b_ticket[b] = 0u;               // ready for the next launch
+        if (lane == 0) p.b_ticket[half][b] = 0u;          // ready for the launch after next
         __threadfence();
         __syncwarp();
-        if (lane == 0) last = atomicAdd(p.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
+        if (lane == 0) last = atomicAdd(p.g_ticket[half], 1u) == static_cast<unsigned int>(p.B) - 1u;
         last = __shfl_sync(kFull, last, 0);
         if (!last) continue;
 
         // ---- every batch row is final: S6 ----
         __threadfence();
-        if (p.do_update) apply_step_update(p, lane, canon);
+        if (p.do_update) apply_step_update(p, half, lane, canon);
         if (lane == 0) {
             OcmStatsDev *st = p.ocm.stats;
             __threadfence();
             st->n_keys_start = atomicAdd(&st->n_keys, 0ull);
             atomicAdd(&st->steps, 1ull);
-            *p.g_ticket = 0u;
+            *p.g_ticket[half] = 0u;
+            __stcg(p.completed, seq + 1u);
         }
     }
 }
@@ -617,8 +639,22 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
     __shared__ CanonScratch canon;
 
     using E = typename L::elem;
-    pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
+    if (threadIdx.x < 32) {
+        // Launch sequence number, one atomic: the word holds (sequence << 32 | blocks counted
+        // in).  Every block counts itself in and learns the sequence from the same answer;
+        // the block that is last to do so moves the word on to the next launch.  That launch
+        // can begin only after every block of this one has released it, which a block does
+        // after counting itself in -- so all blocks of a launch see the same number.
+        if (lane == 0) {
+            const unsigned long long old = atomicAdd(p.launch_seq, 1ull);
+            if (static_cast<unsigned int>(old) == gridDim.x - 1)
+                atomicAdd(p.launch_seq, (1ull << 32) - static_cast<unsigned long long>(gridDim.x));
+            bs.seq = static_cast<unsigned int>(old >> 32);     // read after the first block barrier
+        }
+        __syncwarp();
+        pdl_launch_dependents();
+    }
     const int K1 = p.K + 1;
     const int U = p.units_per_row;
     const int CH = p.chunk_units;

@@ -57,7 +57,7 @@ def test_shapes_and_workspace(L):
         assert s["block"] == 256 and 1 <= s["grid"] <= min(148 * 4, units, 64 * rows)
         assert (s["chunk_elems"] * eb) % 512 == 0 and 1 <= s["parts_per_row"] <= 66
         ws = binding.csd_workspace_bytes(B, K, V, dt)
-        assert ws >= rows * s["parts_per_row"] * 16 + 4 * B * K + 4 * B + 4
+        assert ws >= 2 * (rows * s["parts_per_row"] * 16 + 4 * B * K + 4 * B + 4) + 12
         assert binding.csd_host_staging_bytes(B, K, V, dt) >= rows * V * eb + ws
     assert binding.csd_workspace_bytes(0, 4, 100, 0) == 0
     assert binding.csd_workspace_bytes(1, 33, 100, 0) == 0
@@ -111,7 +111,7 @@ def test_argument_checks_refuse_before_launch(L):
     assert L.csd_ocm_create(ctypes.byref(out), 32, 6, 0) == 1
     assert L.csd_ocm_create(None, 1024, 6, 0) == 1
     assert L.csd_ocm_create(ctypes.byref(out), 1 << 31, 6, 0) == 1
-    assert L.csd_set_tuning(1000, 0, 0) == 1 and L.csd_set_tuning(0, 9, 0) == 1 and L.csd_set_tuning(0, 0, 48) == 1
+    assert L.csd_set_tuning(1000, 0, 0) == 1 and L.csd_set_tuning(0, 33, 0) == 1 and L.csd_set_tuning(0, 0, 48) == 1
     assert L.csd_set_tuning(0, 0, 0) == 0
 
 
