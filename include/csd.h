@@ -188,6 +188,38 @@ csd_status_t csd_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
                       const csd_diag_t *diag,
                       void *workspace, size_t workspace_bytes, void *stream);
 
+/* csd_verify without a workspace argument and without any allocation.  (The paper has
+ * no counterpart: this is a deployment convenience of the library.)
+ *
+ * Who needs it: code that runs the verification from a place where device memory can
+ * no longer be obtained -- an inference server whose framework reserved the whole GPU
+ * for its own pool at start-up, a plug-in that is handed tensors but no allocator, a
+ * latency-critical loop where an allocation (which may synchronise the device or
+ * fail) is not acceptable.  Such a caller cannot provide the workspace csd_verify
+ * asks for.  Here the kernel's scratch is a fixed array of CSD_STATIC_SCRATCH_BYTES
+ * that is part of the library image: every GPU that loads the library holds it until
+ * the process exits.  The call performs no cudaMalloc / cudaFree and calls no
+ * allocating routine.  (The csd_ocm_t it reads was allocated earlier by
+ * csd_ocm_create, which such a caller runs during its set-up phase.)
+ *
+ * Arguments and results are those of csd_verify (inputs and outputs remain the
+ * caller's device buffers); the current device must be the memory's device.
+ * Shapes whose csd_workspace_bytes exceeds CSD_STATIC_SCRATCH_BYTES are refused with
+ * CSD_ERR_WORKSPACE before anything is launched (all five reference workloads need
+ * less than 100 KiB).  The first call on each device looks up the array's device
+ * address; make that first call outside any stream capture.  All calls share the one
+ * array, which keeps the previous call's contents, so every call first clears the
+ * part it uses (asynchronously, on `stream`); two calls that overlap on the GPU (two
+ * streams, or this call next to a csd_step launched with csd_set_overlap) would race
+ * on it: issue them on one stream, one after the other. */
+#define CSD_STATIC_SCRATCH_BYTES (1u << 20)
+csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int K, int V,
+                               int64_t stride_b, int64_t stride_k,
+                               const int32_t *draft, const csd_ocm_t *ocm, float tau,
+                               int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                               int32_t *rej_draft, int32_t *rej_target,
+                               const csd_diag_t *diag, void *stream);
+
 /* csd_step for callers whose tensors live in HOST memory (pinned memory gives
  * the full copy rate).  Copies logits and draft to `staging`, runs the step, and
  * copies accept_len, next_token and rescued_mask back; returns after the stream

@@ -24,7 +24,7 @@ FLAG_NAN_LOGIT, FLAG_BAD_DRAFT, FLAG_PROBE_EXHAUSTED, FLAG_COUNT_SATURATED = 1, 
 EXPORTS = [
     "csd_ocm_create", "csd_ocm_reset", "csd_ocm_destroy", "csd_ocm_set_lambda",
     "csd_workspace_bytes", "csd_workspace_init", "csd_verify", "csd_ocm_update", "csd_step",
-    "csd_host_staging_bytes", "csd_step_host", "csd_ocm_export", "csd_ocm_import", "csd_ocm_stats",
+    "csd_host_staging_bytes", "csd_step_host", "csd_verify_static", "csd_ocm_export", "csd_ocm_import", "csd_ocm_stats",
     "csd_scg_threshold", "csd_launch_shape", "csd_set_tuning", "csd_set_overlap", "csd_status_string",
 ]
 
@@ -69,6 +69,7 @@ def lib():
         "csd_workspace_init": (c_int, [c_void_p, c_size_t, c_void_p]),
         "csd_verify": (c_int, step_args),
         "csd_step": (c_int, step_args),
+        "csd_verify_static": (c_int, step_args[:-3] + [c_void_p]),
         "csd_ocm_update": (c_int, [c_void_p, c_void_p, c_void_p, c_int64, c_void_p]),
         "csd_host_staging_bytes": (c_size_t, [c_int, c_int, c_int, c_int]),
         "csd_step_host": (c_int, [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_float,
@@ -280,3 +281,20 @@ class HostStep:
                                  self.staging.data_ptr(), self.bytes, _stream_ptr(stream))
         _check(rc, "csd_step_host")
         return self.accept_len, self.next_token, self.rescued_mask
+
+
+STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def csd_verify_static(logits, draft, ocm: Ocm, tau: float, buf: StepBuffers, stream=None):
+    """csd_verify with the scratch in the library's own fixed device array: for callers that
+    cannot allocate device memory (buf.workspace is not used).  Calls must not overlap on the GPU."""
+    assert logits.is_cuda and draft.is_cuda and draft.dtype == torch.int32 and draft.is_contiguous()
+    B, K1, V = logits.shape
+    assert (B, K1 - 1, V) == (buf.B, buf.K, buf.V) and logits.stride(2) == 1 and _dtype_code(logits) == buf.dtype_code
+    rc = lib().csd_verify_static(
+        logits.data_ptr(), buf.dtype_code, B, K1 - 1, V, logits.stride(0), logits.stride(1), draft.data_ptr(),
+        ocm.handle, c_float(tau), _ptr(buf.accept_len), _ptr(buf.next_token), _ptr(buf.rescued_mask),
+        _ptr(buf.rej_draft), _ptr(buf.rej_target),
+        byref(buf._diag_struct) if buf._diag_struct is not None else None, _stream_ptr(stream))
+    _check(rc, "csd_verify_static")

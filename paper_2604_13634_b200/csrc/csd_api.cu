@@ -364,6 +364,57 @@ StagingLayout staging_layout(int B, int K, int V, csd_dtype_t dtype)
 }
 }  // namespace
 
+// ---- csd_verify_static: the verification step for callers that must not allocate ----------
+//
+// The scratch of the step kernel lives in this file-scope device array instead of a
+// caller-provided workspace.  Every GPU that loads the library holds these bytes until the
+// process exits.  In host code the array's name is only a host-side stand-in for the symbol;
+// its device address is looked up once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[CSD_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_ptr[kMaxDevices];   // device address of g_static_scratch, per device
+bool g_static_scratch_known[kMaxDevices];
+}  // namespace
+
+csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b,
+                               int64_t stride_k, const int32_t *draft, const csd_ocm_t *ocm, float tau,
+                               int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask, int32_t *rej_draft,
+                               int32_t *rej_target, const csd_diag_t *diag, void *stream)
+{
+    if (!ocm) return CSD_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || V <= 0 || (dtype != CSD_F32 && dtype != CSD_BF16)) return CSD_ERR_INVALID_ARG;
+    if (K > CSD_MAX_K || !shape_ok(B, K, V, dtype)) return CSD_ERR_UNSUPPORTED;
+    const size_t need = csd_workspace_bytes(B, K, V, dtype);
+    if (need == 0 || need > CSD_STATIC_SCRATCH_BYTES) return CSD_ERR_WORKSPACE;   // shape needs more than the fixed scratch
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    if (dev != ocm->device) return CSD_ERR_INVALID_ARG;   // the memory's device must be the current one
+    if (!g_static_scratch_known[dev]) {
+        // once per device, with that device current (first call: not under stream capture)
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+            (void)cudaGetLastError();
+            return CSD_ERR_CUDA;
+        }
+        g_static_scratch_ptr[dev] = ptr;
+        g_static_scratch_known[dev] = true;
+    }
+    void *scratch = g_static_scratch_ptr[dev];
+    // The array keeps whatever the last call (possibly of another shape) left in it, and the
+    // kernel needs its counters and sequence words to start at zero: clear the part in use.
+    if (cudaMemsetAsync(scratch, 0, need, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    return run_step(logits, dtype, B, K, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
+                    rej_draft, rej_target, diag, scratch, need, stream, false);
+}
+
 size_t csd_host_staging_bytes(int B, int K, int V, csd_dtype_t dtype)
 {
     if (!shape_ok(B, K, V, dtype)) return 0;
