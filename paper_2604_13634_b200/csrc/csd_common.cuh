@@ -37,6 +37,51 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
+// Packed pairs of floats in one 64-bit register: sm_100 executes fma/add on both halves with
+// one instruction (fma.rn.f32x2 / add.rn.f32x2), which halves the issue slots of the
+// per-element multiply-add and accumulate.  Each half is rounded exactly like the scalar op.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+
+__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c)
+{
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b)
+{
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b)
+{
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// acc += (2^(x0*log2e - c), 2^(x1*log2e - c)) for a pair of logits
+__device__ __forceinline__ void accum_pair(float x0, float x1, unsigned long long l2e2, unsigned long long negc2,
+                                           unsigned long long &acc)
+{
+    float t0, t1;
+    unpack2(fma2(pack2(x0, x1), l2e2, negc2), t0, t1);
+    acc = add2(acc, pack2(ex2_approx(t0), ex2_approx(t1)));
+}
+
 // 2^k for an integer-valued k <= 0 (any value <= -127, -inf or NaN gives 0): exact.
 __device__ __forceinline__ float pow2_nonpos(float k)
 {

@@ -104,12 +104,11 @@ struct LaneF32Vec {
     {
         return fmaxf(fmaxf(__uint_as_float(a.x), __uint_as_float(a.y)), fmaxf(__uint_as_float(a.z), __uint_as_float(a.w)));
     }
-    static __device__ __forceinline__ void accum(unit a, float negc, float &s0, float &s1)
+    static __device__ __forceinline__ void accum(unit a, unsigned long long l2e2, unsigned long long negc2,
+                                                 unsigned long long &acc)
     {
-        s0 += ex2_approx(fmaf(__uint_as_float(a.x), kLog2e, negc));
-        s1 += ex2_approx(fmaf(__uint_as_float(a.y), kLog2e, negc));
-        s0 += ex2_approx(fmaf(__uint_as_float(a.z), kLog2e, negc));
-        s1 += ex2_approx(fmaf(__uint_as_float(a.w), kLog2e, negc));
+        accum_pair(__uint_as_float(a.x), __uint_as_float(a.y), l2e2, negc2, acc);
+        accum_pair(__uint_as_float(a.z), __uint_as_float(a.w), l2e2, negc2, acc);
     }
     static __device__ __forceinline__ int first_eq(unit a, float v)
     {
@@ -150,17 +149,13 @@ struct LaneBf16Vec {
         const unsigned int w = max2(max2(a.x, a.y), max2(a.z, a.w));
         return fmaxf(lo(w), hi(w));
     }
-    static __device__ __forceinline__ void accum2(unsigned int w, float negc, float &s0, float &s1)
+    static __device__ __forceinline__ void accum(unit a, unsigned long long l2e2, unsigned long long negc2,
+                                                 unsigned long long &acc)
     {
-        s0 += ex2_approx(fmaf(lo(w), kLog2e, negc));
-        s1 += ex2_approx(fmaf(hi(w), kLog2e, negc));
-    }
-    static __device__ __forceinline__ void accum(unit a, float negc, float &s0, float &s1)
-    {
-        accum2(a.x, negc, s0, s1);
-        accum2(a.y, negc, s0, s1);
-        accum2(a.z, negc, s0, s1);
-        accum2(a.w, negc, s0, s1);
+        accum_pair(lo(a.x), hi(a.x), l2e2, negc2, acc);
+        accum_pair(lo(a.y), hi(a.y), l2e2, negc2, acc);
+        accum_pair(lo(a.z), hi(a.z), l2e2, negc2, acc);
+        accum_pair(lo(a.w), hi(a.w), l2e2, negc2, acc);
     }
     static __device__ __forceinline__ int first_eq(unit a, float v)
     {
@@ -184,10 +179,11 @@ struct LaneF32Scalar {
     static __device__ __forceinline__ unit neg_inf() { return -INFINITY; }
     static __device__ __forceinline__ unit vmax(unit a, unit b) { return fmaxf(a, b); }
     static __device__ __forceinline__ float hmax(unit a) { return a; }
-    static __device__ __forceinline__ void accum(unit a, float negc, float &s0, float &s1)
+    static __device__ __forceinline__ void accum(unit a, unsigned long long l2e2, unsigned long long negc2,
+                                                 unsigned long long &acc)
     {
-        s0 += ex2_approx(fmaf(a, kLog2e, negc));
-        (void)s1;
+        // one element: the second half of the pair adds 2^(-inf) = 0
+        accum_pair(a, -INFINITY, l2e2, negc2, acc);
     }
     static __device__ __forceinline__ int first_eq(unit a, float v) { return a == v ? 0 : -1; }
 };
@@ -205,10 +201,11 @@ struct LaneBf16Scalar {
     static __device__ __forceinline__ unit neg_inf() { return -INFINITY; }
     static __device__ __forceinline__ unit vmax(unit a, unit b) { return fmaxf(a, b); }
     static __device__ __forceinline__ float hmax(unit a) { return a; }
-    static __device__ __forceinline__ void accum(unit a, float negc, float &s0, float &s1)
+    static __device__ __forceinline__ void accum(unit a, unsigned long long l2e2, unsigned long long negc2,
+                                                 unsigned long long &acc)
     {
-        s0 += ex2_approx(fmaf(a, kLog2e, negc));
-        (void)s1;
+        // one element: the second half of the pair adds 2^(-inf) = 0
+        accum_pair(a, -INFINITY, l2e2, negc2, acc);
     }
     static __device__ __forceinline__ int first_eq(unit a, float v) { return a == v ? 0 : -1; }
 };
@@ -227,7 +224,9 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
     float m_thr = -INFINITY;   // running maximum of this lane
     float c_thr = kNoRef;      // integer reference exponent of the accumulators
     int it_thr = -1;           // iteration of the last strict improvement
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    // four sums as two packed pairs: acc0 = (s0, s1), acc1 = (s2, s3)
+    unsigned long long acc0 = pack2(0.f, 0.f), acc1 = acc0;
+    const unsigned long long l2e2 = pack2(kLog2e, kLog2e);
     U v[kUnroll];
 
     auto consume = [&](const U (&v)[kUnroll], int it) {
@@ -240,21 +239,26 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
             const float cn = rintf(bmax * kLog2e);
             if (cn > c_thr) {
                 const float f = pow2_nonpos(c_thr - cn);
-                s0 *= f; s1 *= f; s2 *= f; s3 *= f;
+                const unsigned long long f2 = pack2(f, f);
+                acc0 = mul2(acc0, f2);
+                acc1 = mul2(acc1, f2);
                 c_thr = cn;
             }
         }
-        const float negc = -c_thr;
+        const unsigned long long negc2 = pack2(-c_thr, -c_thr);
 #pragma unroll
         for (int k = 0; k < kUnroll; k += 2) {
-            L::accum(v[k], negc, s0, s1);
-            L::accum(v[k + 1], negc, s2, s3);
+            L::accum(v[k], l2e2, negc2, acc0);
+            L::accum(v[k + 1], l2e2, negc2, acc1);
         }
     };
 
+    // full iterations: one pointer, constant offsets, no bounds checks
+    const typename L::elem *lp = base + (size_t)lane * L::kPer;
     for (int it = 0; it < nfull; ++it) {
 #pragma unroll
-        for (int k = 0; k < kUnroll; ++k) v[k] = L::load(base, (it * kUnroll + k) * 32 + lane);
+        for (int k = 0; k < kUnroll; ++k) v[k] = L::load(lp, k * 32);
+        lp += (size_t)kPerIter * L::kPer;
         consume(v, it);
     }
     if (nfull * kPerIter < nunits) {
@@ -265,6 +269,9 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
         }
         consume(v, nfull);
     }
+    float s0, s1, s2, s3;
+    unpack2(acc0, s0, s1);
+    unpack2(acc1, s2, s3);
 
     // warp maximum, then everything is rescaled to the warp's reference exponent
     float wmax = m_thr;
