@@ -1,0 +1,87 @@
+#!/usr/bin/env python
+"""Long lock-step run of one workload: the CUDA path against the CPU oracle, step by step.
+
+Test infrastructure (it imports the oracle); not collected by pytest.  For every step the
+accepted lengths, next tokens, rescue masks and rejection lists must be identical; the
+diagnostics (t*, m, counts exact; s, lse, score, p_d, p_t within 1e-5) are compared on the
+first 100 steps and every 100th after; the memory's (pair, count) set, n_keys and n_dropped
+are compared at every checkpoint and at the end.  Prints one JSON line per (workload, tau).
+
+    python tests/lockstep_run.py --workload ocm_contention --steps 20000 --checkpoint 10000
+"""
+
+import argparse
+import json
+import os
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+import test_gpu_parity as T                                     # noqa: E402
+from oracle import csd_oracle as ORACLE                          # noqa: E402
+from paper_2604_13634_b200 import Ocm, StepBuffers, csd_step     # noqa: E402
+from paper_2604_13634_b200.synth import WORKLOADS, Synth         # noqa: E402
+
+
+def run(wl, tau, steps, checkpoint, prewarm_steps, seed=0):
+    syn = Synth(wl, seed, "cuda")
+    ocm = Ocm(wl.ocm_slots, wl.lam)
+    mem = ORACLE.OCM(wl.ocm_slots, wl.lam)
+    kind, n = wl.prewarm
+    if kind == "pairs":
+        pd, pt = syn.prewarm_pairs(n)
+        ocm.update(pd, pt)
+        mem.update(zip(pd.cpu().tolist(), pt.cpu().tolist()))
+    buf = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True)
+    first = 0
+    if kind == "steps":
+        # pre-warming steps are ordinary steps of the same stream, checked like the others
+        first = -min(prewarm_steps, n)
+    t0 = time.time()
+    near = acc = resc = checked_diag = 0
+    for s in range(first, steps):
+        z, d = syn.step(s + 10 ** 6 if s < 0 else s)
+        csd_step(z, d, ocm, tau, buf)
+        ref = T.oracle_step(z, d, mem, tau)
+        sample = (s < 100) or (s % 100 == 0)
+        near += T.compare(buf, ref, check_diag=sample)
+        checked_diag += int(sample)
+        if s >= 0:
+            acc += int(ref["accept_len"].sum())
+            resc += int(ref["rescued_mask"].sum())
+        if checkpoint and s >= 0 and (s + 1) % checkpoint == 0:
+            T.compare_memory(ocm, mem)
+    st = T.compare_memory(ocm, mem)
+    assert st["flags"] == 0, st
+    out = dict(workload=wl.name, tau=tau, steps=steps, prewarm_steps=-first, B=wl.B, K=wl.K, V=wl.V, dtype=wl.dtype,
+               accepted=acc, rescued=resc, acceptance_rate=acc / (steps * wl.B * wl.K), near_ties=near,
+               diag_steps_checked=checked_diag, n_keys=st["n_keys"], n_dropped=st["n_dropped"],
+               checkpoints=(steps // checkpoint if checkpoint else 0), seconds=round(time.time() - t0, 1),
+               verdict="identical")
+    ocm.close()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", required=True)
+    ap.add_argument("--steps", type=int, default=0, help="0 = the workload's own step count")
+    ap.add_argument("--checkpoint", type=int, default=0)
+    ap.add_argument("--prewarm-steps", type=int, default=10 ** 9, help="cap on step-type pre-warming")
+    ap.add_argument("--taus", default="")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+    taus = [float(x) for x in args.taus.split(",")] if args.taus else list(wl.taus)
+    for tau in taus:
+        res = run(wl, tau, args.steps or wl.steps, args.checkpoint or wl.checkpoint_every, args.prewarm_steps)
+        print(json.dumps(res), flush=True)
+
+
+if __name__ == "__main__":
+    main()
