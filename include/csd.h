@@ -266,7 +266,7 @@ csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype,
                               int *grid, int *block, int *chunk_elems, int *parts_per_row);
 
 /* Expert knob, process-wide: override the automatic work split.  chunk_bytes: bytes of
- * one logit row reduced by a warp at a time (multiple of 512; 0 = automatic, 16384);
+ * one logit row reduced by a warp at a time (multiple of 512; 0 = automatic, 4 to 32 KiB);
  * ctas_per_sm: blocks of the persistent grid per SM (0 = automatic, 4); block_threads:
  * threads per block (multiple of 32, at most 1024; 0 = automatic, 256).  Changes
  * csd_workspace_bytes: size workspaces after calling it.  Results stay

@@ -86,9 +86,15 @@ Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
     long long slots = ((s.units_per_row - 1) * blocks + s.total_units - 1) / s.total_units + 1;
     if (slots > s.units_per_row) slots = s.units_per_row;
     s.slots_per_row = static_cast<int>(slots < 1 ? 1 : slots);
-    // chunks: 16 KiB unless overridden, grown so that a block's span fits its chunk table
-    long long chunk_units = (g_chunk_bytes_override > 0 ? g_chunk_bytes_override : 16384) / kUnitBytes;
+    // chunks: about one per warp of the block for small spans (least per-chunk overhead), 4 to
+    // 32 KiB in whole warp iterations (4 KiB), so that larger spans are still handed out in many
+    // pieces; grown where needed so that a block's span fits its chunk table
     const long long span_max = (s.total_units + blocks - 1) / blocks;
+    const int warps = s.block / 32;
+    long long chunk_units = ((span_max + warps - 1) / warps + 7) / 8 * 8;
+    if (chunk_units < 8) chunk_units = 8;
+    if (chunk_units > 64) chunk_units = 64;
+    if (g_chunk_bytes_override > 0) chunk_units = g_chunk_bytes_override / kUnitBytes;
     const long long need = (span_max + (kMaxChunks - kMaxSegs - 2) - 1) / (kMaxChunks - kMaxSegs - 2);
     if (chunk_units < need) chunk_units = (need + 7) / 8 * 8;
     s.chunk_units = static_cast<int>(chunk_units);
@@ -176,6 +182,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.slots_per_row = s.slots_per_row;
     p.chunk_units = s.chunk_units;
     p.total_units = s.total_units;
+    p.narrow = (s.total_units + 1) * (static_cast<long long>(s.grid) + 1) < (1ll << 32) ? 1 : 0;
 
     const int eb = elt_bytes(dtype);
     const int per_vec = 16 / eb;

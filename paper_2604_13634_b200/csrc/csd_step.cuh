@@ -6,7 +6,7 @@
 //   * The R = B*(K+1) logit rows, each cut into 512-byte units, form one long unit
 //     space that is split EVENLY and contiguously over the G blocks of a persistent
 //     grid (block c owns units [c*T/G, (c+1)*T/G)); a block touches one or a few rows.
-//   * Inside a block the span is cut into fixed chunks (16 KiB by default, never across
+//   * Inside a block the span is cut into fixed chunks (4 to 32 KiB, never across
 //     a row) that the block's warps pull from a shared-memory counter.  Shared-memory
 //     atomics cost next to nothing, so the hand-out can be this fine, and it evens out
 //     the large warp-to-warp differences in memory latency: a block is done when its
@@ -77,6 +77,7 @@ struct StepParams {
     int slots_per_row;       // S >= most blocks that can touch one row
     int chunk_units;         // units per chunk
     long long total_units;   // T = R * U
+    int narrow;              // 1 if the span arithmetic fits 32 bits
 };
 
 constexpr int kHintNone = -1;          // nothing to record at this position
@@ -312,12 +313,17 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 
 __device__ __forceinline__ long long span_begin(const StepParams &p, int c)
 {
+    if (p.narrow)   // (T + 1) * (G + 1) < 2^32: 32-bit division is several times cheaper
+        return static_cast<unsigned int>(c) * static_cast<unsigned int>(p.total_units) / static_cast<unsigned int>(p.n_spans);
     return static_cast<long long>(c) * p.total_units / p.n_spans;
 }
 
 // The block whose span holds global unit g: the largest c with span_begin(c) <= g.
 __device__ __forceinline__ int owner_of(const StepParams &p, long long g)
 {
+    if (p.narrow)
+        return static_cast<int>(((static_cast<unsigned int>(g) + 1u) * static_cast<unsigned int>(p.n_spans) - 1u) /
+                                static_cast<unsigned int>(p.total_units));
     return static_cast<int>(((g + 1) * p.n_spans - 1) / p.total_units);
 }
 

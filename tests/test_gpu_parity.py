@@ -428,13 +428,21 @@ def test_overlapped_launches_match():
 
 
 def test_long_rows():
-    """Rows of 4 MiB: each is shared by several blocks, and a block's span needs larger chunks."""
-    B, K, V = 48, 1, 1 << 20
-    z, d = _random_inputs(B, K, V, torch.float32, seed=11)
-    ocm = Ocm(256, 0)
-    mem = ORACLE.OCM(256, 0)
-    buf = StepBuffers(B, K, V, torch.float32, diag=True)
-    csd_step(z, d, ocm, 0.01, buf)
-    compare(buf, oracle_step(z, d, mem, 0.01))
-    compare_memory(ocm, mem)
-    ocm.close()
+    """Rows of 4 MiB: each is shared by several blocks, and a block's span needs larger chunks.
+    The second case has so many units and blocks that the span arithmetic leaves 32 bits."""
+    for (B, tuning) in ((48, (0, 0, 0)), (64, (0, 32, 128))):
+        try:
+            csd_set_tuning(*tuning)
+            K, V = 1, 1 << 20
+            z, d = _random_inputs(B, K, V, torch.float32, seed=11)
+            ocm = Ocm(256, 0)
+            mem = ORACLE.OCM(256, 0)
+            buf = StepBuffers(B, K, V, torch.float32, diag=True)
+            csd_step(z, d, ocm, 0.01, buf)
+            compare(buf, oracle_step(z, d, mem, 0.01))
+            compare_memory(ocm, mem)
+            ocm.close()
+            del z, d, buf
+            torch.cuda.empty_cache()
+        finally:
+            csd_set_tuning(0, 0, 0)
