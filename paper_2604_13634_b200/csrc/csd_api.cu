@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "../../include/csd.h"
@@ -28,6 +29,53 @@ int g_chunk_bytes_override = 0;
 int g_ctas_per_sm_override = 0;
 int g_block_threads_override = 0;
 int g_overlap_steps = 0;
+
+// ---- which launch preceded which ----------------------------------------------------------
+// A step launched with overlap may poll the completion count that the previous step leaves in
+// the workspace instead of waiting for that whole grid to retire -- but only if that previous
+// step launch on the stream really was issued with the same workspace, memory, outputs and
+// shape, and nothing of this library touched them since.  The host keeps the last step launch
+// per stream for that; any other call that launches work or changes the layout starts a new
+// generation, which voids every record.
+struct ChainRecord {
+    void *stream;
+    const void *ws, *ocm, *out;
+    int B, K, V, dtype;
+    unsigned long long generation;
+};
+constexpr int kChainRecords = 16;
+std::mutex g_chain_mutex;
+ChainRecord g_chain[kChainRecords];
+int g_chain_used = 0, g_chain_next = 0;
+unsigned long long g_chain_generation = 1;
+
+void chain_break()
+{
+    std::lock_guard<std::mutex> lock(g_chain_mutex);
+    ++g_chain_generation;
+}
+
+// Records this launch as the stream's latest; true if the stream's previous record matches it.
+bool chain_follows(void *stream, const void *ws, const void *ocm, const void *out, int B, int K, int V, int dtype)
+{
+    std::lock_guard<std::mutex> lock(g_chain_mutex);
+    const ChainRecord now = {stream, ws, ocm, out, B, K, V, dtype, g_chain_generation};
+    for (int i = 0; i < g_chain_used; ++i) {
+        ChainRecord &r = g_chain[i];
+        if (r.stream != stream) continue;
+        const bool same = r.ws == ws && r.ocm == ocm && r.out == out && r.B == B && r.K == K && r.V == V &&
+                          r.dtype == dtype && r.generation == g_chain_generation;
+        r = now;
+        return same;
+    }
+    if (g_chain_used < kChainRecords) {
+        g_chain[g_chain_used++] = now;
+    } else {
+        g_chain[g_chain_next] = now;
+        g_chain_next = (g_chain_next + 1) % kChainRecords;
+    }
+    return false;
+}
 
 int sm_count()
 {
@@ -139,7 +187,7 @@ OcmView view_of(const csd_ocm *o)
 csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b, int64_t stride_k,
                       const int32_t *draft, const csd_ocm *ocm, float tau, int32_t *accept_len, int32_t *next_token,
                       uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
-                      void *workspace, size_t workspace_bytes, void *stream, bool do_update)
+                      void *workspace, size_t workspace_bytes, void *stream, bool do_update, bool may_chain = true)
 {
     if (!logits || !draft || !ocm || !accept_len || !next_token || !rescued_mask || !rej_draft || !rej_target || !workspace)
         return CSD_ERR_INVALID_ARG;
@@ -183,6 +231,8 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.chunk_units = s.chunk_units;
     p.total_units = s.total_units;
     p.narrow = (s.total_units + 1) * (static_cast<long long>(s.grid) + 1) < (1ll << 32) ? 1 : 0;
+    const bool follows = chain_follows(stream, workspace, ocm, accept_len, B, K, V, static_cast<int>(dtype));
+    p.chain_by_flag = (may_chain && follows) ? 1 : 0;
 
     const int eb = elt_bytes(dtype);
     const int per_vec = 16 / eb;
@@ -212,6 +262,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     }
     if (err != cudaSuccess) {
         (void)cudaGetLastError();
+        chain_break();
         return CSD_ERR_CUDA;
     }
     return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
@@ -221,6 +272,7 @@ csd_status_t run_update(csd_ocm *ocm, const int32_t *d, const int32_t *t, const 
 {
     if (!ocm || n < 0 || (n > 0 && (!d || !t))) return CSD_ERR_INVALID_ARG;
     if (n == 0) return CSD_OK;
+    chain_break();
     long long blocks = (n + 1023) / 1024;
     const long long cap = static_cast<long long>(sm_count()) * 2;
     if (blocks > cap) blocks = cap;
@@ -271,6 +323,7 @@ csd_status_t csd_ocm_create(csd_ocm_t **out, uint64_t n_slots, uint32_t lambda, 
 csd_status_t csd_ocm_reset(csd_ocm_t *ocm, void *stream)
 {
     if (!ocm) return CSD_ERR_INVALID_ARG;
+    chain_break();
     unsigned long long blocks = (ocm->n_slots + 255) / 256;
     const unsigned long long cap = static_cast<unsigned long long>(sm_count()) * 8;
     if (blocks > cap) blocks = cap;
@@ -282,6 +335,7 @@ csd_status_t csd_ocm_reset(csd_ocm_t *ocm, void *stream)
 csd_status_t csd_ocm_destroy(csd_ocm_t *ocm)
 {
     if (!ocm) return CSD_ERR_INVALID_ARG;
+    chain_break();
     cudaError_t a = cudaFree(ocm->slots);
     cudaError_t b = cudaFree(ocm->stats);
     delete ocm;
@@ -304,6 +358,7 @@ size_t csd_workspace_bytes(int B, int K, int V, csd_dtype_t dtype)
 csd_status_t csd_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!workspace || workspace_bytes == 0) return CSD_ERR_INVALID_ARG;
+    chain_break();
     if (cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return CSD_ERR_CUDA;
@@ -419,7 +474,7 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
         return CSD_ERR_CUDA;
     }
     return run_step(logits, dtype, B, K, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
-                    rej_draft, rej_target, diag, scratch, need, stream, false);
+                    rej_draft, rej_target, diag, scratch, need, stream, false, false);
 }
 
 size_t csd_host_staging_bytes(int B, int K, int V, csd_dtype_t dtype)
@@ -440,6 +495,7 @@ csd_status_t csd_step_host(const void *logits_host, csd_dtype_t dtype, int B, in
     if (staging_bytes < s.total || (reinterpret_cast<uintptr_t>(staging) & 255u)) return CSD_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char *dev = static_cast<char *>(staging);
+    chain_break();   // the workspace inside the staging area is cleared below
     const size_t lbytes = static_cast<size_t>(B) * (K + 1) * V * elt_bytes(dtype);
     bool ok = true;
     ok = ok && cudaMemcpyAsync(dev + s.logits, logits_host, lbytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -539,6 +595,7 @@ csd_status_t csd_set_tuning(int chunk_bytes, int ctas_per_sm, int block_threads)
     if (chunk_bytes != 0 && (chunk_bytes < 512 || chunk_bytes % 512 != 0 || chunk_bytes > (1 << 22))) return CSD_ERR_INVALID_ARG;
     if (ctas_per_sm < 0 || ctas_per_sm > 32) return CSD_ERR_INVALID_ARG;
     if (block_threads != 0 && (block_threads < 32 || block_threads > 1024 || block_threads % 32 != 0)) return CSD_ERR_INVALID_ARG;
+    chain_break();
     g_chunk_bytes_override = chunk_bytes;
     g_ctas_per_sm_override = ctas_per_sm;
     g_block_threads_override = block_threads;
@@ -547,6 +604,7 @@ csd_status_t csd_set_tuning(int chunk_bytes, int ctas_per_sm, int block_threads)
 
 csd_status_t csd_set_overlap(int enable)
 {
+    chain_break();
     g_overlap_steps = enable ? 1 : 0;
     return CSD_OK;
 }

@@ -72,9 +72,12 @@ __device__ __forceinline__ void load_slot(const OcmSlot *s, unsigned long long &
     count = v.z;
 }
 
-// Count stored for `key`, 0 if absent.  *slot_out = slot index or -1.
-__device__ __forceinline__ unsigned int ocm_lookup(const OcmView &tb, unsigned long long key, long long *slot_out = nullptr)
+// Count stored for `key`, 0 if absent.  *slot_out = slot index or -1; *empty_out = the empty
+// slot that ended the probe of an absent key (where an insertion would begin), else -1.
+__device__ __forceinline__ unsigned int ocm_lookup(const OcmView &tb, unsigned long long key, long long *slot_out = nullptr,
+                                                   long long *empty_out = nullptr)
 {
+    if (empty_out) *empty_out = -1;
     unsigned long long slot = mix64(key) & tb.mask;
     for (unsigned long long probe = 0; probe <= tb.mask; ++probe) {
         unsigned long long k;
@@ -86,6 +89,7 @@ __device__ __forceinline__ unsigned int ocm_lookup(const OcmView &tb, unsigned l
         }
         if (k == kEmptyKey) {
             if (slot_out) *slot_out = -1;
+            if (empty_out) *empty_out = static_cast<long long>(slot);
             return 0;
         }
         slot = (slot + 1) & tb.mask;
@@ -133,13 +137,16 @@ __device__ __forceinline__ void ocm_insert_or_add(const OcmView &tb, unsigned lo
 // Slot of `key`, claiming an empty slot (count 0) if the key is absent.  A slot with
 // count 0 reads as "absent" to every look-up, so a reservation is invisible until the
 // count is raised.  The caller has established that there is room.  -1 only if the
-// probe wrapped around (flagged).
-__device__ __forceinline__ long long ocm_reserve(const OcmView &tb, unsigned long long key)
+// probe wrapped around (flagged).  `from` >= 0 is the empty slot at which a look-up of this
+// key just ended: the probe resumes there (every slot before it holds another key, and
+// keys never move or vanish) and tries to claim it without reading it again.
+__device__ __forceinline__ long long ocm_reserve(const OcmView &tb, unsigned long long key, long long from = -1)
 {
-    unsigned long long slot = mix64(key) & tb.mask;
+    unsigned long long slot = from >= 0 ? static_cast<unsigned long long>(from) : (mix64(key) & tb.mask);
     for (unsigned long long probe = 0; probe <= tb.mask; ++probe) {
         unsigned long long *kp = &tb.slots[slot].key;
-        unsigned long long k = *reinterpret_cast<volatile unsigned long long *>(kp);
+        unsigned long long k = ~0ull;   // kEmptyKey: what the look-up saw at `from`
+        if (!(from >= 0 && probe == 0)) k = *reinterpret_cast<volatile unsigned long long *>(kp);
         if (k == kEmptyKey) {
             k = atomicCAS(kp, kEmptyKey, key);
             if (k == kEmptyKey) {

@@ -78,11 +78,52 @@ struct StepParams {
     int chunk_units;         // units per chunk
     long long total_units;   // T = R * U
     int narrow;              // 1 if the span arithmetic fits 32 bits
+    int chain_by_flag;       // 1 if the host vouches that the previous step launch on the stream used this
+                             // very workspace, memory and outputs: its completion word is then enough
 };
+
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ unsigned int ld_acquire(const unsigned int *p)
+{
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(unsigned int *p, unsigned int v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fence_acq_rel() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+
+constexpr int kFlagPolls = 1 << 14;   // bounded: a few milliseconds, then the hardware wait takes over
+
+// Named barriers (ids 1..15; id 0 is __syncthreads): `count` threads, whole warps, take part.
+__device__ __forceinline__ void named_barrier_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+__device__ __forceinline__ void named_barrier_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 
 constexpr int kHintNone = -1;          // nothing to record at this position
 constexpr int kHintAbsent = -2;        // recorded pair not in the table and no slot reserved
 constexpr int kHintCareful = 1 << 30;  // count close to saturation: add with the wrap check
+
+// Wait until at least `need` launches have completed on this workspace (all of their
+// writes to the memory, the outputs and the scratch are then visible).  The last warp of
+// a launch publishes the count with a release store; waiting for the whole previous grid
+// to retire (griddepcontrol.wait) costs several microseconds more per step, so when the
+// host vouches that the previous step launch on the stream is the one that will publish
+// the count (same workspace, memory and outputs), the count is polled instead.  That
+// launch is resident by then (a dependent launch begins only after every block of its
+// predecessor has started), so the poll ends; it is bounded all the same, and whenever
+// it runs out, or the host could not vouch, the hardware wait decides.
+__device__ __forceinline__ void wait_completed(const StepParams &p, unsigned int need)
+{
+    if (p.chain_by_flag) {
+        for (int i = 0; i < kFlagPolls; ++i)
+            if (static_cast<int>(ld_acquire(p.completed) - need) >= 0) return;
+    }
+    pdl_wait();
+}
 
 // ---- element access policies ---------------------------------------------------------
 
@@ -306,9 +347,6 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
     return p;
 }
 
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 // ---- the even split of the unit space over blocks -----------------------------------------
 
 __device__ __forceinline__ long long span_begin(const StepParams &p, int c)
@@ -438,7 +476,7 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, int half, int b, 
 }
 
 template <typename L>
-__device__ void finalize_batch_row(const StepParams &p, int half, int b, int lane, RowScratch &rs)
+__device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, int lane, RowScratch &rs)
 {
     using E = typename L::elem;
     const int K = p.K;
@@ -456,13 +494,25 @@ __device__ void finalize_batch_row(const StepParams &p, int half, int b, int lan
             zd = L::load_elem(rowp, d);
         }
     }
+    const int half = static_cast<int>(seq & 1u);
     fold_rows(p, half, b, lane, rs);
 
     // Everything above read only this launch's inputs and its own half of the scratch.
     // From here on the previous launch must be complete: the memory, its statistics and
     // the output buffers come into play.
-    pdl_wait();
+    wait_completed(p, seq);
+    // S3.  The update regime (one load, used only after the look-up) is requested first so
+    // that it travels together with the probe.
     const int regime = p.do_update ? update_regime(p) : kRegimeFull;
+    bool match = false, ok = false;
+    int t = -1;
+    unsigned int cnt = 0;
+    long long slot = -1, empty_slot = -1;
+    if (lane < K) {
+        t = rs.t[lane];
+        match = (d == t);
+        if (valid) cnt = ocm_lookup(p.ocm, make_key(d, t), &slot, &empty_slot);
+    }
     for (int row = lane; row <= K; row += 32) {
         const size_t at = (size_t)b * (K + 1) + row;
         const float s_m = rs.s[row];
@@ -473,17 +523,10 @@ __device__ void finalize_batch_row(const StepParams &p, int half, int b, int lan
         if (p.diag.t) p.diag.t[at] = rs.t[row];
     }
 
-    // S2 (second half), S3, S4 per position; S5 across the warp.
-    bool match = false, ok = false;
-    int t = -1;
-    unsigned int cnt = 0;
-    long long slot = -1;
+    // S2 (second half), S4 per position; S5 across the warp.
     if (lane < K) {
-        t = rs.t[lane];
         const float m = rs.m[lane];
         const float s_m = rs.s[lane];
-        match = (d == t);
-        if (valid) cnt = ocm_lookup(p.ocm, make_key(d, t), &slot);                     // S3
         const bool is_freq = cnt >= p.ocm.lambda;
         const bool is_safe = (static_cast<double>(zd) - static_cast<double>(m)) >= static_cast<double>(p.log_tau);  // S4, Eq. 3
         ok = match || (valid && is_freq && is_safe);
@@ -512,7 +555,7 @@ __device__ void finalize_batch_row(const StepParams &p, int half, int b, int lan
             // S6, first half: leave the slot of every recorded pair for the final adder
             int hint = kHintNone;
             if (record) {
-                if (slot < 0 && regime == kRegimeRoom) slot = ocm_reserve(p.ocm, make_key(d, t));
+                if (slot < 0 && regime == kRegimeRoom) slot = ocm_reserve(p.ocm, make_key(d, t), empty_slot);
                 hint = slot < 0 ? kHintAbsent : static_cast<int>(slot);
                 const unsigned int room = 0xffffffffu - static_cast<unsigned int>(p.B * p.K);
                 if (slot >= 0 && cnt > room) hint |= kHintCareful;
@@ -535,14 +578,14 @@ __device__ void finalize_batch_row(const StepParams &p, int half, int b, int lan
         if (m_bad) atomicOr(&st->flags, CSD_FLAG_BAD_DRAFT);
     }
     __syncwarp();
+    return regime;
 }
 
 // S6, second half, by the warp that finalised the last batch row: every look-up of the
 // step is done, so the counts may change now.
-__device__ void apply_step_update(const StepParams &p, int half, int lane, CanonScratch &canon)
+__device__ void apply_step_update(const StepParams &p, int half, int lane, CanonScratch &canon, int regime)
 {
     const int n = p.B * p.K;
-    const int regime = update_regime(p);
     if (regime == kRegimeTransition) {
         ocm_update_group<false>(p.ocm, p.rej_d, p.rej_t, nullptr, n, canon, lane, 32);
         return;
@@ -589,8 +632,7 @@ __device__ void publish_and_finalize(const StepParams &p, BlockState &bs, RowScr
     // This half was last used by launch seq-2.  If that launch is known to be complete the
     // scratch can be written right away; otherwise wait for the previous launch first
     // (launches complete in order, so that covers seq-2 as well).
-    const unsigned int completed = __ldcg(p.completed);
-    if (static_cast<int>(completed - (seq - 1u)) < 0) pdl_wait();
+    if (static_cast<int>(ld_acquire(p.completed) - (seq - 1u)) < 0) wait_completed(p, seq - 1u);
     int my_b = -1;
     if (lane < nseg) {
         const int row = first_row + lane;
@@ -619,25 +661,33 @@ __device__ void publish_and_finalize(const StepParams &p, BlockState &bs, RowScr
         todo &= todo - 1;
         const int b = __shfl_sync(kFull, my_b, src);
         __threadfence();
-        finalize_batch_row<L>(p, half, b, lane, rs);
+        const int regime = finalize_batch_row<L>(p, seq, b, lane, rs);   // the same for every row of a launch
         bool last = false;
         if (lane == 0) p.b_ticket[half][b] = 0u;          // ready for the launch after next
-        __threadfence();
-        __syncwarp();
+        fence_acq_rel();                                  // each lane's outputs and hints of this row ...
+        __syncwarp();                                     // ... all of them before the row's ticket
         if (lane == 0) last = atomicAdd(p.g_ticket[half], 1u) == static_cast<unsigned int>(p.B) - 1u;
         last = __shfl_sync(kFull, last, 0);
         if (!last) continue;
 
         // ---- every batch row is final: S6 ----
-        __threadfence();
-        if (p.do_update) apply_step_update(p, half, lane, canon);
+        fence_acq_rel();
+        OcmStatsDev *st = p.ocm.stats;
+        // new keys are claimed by the look-ups (above) except near the key limit, where the
+        // update itself inserts: only then does the key count have to be read afterwards
+        const bool keys_settled = !p.do_update || regime != kRegimeTransition;
+        unsigned long long nk = 0;
+        if (lane == 0 && keys_settled) nk = atomicAdd(&st->n_keys, 0ull);   // in flight next to the hint loads
+        if (p.do_update) apply_step_update(p, half, lane, canon, regime);
         if (lane == 0) {
-            OcmStatsDev *st = p.ocm.stats;
-            __threadfence();
-            st->n_keys_start = atomicAdd(&st->n_keys, 0ull);
+            if (!keys_settled) {
+                fence_acq_rel();
+                nk = atomicAdd(&st->n_keys, 0ull);
+            }
+            st->n_keys_start = nk;
             atomicAdd(&st->steps, 1ull);
             *p.g_ticket[half] = 0u;
-            __stcg(p.completed, seq + 1u);
+            st_release(p.completed, seq + 1u);            // everything above, and all it observed, first
         }
     }
 }
@@ -653,21 +703,19 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
 
     using E = typename L::elem;
     const int lane = threadIdx.x & 31;
-    if (threadIdx.x < 32) {
-        // Launch sequence number, one atomic: the word holds (sequence << 32 | blocks counted
-        // in).  Every block counts itself in and learns the sequence from the same answer;
-        // the block that is last to do so moves the word on to the next launch.  That launch
-        // can begin only after every block of this one has released it, which a block does
-        // after counting itself in -- so all blocks of a launch see the same number.
-        if (lane == 0) {
-            const unsigned long long old = atomicAdd(p.launch_seq, 1ull);
-            if (static_cast<unsigned int>(old) == gridDim.x - 1)
-                atomicAdd(p.launch_seq, (1ull << 32) - static_cast<unsigned long long>(gridDim.x));
-            bs.seq = static_cast<unsigned int>(old >> 32);     // read after the first block barrier
-        }
-        __syncwarp();
-        pdl_launch_dependents();
-    }
+    const int warp = threadIdx.x >> 5;
+    const int nwarps = blockDim.x >> 5;
+    // Launch sequence number, one atomic: the word holds (sequence << 32 | blocks counted
+    // in).  Every block counts itself in and learns the sequence from the same answer;
+    // the block that is last to do so moves the word on to the next launch.  That launch
+    // can begin only after every block of this one has released it, which a block does
+    // after counting itself in -- so all blocks of a launch see the same number.
+    // The block's LAST warp does this, so that the round trip of the (contended) atomic
+    // delays neither the other warps' start nor the set-up of the shared tables; it joins
+    // the streaming afterwards.
+    const bool seq_warp = warp == nwarps - 1;
+    unsigned long long seq_old = 0;
+    if (seq_warp && lane == 0) seq_old = atomicAdd(p.launch_seq, 1ull);
     const int K1 = p.K + 1;
     const int U = p.units_per_row;
     const int CH = p.chunk_units;
@@ -675,6 +723,7 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
     long long g = span_begin(p, blockIdx.x);
     const long long g_end = span_begin(p, blockIdx.x + 1);
 
+    bool first_window = true;
     while (g < g_end) {
         // ---- a window: up to kMaxSegs consecutive row parts of this block's span ----
         const long long row0 = g / U;
@@ -689,12 +738,41 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
         const int n_last = (last_units + CH - 1) / CH;
         const int nchunks = nseg == 1 ? n0 : n0 + (nseg - 2) * cpr + n_last;
 
+        // the first window's fold count has one extra party: the sequence number's arrival
+        const unsigned int fold_target = static_cast<unsigned int>(nseg) + (first_window ? 1u : 0u);
         if (threadIdx.x == 0) {
             bs.next_chunk = 0u;
             bs.segs_folded = 0u;
         }
-        if (threadIdx.x < kMaxSegs) bs.seg_done[threadIdx.x] = 0u;
-        __syncthreads();
+        if (threadIdx.x < kMaxSegs) bs.seg_done[threadIdx.x] = 0u;   // kMaxSegs <= 32: warp 0 only
+        if (!first_window || nwarps == 1) {
+            __syncthreads();
+        } else if (seq_warp) {
+            named_barrier_sync(2, 64);                  // tables are set up (warp 0 arrived)
+        } else {
+            if (warp == 0) named_barrier_arrive(2, 64);
+            named_barrier_sync(1, 32 * (nwarps - 1));   // the streaming warps start without the last warp
+        }
+        if (first_window && seq_warp) {
+            if (lane == 0) {
+                if (static_cast<unsigned int>(seq_old) == gridDim.x - 1)
+                    atomicAdd(p.launch_seq, (1ull << 32) - static_cast<unsigned long long>(gridDim.x));
+                bs.seq = static_cast<unsigned int>(seq_old >> 32);
+            }
+            __syncwarp();
+            pdl_launch_dependents();
+            bool block_complete = false;
+            if (lane == 0) {
+                __threadfence_block();
+                block_complete = atomicAdd(&bs.segs_folded, 1u) == fold_target - 1u;
+            }
+            if (__shfl_sync(kFull, block_complete, 0)) {   // everything else was already folded
+                __threadfence_block();
+                const int next_b = w_end < g_end ? static_cast<int>((w_end / U) / K1) : -1;
+                publish_and_finalize<L>(p, bs, row_scratch, canon, static_cast<int>(row0), nseg, next_b, lane);
+            }
+        }
+        first_window = false;
 
         while (true) {
             unsigned int q = 0;
@@ -744,7 +822,7 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             if (lane == 0) {
                 bs.seg_result[seg] = v;
                 __threadfence_block();
-                block_complete = atomicAdd(&bs.segs_folded, 1u) == static_cast<unsigned int>(nseg) - 1u;
+                block_complete = atomicAdd(&bs.segs_folded, 1u) == fold_target - 1u;
             }
             if (!__shfl_sync(kFull, block_complete, 0)) continue;
             __threadfence_block();
