@@ -153,7 +153,6 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
     size_t seq_off, half_bytes, partials_off, hint_off, b_ticket_off, g_ticket_off, total;   // *_off within a half
-    size_t half_off[2];
 };
 
 // header {launch sequence, blocks counted in, launches completed} followed by two halves,
@@ -167,9 +166,7 @@ WorkspaceLayout ws_layout(int B, int K, const Shape &s)
     w.b_ticket_off = align_up(w.hint_off + static_cast<size_t>(B) * K * sizeof(int), 256);
     w.g_ticket_off = align_up(w.b_ticket_off + static_cast<size_t>(B) * sizeof(unsigned int), 16);
     w.half_bytes = align_up(w.g_ticket_off + 16, 256);
-    w.half_off[0] = 256;
-    w.half_off[1] = 256 + w.half_bytes;
-    w.total = 256 + 2 * w.half_bytes;
+    w.total = 256 + kScratchRing * w.half_bytes;
     return w;
 }
 
@@ -215,13 +212,12 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.rej_d = rej_draft; p.rej_t = rej_target;
     if (diag) p.diag = *diag;
     char *ws = static_cast<char *>(workspace);
-    for (int h = 0; h < 2; ++h) {
-        char *half = ws + w.half_off[h];
-        p.partials[h] = reinterpret_cast<Partial *>(half + w.partials_off);
-        p.slot_hint[h] = reinterpret_cast<int *>(half + w.hint_off);
-        p.b_ticket[h] = reinterpret_cast<unsigned int *>(half + w.b_ticket_off);
-        p.g_ticket[h] = reinterpret_cast<unsigned int *>(half + w.g_ticket_off);
-    }
+    if (w.half_bytes > 0xffffffffull) return CSD_ERR_UNSUPPORTED;
+    p.scratch = ws + 256;
+    p.copy_bytes = static_cast<unsigned int>(w.half_bytes);
+    p.hint_off = static_cast<unsigned int>(w.hint_off);
+    p.b_ticket_off = static_cast<unsigned int>(w.b_ticket_off);
+    p.g_ticket_off = static_cast<unsigned int>(w.g_ticket_off);
     p.launch_seq = reinterpret_cast<unsigned long long *>(ws + w.seq_off);
     p.completed = reinterpret_cast<unsigned int *>(ws + w.seq_off + 8);
     p.n_spans = s.grid;

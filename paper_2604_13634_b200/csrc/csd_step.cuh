@@ -63,12 +63,14 @@ struct StepParams {
     int *rej_d;
     int *rej_t;
     csd_diag_t diag;
-    // Two copies of the scratch ("halves"), used by consecutive launches in turn, so that
-    // a launch can publish and fold while the previous one is still finishing.
-    Partial *partials[2];       // [R * slots_per_row]: one slot per (row, block touching it)
-    int *slot_hint[2];          // [B * K] slot of each recorded pair (see kHint*)
-    unsigned int *b_ticket[2];  // [B]
-    unsigned int *g_ticket[2];  // [1]
+    // kScratchRing copies of the scratch, used by consecutive launches in turn, so that a
+    // launch can publish and fold while the launches before it are still finishing.  A copy:
+    //   partials [R * slots_per_row]  one slot per (row, block touching it)       at 0
+    //   slot hints [B * K]            slot of each recorded pair (see kHint*)     at hint_off
+    //   batch-row tickets [B]                                                     at b_ticket_off
+    //   global ticket [1]                                                         at g_ticket_off
+    char *scratch;
+    unsigned int copy_bytes, hint_off, b_ticket_off, g_ticket_off;
     unsigned long long *launch_seq;  // (sequence number of the launch now starting << 32) | blocks counted in
     unsigned int *completed;         // launches completed on this workspace
     int n_spans;             // G: blocks that own a span of the unit space
@@ -102,6 +104,27 @@ constexpr int kFlagPolls = 1 << 14;   // bounded: a few milliseconds, then the h
 // Named barriers (ids 1..15; id 0 is __syncthreads): `count` threads, whole warps, take part.
 __device__ __forceinline__ void named_barrier_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 __device__ __forceinline__ void named_barrier_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+
+constexpr unsigned int kScratchRing = 4;   // power of two
+
+struct ScratchCopy {
+    Partial *partials;
+    int *slot_hint;
+    unsigned int *b_ticket;
+    unsigned int *g_ticket;
+};
+
+// The scratch copy that launch number `seq` on this workspace works in.
+__device__ __forceinline__ ScratchCopy scratch_of(const StepParams &p, unsigned int seq)
+{
+    char *base = p.scratch + static_cast<size_t>(seq & (kScratchRing - 1u)) * p.copy_bytes;
+    ScratchCopy c;
+    c.partials = reinterpret_cast<Partial *>(base);
+    c.slot_hint = reinterpret_cast<int *>(base + p.hint_off);
+    c.b_ticket = reinterpret_cast<unsigned int *>(base + p.b_ticket_off);
+    c.g_ticket = reinterpret_cast<unsigned int *>(base + p.g_ticket_off);
+    return c;
+}
 
 constexpr int kHintNone = -1;          // nothing to record at this position
 constexpr int kHintAbsent = -2;        // recorded pair not in the table and no slot reserved
@@ -365,6 +388,7 @@ __device__ __forceinline__ int owner_of(const StepParams &p, long long g)
     return static_cast<int>(((g + 1) * p.n_spans - 1) / p.total_units);
 }
 
+constexpr int kFinalizeWarps = 8;  // warps of a block that share its batch rows to finalise
 constexpr int kMaxSegs = 32;       // row parts a block handles between two block barriers
 constexpr int kMaxChunks = 1024;   // chunk results held in shared memory at a time
 
@@ -375,6 +399,8 @@ struct BlockState {
     unsigned int seg_done[kMaxSegs];    // chunks delivered per row part
     Partial seg_result[kMaxSegs];
     Partial chunk_part[kMaxChunks];
+    int n_todo;                         // batch rows this block has to finalise in this window ...
+    int todo_b[kMaxSegs];               // ... and which
 };
 
 // ---- S2..S5 for one batch row, by one warp ------------------------------------------
@@ -427,7 +453,7 @@ __device__ __forceinline__ Partial butterfly_fold(Partial v, int width)
 // Fold the per-block partials of the K+1 logit rows of batch row b (S1, last level).  The
 // lanes are arranged as (32 / width) rows x width slots, width = the power of two >= the
 // slots per row (at most 32; more slots are pre-folded in lane order).
-__device__ __forceinline__ void fold_rows(const StepParams &p, int half, int b, int lane, RowScratch &rs)
+__device__ __forceinline__ void fold_rows(const StepParams &p, const ScratchCopy &sc, int b, int lane, RowScratch &rs)
 {
     const int K1 = p.K + 1, S = p.slots_per_row;
     int width = 1;
@@ -436,7 +462,7 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, int half, int b, 
     const int sub = lane / width;          // which row of the pass
     const int k0 = lane - sub * width;     // first slot this lane folds
     const size_t row0 = (size_t)b * K1;
-    const Partial *part = p.partials[half] + row0 * S;
+    const Partial *part = sc.partials + row0 * S;
 
     for (int r = lane; r < K1; r += 32) {
         const long long u0 = static_cast<long long>(row0 + r) * p.units_per_row;
@@ -494,8 +520,8 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
             zd = L::load_elem(rowp, d);
         }
     }
-    const int half = static_cast<int>(seq & 1u);
-    fold_rows(p, half, b, lane, rs);
+    const ScratchCopy sc = scratch_of(p, seq);
+    fold_rows(p, sc, b, lane, rs);
 
     // Everything above read only this launch's inputs and its own half of the scratch.
     // From here on the previous launch must be complete: the memory, its statistics and
@@ -560,7 +586,7 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
                 const unsigned int room = 0xffffffffu - static_cast<unsigned int>(p.B * p.K);
                 if (slot >= 0 && cnt > room) hint |= kHintCareful;
             }
-            __stcg(p.slot_hint[half] + pos, hint);
+            __stcg(sc.slot_hint + pos, hint);
         }
     }
     const unsigned int m_match = __ballot_sync(kFull, reached && match);
@@ -583,7 +609,7 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
 
 // S6, second half, by the warp that finalised the last batch row: every look-up of the
 // step is done, so the counts may change now.
-__device__ void apply_step_update(const StepParams &p, int half, int lane, CanonScratch &canon, int regime)
+__device__ void apply_step_update(const StepParams &p, const ScratchCopy &sc, int lane, CanonScratch &canon, int regime)
 {
     const int n = p.B * p.K;
     if (regime == kRegimeTransition) {
@@ -596,7 +622,7 @@ __device__ void apply_step_update(const StepParams &p, int half, int lane, Canon
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             const int j = j0 + q * 32 + lane;
-            h[q] = j < n ? __ldcg(p.slot_hint[half] + j) : kHintNone;
+            h[q] = j < n ? __ldcg(sc.slot_hint + j) : kHintNone;
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
@@ -617,27 +643,27 @@ __device__ void apply_step_update(const StepParams &p, int half, int lane, Canon
     __syncwarp();
 }
 
-// Publication of a block's row parts and everything that may follow from it: tickets,
-// batch-row finalisation, the memory update.  Executed by ONE warp of the block.
+// Publication of a block's row parts: partials to global memory, one ticket per batch row
+// touched.  Executed by ONE warp of the block.  The batch rows whose last part this block
+// delivered are left in bs.todo_b for the block's warps to finalise.
 //   nseg row parts, rows first_row .. first_row + nseg - 1, results in bs.seg_result;
 //   next_b: batch row of the next row this block will still publish, or -1.
-template <typename L>
-__device__ void publish_and_finalize(const StepParams &p, BlockState &bs, RowScratch &rs, CanonScratch &canon,
-                                     int first_row, int nseg, int next_b, int lane)
+__device__ void publish_parts(const StepParams &p, BlockState &bs, int first_row, int nseg, int next_b, int lane)
 {
     const int K1 = p.K + 1;
     const int U = p.units_per_row;
     const unsigned int seq = bs.seq;
-    const int half = static_cast<int>(seq & 1u);
-    // This half was last used by launch seq-2.  If that launch is known to be complete the
-    // scratch can be written right away; otherwise wait for the previous launch first
-    // (launches complete in order, so that covers seq-2 as well).
-    if (static_cast<int>(ld_acquire(p.completed) - (seq - 1u)) < 0) wait_completed(p, seq - 1u);
+    const ScratchCopy sc = scratch_of(p, seq);
+    // This copy was last used by launch seq - kScratchRing.  If that launch is known to be
+    // complete the scratch can be written right away; otherwise wait for it (launches
+    // complete in order).
+    const unsigned int need = seq - (kScratchRing - 1u);
+    if (static_cast<int>(ld_acquire(p.completed) - need) < 0) wait_completed(p, need);
     int my_b = -1;
     if (lane < nseg) {
         const int row = first_row + lane;
         const int slot = static_cast<int>(blockIdx.x) - owner_of(p, static_cast<long long>(row) * U);
-        if (slot < p.slots_per_row) st_partial_cg(p.partials[half] + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
+        if (slot < p.slots_per_row) st_partial_cg(sc.partials + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
         my_b = row / K1;
     }
     __threadfence();
@@ -650,45 +676,47 @@ __device__ void publish_and_finalize(const StepParams &p, BlockState &bs, RowScr
         if (closes) {
             const long long u0 = static_cast<long long>(my_b) * K1 * U;
             const unsigned int expected = owner_of(p, u0 + static_cast<long long>(K1) * U - 1) - owner_of(p, u0) + 1;
-            completes = atomicAdd(p.b_ticket[half] + my_b, 1u) == expected - 1;
+            completes = atomicAdd(sc.b_ticket + my_b, 1u) == expected - 1;
         }
     }
-    unsigned int todo = __ballot_sync(kFull, completes);
+    const unsigned int todo = __ballot_sync(kFull, completes);
+    if (completes) bs.todo_b[__popc(todo & ((1u << lane) - 1u))] = my_b;
+    if (lane == 0) bs.n_todo = __popc(todo);
+    __threadfence();      // the other blocks' partials of those rows, before this block's warps read them
+}
 
-    // ---- this block delivered a batch row's last part: S2..S5 ----
-    while (todo) {
-        const int src = __ffs(todo) - 1;
-        todo &= todo - 1;
-        const int b = __shfl_sync(kFull, my_b, src);
-        __threadfence();
-        const int regime = finalize_batch_row<L>(p, seq, b, lane, rs);   // the same for every row of a launch
-        bool last = false;
-        if (lane == 0) p.b_ticket[half][b] = 0u;          // ready for the launch after next
-        fence_acq_rel();                                  // each lane's outputs and hints of this row ...
-        __syncwarp();                                     // ... all of them before the row's ticket
-        if (lane == 0) last = atomicAdd(p.g_ticket[half], 1u) == static_cast<unsigned int>(p.B) - 1u;
-        last = __shfl_sync(kFull, last, 0);
-        if (!last) continue;
+// S2..S5 of batch row b by one warp, and, if that was the launch's last row, S6.
+template <typename L>
+__device__ void finalize_and_update(const StepParams &p, unsigned int seq, int b, int lane, RowScratch &rs, CanonScratch &canon)
+{
+    const ScratchCopy sc = scratch_of(p, seq);
+    const int regime = finalize_batch_row<L>(p, seq, b, lane, rs);   // the same for every row of a launch
+    bool last = false;
+    if (lane == 0) sc.b_ticket[b] = 0u;               // ready for this copy's next launch
+    fence_acq_rel();                                  // each lane's outputs and hints of this row ...
+    __syncwarp();                                     // ... all of them before the row's ticket
+    if (lane == 0) last = atomicAdd(sc.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
+    last = __shfl_sync(kFull, last, 0);
+    if (!last) return;
 
-        // ---- every batch row is final: S6 ----
-        fence_acq_rel();
-        OcmStatsDev *st = p.ocm.stats;
-        // new keys are claimed by the look-ups (above) except near the key limit, where the
-        // update itself inserts: only then does the key count have to be read afterwards
-        const bool keys_settled = !p.do_update || regime != kRegimeTransition;
-        unsigned long long nk = 0;
-        if (lane == 0 && keys_settled) nk = atomicAdd(&st->n_keys, 0ull);   // in flight next to the hint loads
-        if (p.do_update) apply_step_update(p, half, lane, canon, regime);
-        if (lane == 0) {
-            if (!keys_settled) {
-                fence_acq_rel();
-                nk = atomicAdd(&st->n_keys, 0ull);
-            }
-            st->n_keys_start = nk;
-            atomicAdd(&st->steps, 1ull);
-            *p.g_ticket[half] = 0u;
-            st_release(p.completed, seq + 1u);            // everything above, and all it observed, first
+    // ---- every batch row is final: S6 ----
+    fence_acq_rel();
+    OcmStatsDev *st = p.ocm.stats;
+    // new keys are claimed by the look-ups (above) except near the key limit, where the
+    // update itself inserts: only then does the key count have to be read afterwards
+    const bool keys_settled = !p.do_update || regime != kRegimeTransition;
+    unsigned long long nk = 0;
+    if (lane == 0 && keys_settled) nk = atomicAdd(&st->n_keys, 0ull);   // in flight next to the hint loads
+    if (p.do_update) apply_step_update(p, sc, lane, canon, regime);
+    if (lane == 0) {
+        if (!keys_settled) {
+            fence_acq_rel();
+            nk = atomicAdd(&st->n_keys, 0ull);
         }
+        st->n_keys_start = nk;
+        atomicAdd(&st->steps, 1ull);
+        *sc.g_ticket = 0u;
+        st_release(p.completed, seq + 1u);            // everything above, and all it observed, first
     }
 }
 
@@ -698,7 +726,7 @@ template <typename L>
 __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ StepParams p)
 {
     __shared__ BlockState bs;
-    __shared__ RowScratch row_scratch;
+    __shared__ RowScratch row_scratch[kFinalizeWarps];
     __shared__ CanonScratch canon;
 
     using E = typename L::elem;
@@ -743,6 +771,7 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
         if (threadIdx.x == 0) {
             bs.next_chunk = 0u;
             bs.segs_folded = 0u;
+            bs.n_todo = 0;
         }
         if (threadIdx.x < kMaxSegs) bs.seg_done[threadIdx.x] = 0u;   // kMaxSegs <= 32: warp 0 only
         if (!first_window || nwarps == 1) {
@@ -769,7 +798,7 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             if (__shfl_sync(kFull, block_complete, 0)) {   // everything else was already folded
                 __threadfence_block();
                 const int next_b = w_end < g_end ? static_cast<int>((w_end / U) / K1) : -1;
-                publish_and_finalize<L>(p, bs, row_scratch, canon, static_cast<int>(row0), nseg, next_b, lane);
+                publish_parts(p, bs, static_cast<int>(row0), nseg, next_b, lane);
             }
         }
         first_window = false;
@@ -827,8 +856,14 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             if (!__shfl_sync(kFull, block_complete, 0)) continue;
             __threadfence_block();
             const int next_b = w_end < g_end ? static_cast<int>((w_end / U) / K1) : -1;
-            publish_and_finalize<L>(p, bs, row_scratch, canon, static_cast<int>(row0), nseg, next_b, lane);
+            publish_parts(p, bs, static_cast<int>(row0), nseg, next_b, lane);
         }
+        // ---- the batch rows this block completed are shared out over its warps: S2..S6 ----
+        __syncthreads();
+        const int fin_warps = nwarps < kFinalizeWarps ? nwarps : kFinalizeWarps;
+        if (warp < fin_warps)
+            for (int j = warp; j < bs.n_todo; j += fin_warps)
+                finalize_and_update<L>(p, bs.seq, bs.todo_b[j], lane, row_scratch[warp], canon);
         g = w_end;
         if (g < g_end) __syncthreads();       // the next window reuses the shared-memory tables
     }
