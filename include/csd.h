@@ -119,7 +119,8 @@ csd_status_t csd_ocm_set_lambda(csd_ocm_t *ocm, uint32_t lambda);
 /* ---- one verification step ---------------------------------------------------- */
 
 /* Bytes of scratch csd_verify / csd_step need for this shape (0 on invalid shape).
- * The scratch holds per-tile partial reductions and arrival counters. */
+ * The scratch holds, four times over (consecutive launches take the copies in turn),
+ * per-block partial reductions, slot hints and arrival counters. */
 size_t csd_workspace_bytes(int B, int K, int V, csd_dtype_t dtype);
 
 /* Zero a workspace.  Required once before its first use (and after any aborted
@@ -206,7 +207,7 @@ csd_status_t csd_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
  * caller's device buffers); the current device must be the memory's device.
  * Shapes whose csd_workspace_bytes exceeds CSD_STATIC_SCRATCH_BYTES are refused with
  * CSD_ERR_WORKSPACE before anything is launched (all five reference workloads need
- * less than 100 KiB).  The first call on each device looks up the array's device
+ * less than 200 KiB).  The first call on each device looks up the array's device
  * address; make that first call outside any stream capture.  All calls share the one
  * array, which keeps the previous call's contents, so every call first clears the
  * part it uses (asynchronously, on `stream`); two calls that overlap on the GPU (two
@@ -258,7 +259,7 @@ csd_status_t csd_ocm_stats(const csd_ocm_t *ocm, csd_stats_t *host_out, void *st
  * -inf for tau == 0.  Host function. */
 float csd_scg_threshold(float tau);
 
-/* Launch shape a step of this size uses: grid blocks (each owns an equal contiguous
+/* Launch shape a step of this size uses under the current csd_set_overlap setting: grid blocks (each owns an equal contiguous
  * share of the logits), threads per block, elements per chunk (the run of one logit row
  * that a warp reduces at a time) and partial results kept per logit row.  Host function;
  * for reports and tests. */
@@ -267,21 +268,30 @@ csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype,
 
 /* Expert knob, process-wide: override the automatic work split.  chunk_bytes: bytes of
  * one logit row reduced by a warp at a time (multiple of 512; 0 = automatic, 4 to 32 KiB);
- * ctas_per_sm: blocks of the persistent grid per SM (0 = automatic, 4); block_threads:
+ * ctas_per_sm: blocks of the persistent grid per SM (0 = automatic: 4, or 1 with
+ * csd_set_overlap); block_threads:
  * threads per block (multiple of 32, at most 1024; 0 = automatic, 256).  Changes
  * csd_workspace_bytes: size workspaces after calling it.  Results stay
  * bit-reproducible for a fixed setting; the low-order bits of the sums s may differ
  * between settings (different summation trees).  Host function. */
 csd_status_t csd_set_tuning(int chunk_bytes, int ctas_per_sm, int block_threads);
 
-/* Process-wide, off by default.  When on, csd_verify / csd_step launch with
- * programmatic stream serialization: the kernel may start, and stream logits, while
- * the previous kernel on the stream is still draining; it waits for that kernel to
- * complete before it first touches the workspace, the memory or any output.  Turn it
- * on only if the logits and draft of a step are never written by the kernel launched
- * directly before that step on the same stream (back-to-back steps over inputs that
- * are already resident qualify; a producer kernel launched right before the step
- * does too as long as it does not itself signal early completion).  Host function. */
+/* Process-wide, off by default: for callers that issue steps back to back.  When on,
+ * csd_verify / csd_step launch with programmatic stream serialization: the kernel may
+ * start, and stream logits, while earlier kernels on the stream are still running; it
+ * waits for the previous step before it first touches the memory or any output.  If
+ * that previous step was launched on the same stream with the same workspace, memory,
+ * output buffers and shape (and no other call of this library came between), the wait
+ * is on a completion count that the previous step leaves in the workspace; in every
+ * other case it is the hardware's wait for the previous kernel on the stream to
+ * retire.  The automatic launch shape also changes: one block per SM and launch
+ * instead of four, so that several steps are resident at a time (the low-order bits of
+ * the diagnostic sums s may therefore differ from those with overlap off; all decisions
+ * are identical).  Turn it on only if the logits and draft of a step are never written
+ * by a kernel that may still be running when the step starts: back-to-back steps over
+ * inputs that are already resident qualify; so does a producer kernel launched right
+ * before the step as long as it does not itself signal early completion.  Steps that
+ * share a memory or output buffers are issued on one stream.  Host function. */
 csd_status_t csd_set_overlap(int enable);
 
 const char *csd_status_string(csd_status_t status);

@@ -113,12 +113,16 @@ bool shape_ok(int B, int K, int V, csd_dtype_t dt)
 }
 
 // The unit space (R rows x U units of 512 bytes) is split evenly over the blocks of a
-// persistent grid: as many blocks as fit the machine, but no more than 64 per row (few
-// partials per row keep the last fold short), at least ~8 KiB each, never more than units.
-Shape pick_shape(int B, int K, int V, csd_dtype_t dt)
+// persistent grid, but no more than 64 blocks per row (few partials per row keep the last
+// fold short), at least ~8 KiB each, never more than units.  Blocks per SM: a launch that
+// runs alone needs the whole machine (4 blocks per SM, all that fit); with step overlap
+// several launches are resident at once and share it, and one block per SM and launch
+// lets the next launches start while this one is still streaming (measured: 1 is best on
+// every reference workload, 4 costs 15 to 50 % there).
+Shape pick_shape(int B, int K, int V, csd_dtype_t dt, bool overlap)
 {
     const int eb = elt_bytes(dt);
-    const int ctas_per_sm = g_ctas_per_sm_override > 0 ? g_ctas_per_sm_override : 4;
+    const int ctas_per_sm = g_ctas_per_sm_override > 0 ? g_ctas_per_sm_override : (overlap ? 1 : 4);
     const long long rows = static_cast<long long>(B) * (K + 1);
     Shape s;
     s.block = g_block_threads_override > 0 ? g_block_threads_override : kThreads;
@@ -195,7 +199,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     if (!(tau >= 0.0f) || std::isinf(tau)) return CSD_ERR_INVALID_ARG;   // also refuses NaN
     if (stride_k < V || stride_b < stride_k * (K + 1)) return CSD_ERR_INVALID_ARG;
 
-    const Shape s = pick_shape(B, K, V, dtype);
+    const Shape s = pick_shape(B, K, V, dtype, g_overlap_steps != 0);
     const WorkspaceLayout w = ws_layout(B, K, s);
     if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
 
@@ -348,7 +352,10 @@ csd_status_t csd_ocm_set_lambda(csd_ocm_t *ocm, uint32_t lambda)
 size_t csd_workspace_bytes(int B, int K, int V, csd_dtype_t dtype)
 {
     if (!shape_ok(B, K, V, dtype)) return 0;
-    return ws_layout(B, K, pick_shape(B, K, V, dtype)).total;
+    // enough for either launch shape, so that csd_set_overlap does not change the answer
+    const size_t a = ws_layout(B, K, pick_shape(B, K, V, dtype, false)).total;
+    const size_t b = ws_layout(B, K, pick_shape(B, K, V, dtype, true)).total;
+    return a > b ? a : b;
 }
 
 csd_status_t csd_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
@@ -578,7 +585,7 @@ csd_status_t csd_launch_shape(int B, int K, int V, csd_dtype_t dtype, int *grid,
                               int *parts_per_row)
 {
     if (!shape_ok(B, K, V, dtype)) return CSD_ERR_INVALID_ARG;
-    const Shape s = pick_shape(B, K, V, dtype);
+    const Shape s = pick_shape(B, K, V, dtype, g_overlap_steps != 0);
     if (grid) *grid = s.grid;
     if (block) *block = s.block;
     if (chunk_elems) *chunk_elems = s.chunk_units * s.unit_elems;
