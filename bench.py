@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0            # earlier measurement on this machine, used wh
 DEFAULT_WORKLOAD = "large_batch"
 # DRAM bytes per launch of the step kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); a workload is absent where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"large_batch": 600073728, "batched_serving": 59502336}
+NCU_TRAFFIC_BYTES = {"large_batch": 596234240, "batched_serving": 58542336}
 
 
 def measured_peak():
@@ -360,7 +360,8 @@ def run_ours(args, wl, tau):
                              f"({bench.ring_len * wl.logit_bytes / 1e6:.0f} MB, > 2x L2)",
                 "launch": ("CUDA graph of %d steps replayed" % bench.graph_steps) if use_graph else "eager",
                 "step_overlap": "off" if args.no_overlap else
-                                "programmatic dependent launch: a step streams its logits while the previous step drains",
+                                "programmatic dependent launch, one block per SM and launch: a step streams its "
+                                "logits while the steps before it finish",
                 "kernel_shape": shape}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_source": f"of {peak_kind}",

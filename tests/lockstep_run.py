@@ -29,6 +29,9 @@ from paper_2604_13634_b200 import Ocm, StepBuffers, csd_step     # noqa: E402
 from paper_2604_13634_b200.synth import WORKLOADS, Synth         # noqa: E402
 
 
+OVERLAP = False
+
+
 def run(wl, tau, steps, checkpoint, prewarm_steps, seed=0):
     syn = Synth(wl, seed, "cuda")
     ocm = Ocm(wl.ocm_slots, wl.lam)
@@ -63,7 +66,7 @@ def run(wl, tau, steps, checkpoint, prewarm_steps, seed=0):
                accepted=acc, rescued=resc, acceptance_rate=acc / (steps * wl.B * wl.K), near_ties=near,
                diag_steps_checked=checked_diag, n_keys=st["n_keys"], n_dropped=st["n_dropped"],
                checkpoints=(steps // checkpoint if checkpoint else 0), seconds=round(time.time() - t0, 1),
-               verdict="identical")
+               overlap_launch_shape=bool(OVERLAP), verdict="identical")
     ocm.close()
     return out
 
@@ -75,7 +78,14 @@ def main():
     ap.add_argument("--checkpoint", type=int, default=0)
     ap.add_argument("--prewarm-steps", type=int, default=10 ** 9, help="cap on step-type pre-warming")
     ap.add_argument("--taus", default="")
+    ap.add_argument("--overlap", action="store_true",
+                    help="the launch shape the benchmark times (csd_set_overlap: one block per SM and launch)")
     args = ap.parse_args()
+    if args.overlap:
+        from paper_2604_13634_b200 import csd_set_overlap
+        global OVERLAP
+        OVERLAP = True
+        csd_set_overlap(True)
     wl = WORKLOADS[args.workload]
     taus = [float(x) for x in args.taus.split(",")] if args.taus else list(wl.taus)
     for tau in taus:
