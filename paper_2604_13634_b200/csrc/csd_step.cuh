@@ -20,25 +20,36 @@
 //   * The warp that delivers the last chunk of a row's part folds that part (fixed
 //     order) while the others keep streaming; the warp that completes the block's last
 //     fold publishes one partial per (block, row) to global memory: one fence and one
-//     ticket per batch row touched, per BLOCK.  Everything before that reads only the
-//     logits, so with programmatic dependent launch the streaming of step n+1 overlaps
-//     the tail of step n.  The scratch exists twice and launches alternate between the
-//     copies by a sequence number kept in the workspace itself (every block reads it,
-//     the last block to do so advances it, and only then can the next launch begin), so
-//     publication, tickets and the per-row fold of step n+1 also happen while step n is
-//     still finishing; step n+1 waits for step n only before its first OCM look-up and
-//     its first write to an output buffer.
-//   * Whichever block delivers a batch row's last part finalises it (one warp): the
-//     few partials per row are folded by fixed-shape butterflies (maximum first, then
-//     the sums rescaled to the row's reference: bit-reproducible), lanes 0..K-1 take
-//     the per-position decisions, a ballot gives the accepted prefix.
+//     ticket per batch row touched, per BLOCK.  Everything up to here reads only the
+//     logits and writes only this launch's scratch.
+//   * Whichever block delivers a batch row's last part finalises it: the rows a block
+//     completed are shared out over its warps, one warp per row.  The few partials per
+//     row are folded by fixed-shape butterflies (maximum first, then the sums rescaled
+//     to the row's reference: bit-reproducible), lanes 0..K-1 take the per-position
+//     decisions, a ballot gives the accepted prefix.
 //   * Memory update without a second probe: the look-up already found each recorded
 //     pair's slot (absent pairs get an empty slot reserved with count 0, which no
 //     look-up can tell from "absent"), and leaves it as a hint.  The warp finalising
 //     the LAST batch row then only adds 1 to the hinted slots, so every look-up of the
 //     step saw the step-start counts.  Near the key limit, where admission order
 //     matters, that warp falls back to the canonical-order path.
-//   * Nothing ever spins on another block: arrival counters only, so no launch can hang.
+//   * Within a launch nothing ever waits for another block: arrival counters only.
+//
+// Consecutive steps (programmatic dependent launch, opt-in)
+//   * A launch may begin as soon as every block of the previous launch on the stream has
+//     started.  The scratch exists kScratchRing times and launches take the copies in
+//     turn, by a sequence number kept in the workspace itself (every block draws it with
+//     one atomic; the block that draws last advances it; only then can the next launch
+//     begin, so all blocks of a launch see the same number).  Streaming, publication,
+//     tickets and the per-row fold of step n therefore run while steps n-1, n-2, ... are
+//     still finishing.
+//   * What does depend on step n-1 is the memory (its update) and the output buffers.
+//     The finalising warps wait for it just before their look-up: for the completion
+//     count that the last warp of every launch publishes in the workspace (release store,
+//     acquire polls) when the host vouches that step n-1 is the launch that will publish
+//     it, else -- and whenever the bounded poll runs out -- for the previous grid to
+//     retire (griddepcontrol.wait).  A copy of the scratch is reused only after the
+//     launch that last used it has completed (same wait).
 #pragma once
 
 #include <cuda_bf16.h>
