@@ -1,0 +1,267 @@
+"""Pins of the stochastic-verification oracle (oracle/csd_sampled_oracle.py), CPU only.
+
+What fixes it from outside: the published known-answer vectors of Philox4x32-10, the
+exactness of the exponential race (winner frequencies = normalised weights), the
+property the paper states for speculative sampling (Sec. 3.1: the emitted token follows
+the target distribution exactly when nothing is rescued), the reduction to the greedy
+oracle as T -> 0, Eq. 3's temperature invariance, hand traces of the rescue / update
+logic, and planted mistakes that some pin must catch.
+"""
+import importlib.util
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import csd_oracle as GREEDY
+from oracle import csd_sampled_oracle as ORACLE
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def pin_philox_known_answers(mod):
+    rows = [l.split() for l in open(os.path.join(HERE, "golden", "philox4x32_10_kat.txt")) if l.strip() and l[0] != "#"]
+    assert len(rows) == 3
+    for w in rows:
+        v = [int(x, 16) for x in w]
+        out = mod.philox4x32_10([v[0]], [v[1]], [v[2]], [v[3]], v[4], v[5])
+        assert [int(o[0]) for o in out] == v[6:], w
+
+
+def pin_clocks_are_exponential(mod):
+    e = mod.race_clocks(12345, 7, 200001)
+    assert e.shape == (200001,) and np.all(e > 0) and np.all(np.isfinite(e))
+    assert abs(e.mean() - 1.0) < 0.01 and abs(np.median(e) - math.log(2)) < 0.01      # Exp(1)
+    assert abs((e > 2.0).mean() - math.exp(-2.0)) < 0.003
+    assert np.array_equal(e, mod.race_clocks(12345, 7, 200001))                         # a pure function
+    assert not np.array_equal(e[:100], mod.race_clocks(12345, 8, 100))                  # of (seed, row, v)
+    assert not np.array_equal(e[:100], mod.race_clocks(12346, 7, 100))
+    assert np.array_equal(e[:1001], mod.race_clocks(12345, 7, 1001))                    # prefix-stable in V
+    # the smallest and largest clock the 24-bit grid allows
+    assert e.min() >= -math.log1p(-0.5 / 2 ** 24) and e.max() <= -math.log(0.5 / 2 ** 24)
+
+
+def pin_race_draws_from_the_weights(mod):
+    w = np.array([0.0, 3.0, 1.0, 0.0, 6.0, 2.0e-3])
+    n = 12000
+    wins = np.zeros(len(w))
+    for s in range(n):
+        t, _ = mod.race(w, mod.race_clocks(99, s, len(w)), fallback=0)
+        wins[t] += 1
+    pr = w / w.sum()
+    assert wins[0] == 0 and wins[3] == 0
+    assert np.all(np.abs(wins / n - pr) < 4 * np.sqrt(pr * (1 - pr) / n) + 1e-9)
+    # all-zero weights: the stated fallback; ties: lowest index
+    assert mod.race(np.zeros(4), np.ones(4), fallback=2)[0] == 2
+    assert mod.race(np.array([1.0, 2.0, 2.0]), np.array([1.0, 1.0, 1.0]), 0)[0] == 1
+
+
+def _emitted_first_token(mod, z, y, T, n, seed0):
+    """n independent single-position steps with an empty memory: the token emitted at position 0."""
+    V = z.shape[-1]
+    q = np.exp(mod.log_softmax_T(y[0], T)[0])
+    rng = np.random.default_rng(seed0)
+    counts = np.zeros(V)
+    mem = mod.OCM(64, 10 ** 9)
+    zz = np.stack([z[0], z[0]])[None]            # [1, 2, V]: one position plus the bonus row
+    for s in range(n):
+        d = rng.choice(V, p=q)
+        r = rng.random()
+        out = mod.verify(zz, y[None, :1], np.array([[d]]), np.array([[r]]), seed0 * 7919 + s, T, mem, 0.5)
+        counts[d if out["accept_len"][0] == 1 else out["next_token"][0]] += 1
+    return counts
+
+
+def pin_lossless_without_rescue(mod):
+    """Sec. 3.1: accept with min(1, p/q), else draw from norm(max(0, p - q)): the result follows p."""
+    z = np.array([[1.2, -0.3, 0.4, 2.0, -1.0, 0.1]])
+    y = np.array([[0.2, 1.5, 0.4, 0.3, -2.0, 1.0]])
+    for T in (1.0, 0.6):
+        n = 6000
+        counts = _emitted_first_token(mod, z, y, T, n, seed0=5)
+        p = np.exp(mod.log_softmax_T(z[0], T)[0])
+        assert abs(p.sum() - 1) < 1e-12
+        assert np.all(np.abs(counts / n - p) < 4 * np.sqrt(p * (1 - p) / n)), (T, counts / n, p)
+
+
+def pin_alpha_and_normalisers(mod):
+    rng = np.random.default_rng(2)
+    z = rng.normal(size=(2, 3, 50)) * 2
+    y = rng.normal(size=(2, 2, 50)) * 2
+    d = rng.integers(0, 50, size=(2, 2))
+    T = 0.7
+    out = mod.verify(z, y, d, np.full((2, 2), 0.5), 1, T, mod.OCM(64, 0), 0.3)
+    from scipy.special import logsumexp, softmax
+    for b in range(2):
+        for i in range(2):
+            p, q = softmax(z[b, i] / T), softmax(y[b, i] / T)
+            assert out["alpha"][b, i] == pytest.approx(min(1.0, p[d[b, i]] / q[d[b, i]]), rel=1e-12)
+            assert out["lse_p"][b, i] == pytest.approx(logsumexp(z[b, i] / T), rel=1e-13)
+            assert out["lse_q"][b, i] == pytest.approx(logsumexp(y[b, i] / T), rel=1e-13)
+            assert out["accepted"][b, i] == (0.5 <= out["alpha"][b, i])
+            if not out["accepted"][b, i]:
+                t = out["t_star"][b, i]
+                assert p[t] > q[t]                                   # the residual lives where p exceeds q
+                assert out["score"][b, i] == pytest.approx(math.exp(z[b, i, d[b, i]] - z[b, i, t]), rel=1e-12)
+    for b in range(2):                                               # S3: draw (b, i) uses the clocks of row b*(K+1)+i
+        pk = softmax(z[b, 2] / T)
+        assert out["bonus"][b] == int(np.argmax(pk / mod.race_clocks(1, b * 3 + 2, 50)))
+        for i in range(2):
+            if not out["accepted"][b, i]:
+                w = np.maximum(0, softmax(z[b, i] / T) - softmax(y[b, i] / T))
+                assert out["t_star"][b, i] == int(np.argmax(w / mod.race_clocks(1, b * 3 + i, 50)))
+    # r == alpha passes ("r <= alpha")
+    a = out["alpha"][0, 0]
+    o2 = mod.verify(z, y, d, np.full((2, 2), a), 1, T, mod.OCM(64, 0), 0.3)
+    assert o2["accepted"][0, 0] and o2["near_accept"][0, 0]
+
+
+def pin_greedy_limit(mod):
+    """T -> 0 with a draft distribution concentrated on the draft token: Algorithm 1 becomes the
+    greedy loop (match <=> accept, t* = arg-max, bonus = arg-max)."""
+    rng = np.random.default_rng(11)
+    B, K, V = 6, 4, 40
+    z = rng.normal(size=(B, K + 1, V))
+    top = rng.integers(0, V, size=(B, K + 1))
+    for b in range(B):
+        for i in range(K + 1):
+            z[b, i, top[b, i]] = 6.0 + rng.random()
+    d = np.where(rng.random((B, K)) < 0.5, top[:, :K], rng.integers(0, V, size=(B, K)))
+    y = rng.normal(size=(B, K, V)) * 0.1
+    for b in range(B):
+        for i in range(K):
+            y[b, i, d[b, i]] = 8.0
+            if d[b, i] != top[b, i]:
+                z[b, i, d[b, i]] = 6.0 - 3 * rng.random()            # a plausible runner-up: ratio in (0.05, 1)
+    mem_s, mem_g = mod.OCM(256, 2), GREEDY.OCM(256, 2)
+    for _ in range(6):                                               # counts reach lambda on the way
+        r = rng.random((B, K)) * 0.9
+        s = mod.step(z, y, d, r, 3, 0.01, mem_s, 0.3)
+        g = GREEDY.step(z, d, mem_g, 0.3)
+        for k in ("accept_len", "next_token", "rescued_mask", "rej_draft", "rej_target"):
+            assert np.array_equal(s[k], g[k]), k
+    assert s["rescued_mask"].sum() > 0 and mem_s.table == mem_g.table
+
+
+def pin_gate_is_temperature_free_and_may_exceed_one(mod):
+    """Eq. 3: the gate compares raw logits whatever T is; against a SAMPLED t* the ratio can exceed 1."""
+    V = 5
+    z = np.zeros((1, 2, V)); z[0, 0] = [0.0, 2.0, 1.9, -1.0, -1.0]
+    y = np.zeros((1, 1, V)); y[0, 0] = [0.0, 6.0, -3.0, 0.0, 0.0]     # drafter far too sure of token 1
+    d = np.array([[1]])
+    seen = set()
+    for T in (0.5, 1.0, 2.0):
+        for seed in range(40):
+            mem = mod.OCM(64, 0)                                       # lambda = 0: the gate alone decides
+            o = mod.verify(z, y, d, np.array([[0.999]]), seed, T, mem, 0.95)
+            if o["accepted"][0, 0]:
+                continue
+            t = int(o["t_star"][0, 0])
+            assert t != 1                                              # residual is zero where q > p
+            ok = (z[0, 0, 1] - z[0, 0, t]) >= math.log(np.float32(0.95))
+            assert bool(o["rescued_mask"][0, 0]) == ok and (o["score"][0, 0] > 1.0) == (z[0, 0, t] < 2.0)
+            seen.add((t, bool(ok)))
+    assert any(ok for _, ok in seen)                                   # rescued with score > 1 at least once
+    # the gate is taken against the DRAWN t*, not against the arg-max: here the drafter covers the
+    # arg-max (token 0) and the draft token, so the residual sits on token 2, below the draft token
+    z[0, 0] = [3.0, 1.0, 0.5, -6.0, -6.0]
+    y[0, 0] = [3.6, 2.2, -5.0, -6.0, -6.0]
+    hits = 0
+    for seed in range(20):
+        o = mod.verify(z, y, d, np.array([[0.999]]), seed, 1.0, mod.OCM(64, 0), 0.3)
+        assert not o["accepted"][0, 0]
+        if o["t_star"][0, 0] == 2:
+            hits += 1
+            assert o["rescued_mask"][0, 0] == 1 and o["accept_len"][0] == 1      # 1.0 - 0.5 >= ln 0.3
+    assert hits >= 15
+
+
+def pin_update_semantics(mod):
+    """Every reached rejection is recorded, rescued or not; nothing after the stop; look-up before update."""
+    V = 4
+    z = np.zeros((1, 4, V)); y = np.zeros((1, 3, V))
+    z[0, :, 0] = 5.0                       # target wants token 0 everywhere
+    y[0, :, 1] = 5.0                       # drafter wants token 1
+    d = np.array([[1, 1, 1]])
+    r = np.array([[0.99, 0.99, 0.99]])     # alpha = p(1)/q(1) is tiny: all three fail the stochastic test
+    mem = mod.OCM(64, 2)
+    o = mod.step(z, y, d, r, 0, 1.0, mem, 0.0)
+    assert not o["accepted"].any() and np.all(o["t_star"][0] == 0)       # residual mass is on token 0
+    assert o["accept_len"][0] == 0 and o["next_token"][0] == 0
+    assert o["rej_draft"].tolist() == [[1, -1, -1]] and mem.table == {(1, 0): 1}
+    o = mod.step(z, y, d, r, 1, 1.0, mem, 0.0)
+    assert o["accept_len"][0] == 0 and mem.table == {(1, 0): 2}           # count 1 < lambda at look-up time
+    o = mod.step(z, y, d, r, 2, 1.0, mem, 0.0)                            # now 2 >= lambda, tau = 0: rescued
+    assert o["accept_len"][0] == 3 and o["rescued_mask"].tolist() == [[1, 1, 1]]
+    assert mem.table == {(1, 0): 5} and o["next_token"][0] == o["bonus"][0]
+    # tau = 1.5 can still pass when the drawn t* has a lower logit than the draft token; here it cannot
+    o = mod.verify(z, y, d, r, 3, 1.0, mem, 1.5)
+    assert o["accept_len"][0] == 0 and o["rej_draft"].tolist() == [[1, -1, -1]]
+    # bad draft id: rejection, not recorded, not rescued
+    o = mod.verify(z, y, np.array([[1, 9, 1]]), r, 3, 1.0, mem, 0.0)
+    assert o["accept_len"][0] == 1 and o["rej_draft"].tolist() == [[1, -1, -1]] and o["alpha"][0, 1] == 0
+
+
+def pin_unclear_draws_are_flagged(mod):
+    p = np.array([0.5, 0.5 * (1 + 2e-6), 0.0]); clocks = np.ones(3)
+    assert not mod.draw_is_clear(p, None, clocks, 1)
+    assert mod.draw_is_clear(np.array([0.2, 0.8, 0.0]), None, clocks, 1)
+    assert not mod.draw_is_clear(np.array([0.3, 0.5, 0.2]), np.array([0.299999, 0.1, 0.6]), np.array([1e-6, 1.0, 1.0]), 1)
+
+
+PINS = [pin_philox_known_answers, pin_alpha_and_normalisers, pin_update_semantics, pin_unclear_draws_are_flagged,
+        pin_gate_is_temperature_free_and_may_exceed_one, pin_greedy_limit, pin_clocks_are_exponential,
+        pin_race_draws_from_the_weights, pin_lossless_without_rescue]
+
+
+@pytest.mark.parametrize("pin", PINS, ids=[p.__name__ for p in PINS])
+def test_pin(pin):
+    pin(ORACLE)
+
+
+MUTANTS = [
+    ("philox multiplier", "0xD2511F53", "0xD2511F54"),
+    ("philox key schedule", "k0 = (k0 + _W0) & 0xFFFFFFFF", "k0 = (k0 + _W1) & 0xFFFFFFFF"),
+    ("philox output order", "(hi1 ^ c1 ^ np.uint64(k0)), lo1, (hi0 ^ c3 ^ np.uint64(k1)), lo0", "(hi0 ^ c1 ^ np.uint64(k0)), lo0, (hi1 ^ c3 ^ np.uint64(k1)), lo1"),
+    ("clock uses u not 1-u", "return -np.log1p(-u)", "return -np.log(u) * 0 + u"),
+    ("race divides the wrong way", "key = weights / clocks", "key = weights * clocks"),
+    ("race ties take the last", "int(np.flatnonzero(key == best)[0])", "int(np.flatnonzero(key == best)[-1])"),
+    ("residual sign", "np.maximum(0.0, p - q), clocks", "np.maximum(0.0, q - p), clocks"),
+    ("residual not clipped", "np.maximum(0.0, p - q), clocks", "np.abs(p - q), clocks"),
+    ("alpha inverted", "np.exp(lp[d] - lq[d])", "np.exp(lq[d] - lp[d])"),
+    ("acceptance reversed", "bool(r[b, i] <= alpha[b, i])", "bool(r[b, i] >= alpha[b, i])"),
+    ("temperature ignored for the draft", "lq, _, lse_q[b, i] = log_softmax_T(y[b, i], T)", "lq, _, lse_q[b, i] = log_softmax_T(y[b, i], 1.0)"),
+    ("temperature applied to the gate", "is_safe = bool((float(z[b, i, d]) - float(z[b, i, tt])) >= lf)", "is_safe = bool((float(z[b, i, d]) - float(z[b, i, tt])) / T >= lf)"),
+    ("gate against the arg-max", "float(z[b, i, d]) - float(z[b, i, tt])) >= lf", "float(z[b, i, d]) - float(np.max(z[b, i]))) >= lf"),
+    ("bonus from the wrong row", "next_token[b] = bonus[b] if n == K else t_star[b, n]", "next_token[b] = bonus[b] if n == K else t_star[b, 0]"),
+    ("update skipped for rescued", "            rej_d[b, i] = d\n            rej_t[b, i] = tt\n            if is_freq and is_safe:\n                rescued[b, i] = 1\n                continue",
+     "            if is_freq and is_safe:\n                rescued[b, i] = 1\n                continue\n            rej_d[b, i] = d\n            rej_t[b, i] = tt"),
+    ("frequency test strict", "is_freq = cnt[b, i] >= ocm.lam", "is_freq = cnt[b, i] > ocm.lam"),
+    ("bonus row shares the clocks of row 0", "row = b * K1 + i", "row = b * K1 + (0 if i == K else i)"),
+    ("normaliser without max shift", "lse = m + np.log(np.sum(np.exp(x - m)))", "lse = np.log(np.sum(np.exp(x - m)))"),
+]
+
+
+def _mutant(old, new):
+    path = ORACLE.__file__
+    src = open(path).read().replace("from .csd_oracle import", "from oracle.csd_oracle import")
+    assert src.count(old) >= 1, f"mutation anchor not found: {old[:40]!r}"
+    src = src.replace(old, new)
+    spec = importlib.util.spec_from_loader("csd_sampled_oracle_mutant", loader=None)
+    mod = importlib.util.module_from_spec(spec)
+    exec(compile(src, path + "<mutant>", "exec"), mod.__dict__)
+    return mod
+
+
+@pytest.mark.parametrize("name,old,new", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_planted_mistakes(name, old, new):
+    mod = _mutant(old, new)
+    caught = []
+    for pin in PINS:                       # cheap pins first; one that notices is enough
+        try:
+            pin(mod)
+        except Exception:
+            caught.append(pin.__name__)
+            break
+    assert caught, f"no pin notices the planted mistake: {name}"
