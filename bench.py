@@ -383,6 +383,110 @@ def run_ours(args, wl, tau):
         dist.destroy_process_group()
 
 
+# ---------------------------------------------------------------------------------------
+# --mode sampled: the stochastic verification step (Algorithm 1 at T > 0), a separate line
+# ---------------------------------------------------------------------------------------
+def run_sampled(args, wl, tau):
+    """csd_step_sampled (statistics, decision, races, finalisation, memory update: five
+    launches per step) over a ring of resident inputs.  Algorithmic bytes per step: every row of
+    the target and draft logits once, the two rows of every position that fails the acceptance
+    test once more, and the bonus rows once more."""
+    import torch
+
+    import paper_2604_13634_b200 as pkg
+    from paper_2604_13634_b200.synth import Synth
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    pkg.lib()
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    T = args.temperature
+    syn = Synth(wl, 0, device)
+    step_bytes = (wl.rows + wl.B * wl.K) * wl.V * wl.elt_bytes
+    l2 = torch.cuda.get_device_properties(device).L2_cache_size
+    ring_len = max(2, math.ceil(2 * l2 / step_bytes) + 1)
+    ring = [syn.step_sampled(s) for s in range(ring_len)]
+    ocm = pkg.Ocm(wl.ocm_slots, wl.lam, device.index)
+    kind, n = wl.prewarm
+    if kind == "pairs":
+        ocm.update(*syn.prewarm_pairs(n))
+    diag_buf = pkg.SampledBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, device=device, diag=True)
+    failed = []
+    for i, (z, y, d, r) in enumerate(ring):                 # also warms the memory up
+        pkg.csd_step_sampled(z, y, d, r, i, T, ocm, tau, diag_buf)
+        failed.append(int((diag_buf.diag["accepted"] == 0).sum().item()))
+    rows_per_step = wl.rows + wl.B * wl.K + 2 * (sum(failed) / len(failed)) + wl.B
+    algo_bytes = rows_per_step * wl.V * wl.elt_bytes
+    buf = pkg.SampledBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, device=device, diag=False)
+
+    def step(i):
+        z, y, d, r = ring[i % ring_len]
+        pkg.csd_step_sampled(z, y, d, r, 1000 + i % ring_len, T, ocm, tau, buf)
+
+    graph_steps = ring_len * max(1, math.ceil(args.graph_steps / ring_len))
+    side = torch.cuda.Stream(device)
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step(0)
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(graph_steps):
+            step(i)
+    steps = max(graph_steps, args.steps - args.steps % graph_steps)
+    for _ in range(max(1, math.ceil(max(args.warmup, 3) / graph_steps))):
+        g.replay()
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(device.index)
+    sampler.start()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps // graph_steps):
+        g.replay()
+    b.record()
+    b.synchronize()
+    clocks = sampler.stop()
+    sec = a.elapsed_time(b) * 1e-3
+    peak, peak_kind = measured_peak()
+    achieved = algo_bytes * steps / sec / 1e9
+    st = ocm.stats()
+    line = {"metric": METRIC, "value": wl.B * wl.K * steps / sec, "unit": UNIT, "n_gpus": 1, "steps": steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * sec / steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": workload_config(wl, tau, {
+                "mode": f"stochastic verification (Algorithm 1 at T={T}): acceptance test, residual and bonus draws",
+                "draft_logits": "target logits + N(0, 0.3^2), the draft token raised to the row maximum + 1",
+                "l2_policy": f"ring of {ring_len} distinct step inputs ({ring_len * step_bytes / 1e6:.0f} MB, > 2x L2)",
+                "launch": "CUDA graph of %d steps (5 launches each) replayed" % graph_steps,
+                "failed_positions_per_step": sum(failed) / len(failed)}),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_source": f"of {peak_kind}",
+                         "kernel": "sampled_stats_kernel + sampled_race_kernel (whole step)",
+                         "bytes_per_launch": algo_bytes},
+            "gpu_launches": 5 * steps, "clocks": clocks,
+            "ocm": {k: st[k] for k in ("n_keys", "n_dropped", "steps", "matches", "rescues", "rejections", "flags")}}
+    if not args.no_cpu_baseline:
+        import dataclasses
+        from oracle import csd_sampled_oracle as so
+        from paper_2604_13634_b200.synth import logits_to_numpy
+        rows_b = min(wl.B, 2)
+        small = dataclasses.replace(wl, B=rows_b)
+        z, y, d, r = Synth(small, 0, "cpu").step_sampled(0)
+        zz, yy = logits_to_numpy(z).astype("float64"), logits_to_numpy(y).astype("float64")
+        mem = so.OCM(wl.ocm_slots, wl.lam)
+        t0 = time.perf_counter()
+        n = 0
+        while time.perf_counter() - t0 < 10.0:
+            so.step(zz, yy, d.numpy(), r.numpy(), n, T, mem, tau)
+            n += 1
+        secs = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": rows_b * wl.K * n / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"{n} oracle steps over {rows_b} of the workload's {wl.B} batch rows in {secs:.1f} s"}
+    print(json.dumps(line), flush=True)
+    ocm.close()
+
+
 def run_extras(device, skip, peak):
     """Short device-resident runs of the other workloads (extra keys, not bench lines)."""
     import torch
@@ -426,6 +530,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--extras", action="store_true", help="also time the other workloads (extra keys, same line)")
+    ap.add_argument("--mode", default="greedy", choices=["greedy", "sampled"],
+                    help="sampled: the stochastic verification step (its own JSON line; 1 GPU)")
+    ap.add_argument("--temperature", type=float, default=0.3, help="T of --mode sampled")
     args = ap.parse_args()
 
     from paper_2604_13634_b200.synth import WORKLOADS
@@ -433,6 +540,8 @@ def main():
     tau = wl.taus[0] if args.tau is None else args.tau
     if args.impl == "reference":
         run_reference(args, wl, tau)
+    elif args.mode == "sampled":
+        run_sampled(args, wl, tau)
     else:
         run_ours(args, wl, tau)
 

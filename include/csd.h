@@ -221,6 +221,69 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
                                int32_t *rej_draft, int32_t *rej_target,
                                const csd_diag_t *diag, void *stream);
 
+/* ---- stochastic verification: Algorithm 1 as printed, temperature T > 0 ----------
+ *
+ * With p_i = softmax(z_i / T) (target) and q_i = softmax(y_i / T) (draft), for each row
+ * b and position i < K, in order:
+ *     alpha = min(1, p_i(d) / q_i(d));  the position passes iff r[b,i] <= alpha   (Eq. 2)
+ *     otherwise  t* ~ norm(max(0, p_i - q_i))        (the residual distribution, Sec. 3.1)
+ *                is_freq = T[(d, t*)] >= lambda      (candidate proposal, Sec. 4.2)
+ *                is_safe = z_i(d) - z_i(t*) >= ln tau  (Eq. 3: raw logits, whatever T is;
+ *                          against a drawn t* the ratio may exceed 1)
+ *                the pair (d, t*) is recorded for UpdateMemory; rescued iff is_freq and
+ *                is_safe, else the row stops here and emits t*
+ * accept_len[b] = positions passed or rescued before the stop; next_token[b] = t* of the
+ * stopping position, or a draw from p_K (the bonus token) when all K went through.
+ *
+ * The paper does not say how the draws are made; this library's reading:
+ *   - the uniforms r of the acceptance test are an INPUT ([B,K] float, in [0,1));
+ *   - a draw from weights w(v) is an exponential race, argmax_v w(v) / E_v (lowest index on
+ *     ties) with E_v = -ln(1 - u_v), u_v = (j + 1/2) / 2^23, j = the top 23 bits of word
+ *     (v & 3) of Philox4x32-10 (Salmon et al., SC'11) under key (seed low, seed high) and
+ *     counter (v >> 2, b*(K+1)+i, 0, 0); i = K is the bonus draw.  P(v) = w(v) / sum w.
+ * Every position that fails the acceptance test gets its t* (diag.t_star), reached or not.
+ * Look-ups see the memory as it is when the call starts; a draft id outside [0,V) fails
+ * the test, cannot be rescued and is not recorded.
+ *
+ * draft_logits: y[B, K, V], same dtype as logits, strides in elements, V contiguous.
+ * temperature > 0; tau as for csd_verify.  workspace: csd_sampled_workspace_bytes bytes,
+ * 16-byte aligned, no initialisation needed.  diag: NULL or a HOST struct of optional
+ * device arrays.  Four kernel launches (statistics, decision, races, finalisation);
+ * csd_step_sampled appends the memory update of the recorded pairs in (b,i) order.
+ * Errors as csd_verify; also INVALID_ARG for temperature <= 0 or NaN.  Asynchronous. */
+typedef struct {
+    float    *alpha;     /* [B,K]   min(1, p(d)/q(d))                                        */
+    uint8_t  *accepted;  /* [B,K]   1 where r <= alpha                                       */
+    int32_t  *t_star;    /* [B,K]   residual draw where the test failed, -1 where it passed  */
+    float    *lse_p;     /* [B,K+1] ln sum_v exp(z_v / T)                                    */
+    float    *lse_q;     /* [B,K]   ln sum_v exp(y_v / T)                                    */
+    float    *score;     /* [B,K]   exp(z_d - z_t*) where the test failed (NaN elsewhere)    */
+    uint32_t *cnt;       /* [B,K]   memory count of (d, t*) at the start of the step         */
+    int32_t  *bonus;     /* [B]     the draw from p_K                                        */
+} csd_sampled_diag_t;
+
+size_t csd_sampled_workspace_bytes(int B, int K, int V, csd_dtype_t dtype);
+
+csd_status_t csd_verify_sampled(const void *logits, const void *draft_logits, csd_dtype_t dtype,
+                                int B, int K, int V,
+                                int64_t stride_b, int64_t stride_k, int64_t draft_stride_b, int64_t draft_stride_k,
+                                const int32_t *draft, const float *r_accept, uint64_t seed, float temperature,
+                                const csd_ocm_t *ocm, float tau,
+                                int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                                int32_t *rej_draft, int32_t *rej_target,
+                                const csd_sampled_diag_t *diag,
+                                void *workspace, size_t workspace_bytes, void *stream);
+
+csd_status_t csd_step_sampled(const void *logits, const void *draft_logits, csd_dtype_t dtype,
+                              int B, int K, int V,
+                              int64_t stride_b, int64_t stride_k, int64_t draft_stride_b, int64_t draft_stride_k,
+                              const int32_t *draft, const float *r_accept, uint64_t seed, float temperature,
+                              csd_ocm_t *ocm, float tau,
+                              int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                              int32_t *rej_draft, int32_t *rej_target,
+                              const csd_sampled_diag_t *diag,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
 /* csd_step for callers whose tensors live in HOST memory (pinned memory gives
  * the full copy rate).  Copies logits and draft to `staging`, runs the step, and
  * copies accept_len, next_token and rescued_mask back; returns after the stream

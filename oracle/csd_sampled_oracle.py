@@ -24,8 +24,8 @@ Readings (the paper leaves these open; each is a convention of this build):
       and no second pass, and the integer it returns is well conditioned: it can only
       change when two keys nearly coincide.  (An inverse-CDF draw would make the index
       depend on rounding in a 150 000-term prefix sum.)
-  S3  E_v = -ln(1 - u_v), u_v = (j_v + 1/2) / 2^24, j_v = the top 24 bits of one
-      32-bit word of Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy
+  S3  E_v = -ln(1 - u_v), u_v = (j_v + 1/2) / 2^23, j_v = the top 23 bits of one
+      32-bit word (so that u_v and 1 - u_v are exact in binary32 as well) of Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy
       as 1, 2, 3", SC'11) with key = (seed low, seed high) and counter
       = (v >> 2, row, 0, 0), word v & 3, row = b * (K+1) + i (i = K: bonus draw).
   S4  look-ups see the memory as it was when the step began; rejections are added
@@ -82,8 +82,8 @@ def race_clocks(seed: int, row: int, V: int) -> np.ndarray:
     z = np.zeros(nblk, dtype=np.uint64)
     w = philox4x32_10(blk, z + np.uint64(row), z, z, seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
     words = np.stack(w, axis=1).reshape(-1)[:V]
-    j = (words >> np.uint64(8)).astype(np.float64)
-    u = (j + 0.5) / 16777216.0
+    j = (words >> np.uint64(9)).astype(np.float64)
+    u = (j + 0.5) / 8388608.0
     return -np.log1p(-u)
 
 

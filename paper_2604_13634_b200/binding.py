@@ -26,6 +26,7 @@ EXPORTS = [
     "csd_workspace_bytes", "csd_workspace_init", "csd_verify", "csd_ocm_update", "csd_step",
     "csd_host_staging_bytes", "csd_step_host", "csd_verify_static", "csd_ocm_export", "csd_ocm_import", "csd_ocm_stats",
     "csd_scg_threshold", "csd_launch_shape", "csd_set_tuning", "csd_set_overlap", "csd_status_string",
+    "csd_sampled_workspace_bytes", "csd_verify_sampled", "csd_step_sampled",
 ]
 
 
@@ -35,6 +36,10 @@ class CsdError(RuntimeError):
 
 class Diag(Structure):
     _fields_ = [(n, c_void_p) for n in ("m", "s", "lse", "t", "zd", "score", "p_d", "p_t", "cnt")]
+
+
+class SampledDiag(Structure):
+    _fields_ = [(n, c_void_p) for n in ("alpha", "accepted", "t_star", "lse_p", "lse_q", "score", "cnt", "bonus")]
 
 
 class Stats(Structure):
@@ -60,7 +65,13 @@ def lib():
     L = ctypes.CDLL(LIB_PATH)
     step_args = [c_void_p, c_int, c_int, c_int, c_int, c_int64, c_int64, c_void_p, c_void_p, c_float,
                  c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, POINTER(Diag), c_void_p, c_size_t, c_void_p]
+    sampled_args = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int64, c_int64, c_int64, c_int64, c_void_p, c_void_p,
+                    c_uint64, c_float, c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                    POINTER(SampledDiag), c_void_p, c_size_t, c_void_p]
     sigs = {
+        "csd_sampled_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int]),
+        "csd_verify_sampled": (c_int, sampled_args),
+        "csd_step_sampled": (c_int, sampled_args),
         "csd_ocm_create": (c_int, [POINTER(c_void_p), c_uint64, c_uint32, c_int]),
         "csd_ocm_reset": (c_int, [c_void_p, c_void_p]),
         "csd_ocm_destroy": (c_int, [c_void_p]),
@@ -298,3 +309,59 @@ def csd_verify_static(logits, draft, ocm: Ocm, tau: float, buf: StepBuffers, str
         _ptr(buf.rej_draft), _ptr(buf.rej_target),
         byref(buf._diag_struct) if buf._diag_struct is not None else None, _stream_ptr(stream))
     _check(rc, "csd_verify_static")
+
+
+class SampledBuffers:
+    """Caller-owned device buffers of one stochastic step shape: outputs, diagnostics, workspace."""
+
+    def __init__(self, B: int, K: int, V: int, dtype: torch.dtype, device="cuda", diag: bool = True):
+        self.B, self.K, self.V = B, K, V
+        self.dtype_code = CSD_F32 if dtype == torch.float32 else CSD_BF16
+        dev = torch.device(device)
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.accept_len = torch.empty(B, **i32)
+        self.next_token = torch.empty(B, **i32)
+        self.rescued_mask = torch.empty(B, K, dtype=torch.uint8, device=dev)
+        self.rej_draft = torch.empty(B, K, **i32)
+        self.rej_target = torch.empty(B, K, **i32)
+        self.ws_bytes = int(lib().csd_sampled_workspace_bytes(B, K, V, self.dtype_code))
+        if self.ws_bytes == 0:
+            raise CsdError(f"unsupported shape B={B} K={K} V={V}")
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
+        self.diag = None
+        self._diag_struct = None
+        if diag:
+            f = dict(dtype=torch.float32, device=dev)
+            self.diag = dict(alpha=torch.empty(B, K, **f), accepted=torch.empty(B, K, dtype=torch.uint8, device=dev),
+                             t_star=torch.empty(B, K, **i32), lse_p=torch.empty(B, K + 1, **f), lse_q=torch.empty(B, K, **f),
+                             score=torch.empty(B, K, **f), cnt=torch.empty(B, K, **i32), bonus=torch.empty(B, **i32))
+            self._diag_struct = SampledDiag(**{k: v.data_ptr() for k, v in self.diag.items()})
+
+
+def _sampled_call(fn_name, logits, draft_logits, draft, r_accept, seed, temperature, ocm: Ocm, tau, buf, stream):
+    assert logits.is_cuda and draft_logits.is_cuda and draft.is_cuda and r_accept.is_cuda
+    assert draft.dtype == torch.int32 and draft.is_contiguous() and r_accept.dtype == torch.float32 and r_accept.is_contiguous()
+    B, K1, V = logits.shape
+    assert (B, K1 - 1, V) == (buf.B, buf.K, buf.V) and tuple(draft_logits.shape) == (B, K1 - 1, V)
+    assert logits.stride(2) == 1 and draft_logits.stride(2) == 1 and draft_logits.dtype == logits.dtype
+    assert _dtype_code(logits) == buf.dtype_code and tuple(draft.shape) == (B, K1 - 1) == tuple(r_accept.shape)
+    rc = getattr(lib(), fn_name)(
+        logits.data_ptr(), draft_logits.data_ptr(), buf.dtype_code, B, K1 - 1, V, logits.stride(0), logits.stride(1),
+        draft_logits.stride(0), draft_logits.stride(1), draft.data_ptr(), r_accept.data_ptr(), c_uint64(seed),
+        c_float(temperature), ocm.handle, c_float(tau), _ptr(buf.accept_len), _ptr(buf.next_token),
+        _ptr(buf.rescued_mask), _ptr(buf.rej_draft), _ptr(buf.rej_target),
+        byref(buf._diag_struct) if buf._diag_struct is not None else None, _ptr(buf.workspace), buf.ws_bytes,
+        _stream_ptr(stream))
+    _check(rc, fn_name)
+
+
+def csd_verify_sampled(logits, draft_logits, draft, r_accept, seed: int, temperature: float, ocm: Ocm, tau: float,
+                       buf: SampledBuffers, stream=None):
+    """Algorithm 1 at temperature T > 0 (stochastic acceptance, residual draws); the memory is only read."""
+    _sampled_call("csd_verify_sampled", logits, draft_logits, draft, r_accept, seed, temperature, ocm, tau, buf, stream)
+
+
+def csd_step_sampled(logits, draft_logits, draft, r_accept, seed: int, temperature: float, ocm: Ocm, tau: float,
+                     buf: SampledBuffers, stream=None):
+    """csd_verify_sampled followed by the memory update with the step's recorded pairs."""
+    _sampled_call("csd_step_sampled", logits, draft_logits, draft, r_accept, seed, temperature, ocm, tau, buf, stream)

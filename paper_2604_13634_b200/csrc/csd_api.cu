@@ -10,6 +10,7 @@
 #include "csd_common.cuh"
 #include "csd_ocm.cuh"
 #include "csd_step.cuh"
+#include "csd_sampled.cuh"
 
 using namespace csd;
 
@@ -283,6 +284,120 @@ csd_status_t run_update(csd_ocm *ocm, const int32_t *d, const int32_t *t, const 
 
 }  // namespace
 
+// ---- stochastic verification (Algorithm 1 at T > 0) ----------------------------------------
+namespace {
+
+constexpr int kSampledChunkElems = 8192;   // elements of a row reduced by a warp at a time
+
+struct SampledLayout {
+    size_t stat_part, rownorm, alpha, accepted, race_part, total;
+    int nchunks;
+};
+
+SampledLayout sampled_layout(int B, int K, int V)
+{
+    SampledLayout w;
+    w.nchunks = (V + kSampledChunkElems - 1) / kSampledChunkElems;
+    const size_t rows = static_cast<size_t>(B) * (2 * K + 1);
+    const size_t draws = static_cast<size_t>(B) * (K + 1);
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    w.stat_part = take(rows * w.nchunks * sizeof(Partial));
+    w.rownorm = take(rows * sizeof(RowNorm));
+    w.alpha = take(static_cast<size_t>(B) * K * sizeof(float));
+    w.accepted = take(static_cast<size_t>(B) * K);
+    w.race_part = take(draws * w.nchunks * sizeof(RacePart));
+    w.total = off;
+    return w;
+}
+
+template <typename L>
+cudaError_t launch_sampled(const SampledParams &p, cudaStream_t st)
+{
+    const long long rows = static_cast<long long>(p.B) * (2 * p.K + 1);
+    const long long draws = static_cast<long long>(p.B) * (p.K + 1);
+    const long long cap = static_cast<long long>(sm_count()) * 4;
+    auto blocks_for = [&](long long tiles) {
+        long long b = (tiles + 7) / 8;            // 8 warps per block
+        return static_cast<unsigned int>(b < 1 ? 1 : (b > cap ? cap : b));
+    };
+    sampled_stats_kernel<L><<<blocks_for(rows * p.nchunks), 256, 0, st>>>(p);
+    sampled_decide_kernel<L><<<static_cast<unsigned int>((draws + 127) / 128), 128, 0, st>>>(p);
+    sampled_race_kernel<L><<<blocks_for(draws * p.nchunks), 256, 0, st>>>(p);
+    sampled_finalize_kernel<L><<<static_cast<unsigned int>((p.B + 3) / 4), 128, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+csd_status_t run_sampled(const void *logits, const void *draft_logits, csd_dtype_t dtype, int B, int K, int V,
+                         int64_t stride_b, int64_t stride_k, int64_t dstride_b, int64_t dstride_k, const int32_t *draft,
+                         const float *r_accept, uint64_t seed, float temperature, csd_ocm *ocm, float tau,
+                         int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask, int32_t *rej_draft,
+                         int32_t *rej_target, const csd_sampled_diag_t *diag, void *workspace, size_t workspace_bytes,
+                         void *stream, bool do_update)
+{
+    if (!logits || !draft_logits || !draft || !r_accept || !ocm || !accept_len || !next_token || !rescued_mask ||
+        !rej_draft || !rej_target || !workspace)
+        return CSD_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || V <= 0) return CSD_ERR_INVALID_ARG;
+    if (dtype != CSD_F32 && dtype != CSD_BF16) return CSD_ERR_INVALID_ARG;
+    if (K > CSD_MAX_K) return CSD_ERR_UNSUPPORTED;
+    if (!shape_ok(B, K, V, dtype) || static_cast<long long>(B) * (2 * K + 1) >= (1ll << 31)) return CSD_ERR_UNSUPPORTED;
+    if (!(tau >= 0.0f) || std::isinf(tau)) return CSD_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || std::isinf(temperature)) return CSD_ERR_INVALID_ARG;
+    if (stride_k < V || stride_b < stride_k * (K + 1) || dstride_k < V || dstride_b < dstride_k * K) return CSD_ERR_INVALID_ARG;
+    const SampledLayout w = sampled_layout(B, K, V);
+    if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
+    chain_break();
+
+    SampledParams p;
+    std::memset(&p, 0, sizeof p);
+    p.z = logits; p.y = draft_logits;
+    p.B = B; p.K = K; p.V = V;
+    p.z_sb = stride_b; p.z_sk = stride_k; p.y_sb = dstride_b; p.y_sk = dstride_k;
+    p.draft = draft; p.r = r_accept;
+    p.seed_lo = static_cast<unsigned int>(seed & 0xffffffffull);
+    p.seed_hi = static_cast<unsigned int>(seed >> 32);
+    p.l2e_T = static_cast<float>(1.4426950408889634 / static_cast<double>(temperature));
+    p.ocm = view_of(ocm);
+    p.log_tau = csd_scg_threshold(tau);
+    p.accept_len = accept_len; p.next_token = next_token; p.rescued = rescued_mask;
+    p.rej_d = rej_draft; p.rej_t = rej_target;
+    if (diag) p.diag = *diag;
+    char *ws = static_cast<char *>(workspace);
+    p.stat_part = reinterpret_cast<Partial *>(ws + w.stat_part);
+    p.rownorm = reinterpret_cast<RowNorm *>(ws + w.rownorm);
+    p.alpha = reinterpret_cast<float *>(ws + w.alpha);
+    p.accepted = reinterpret_cast<unsigned char *>(ws + w.accepted);
+    p.race_part = reinterpret_cast<RacePart *>(ws + w.race_part);
+    p.chunk_elems = kSampledChunkElems;
+    p.nchunks = w.nchunks;
+
+    const int eb = elt_bytes(dtype);
+    const int per_vec = 16 / eb;
+    auto aligned = [&](const void *base, int64_t sb, int64_t sk) {
+        return (reinterpret_cast<uintptr_t>(base) % 16 == 0) && (sb * eb) % 16 == 0 && (sk * eb) % 16 == 0;
+    };
+    const bool vec = aligned(logits, stride_b, stride_k) && aligned(draft_logits, dstride_b, dstride_k) && V % per_vec == 0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t err;
+    if (dtype == CSD_F32)
+        err = vec ? launch_sampled<LaneF32Vec>(p, st) : launch_sampled<LaneF32Scalar>(p, st);
+    else
+        err = vec ? launch_sampled<LaneBf16Vec>(p, st) : launch_sampled<LaneBf16Scalar>(p, st);
+    if (err != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    if (do_update) return run_update(ocm, rej_draft, rej_target, nullptr, static_cast<int64_t>(B) * K, stream);
+    return CSD_OK;
+}
+
+}  // namespace
+
 extern "C" {
 
 csd_status_t csd_ocm_create(csd_ocm_t **out, uint64_t n_slots, uint32_t lambda, int device)
@@ -478,6 +593,36 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
     }
     return run_step(logits, dtype, B, K, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
                     rej_draft, rej_target, diag, scratch, need, stream, false, false);
+}
+
+size_t csd_sampled_workspace_bytes(int B, int K, int V, csd_dtype_t dtype)
+{
+    if (!shape_ok(B, K, V, dtype)) return 0;
+    return sampled_layout(B, K, V).total;
+}
+
+csd_status_t csd_verify_sampled(const void *logits, const void *draft_logits, csd_dtype_t dtype, int B, int K, int V,
+                                int64_t stride_b, int64_t stride_k, int64_t draft_stride_b, int64_t draft_stride_k,
+                                const int32_t *draft, const float *r_accept, uint64_t seed, float temperature,
+                                const csd_ocm_t *ocm, float tau, int32_t *accept_len, int32_t *next_token,
+                                uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target,
+                                const csd_sampled_diag_t *diag, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return run_sampled(logits, draft_logits, dtype, B, K, V, stride_b, stride_k, draft_stride_b, draft_stride_k, draft,
+                       r_accept, seed, temperature, const_cast<csd_ocm_t *>(ocm), tau, accept_len, next_token,
+                       rescued_mask, rej_draft, rej_target, diag, workspace, workspace_bytes, stream, false);
+}
+
+csd_status_t csd_step_sampled(const void *logits, const void *draft_logits, csd_dtype_t dtype, int B, int K, int V,
+                              int64_t stride_b, int64_t stride_k, int64_t draft_stride_b, int64_t draft_stride_k,
+                              const int32_t *draft, const float *r_accept, uint64_t seed, float temperature,
+                              csd_ocm_t *ocm, float tau, int32_t *accept_len, int32_t *next_token,
+                              uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target,
+                              const csd_sampled_diag_t *diag, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return run_sampled(logits, draft_logits, dtype, B, K, V, stride_b, stride_k, draft_stride_b, draft_stride_k, draft,
+                       r_accept, seed, temperature, ocm, tau, accept_len, next_token, rescued_mask, rej_draft,
+                       rej_target, diag, workspace, workspace_bytes, stream, true);
 }
 
 size_t csd_host_staging_bytes(int B, int K, int V, csd_dtype_t dtype)

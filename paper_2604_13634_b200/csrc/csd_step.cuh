@@ -186,6 +186,10 @@ struct LaneF32Vec {
         accum_pair(__uint_as_float(a.x), __uint_as_float(a.y), l2e2, negc2, acc);
         accum_pair(__uint_as_float(a.z), __uint_as_float(a.w), l2e2, negc2, acc);
     }
+    static __device__ __forceinline__ void unpack(unit a, float (&f)[4])
+    {
+        f[0] = __uint_as_float(a.x); f[1] = __uint_as_float(a.y); f[2] = __uint_as_float(a.z); f[3] = __uint_as_float(a.w);
+    }
     static __device__ __forceinline__ int first_eq(unit a, float v)
     {
         if (__uint_as_float(a.x) == v) return 0;
@@ -233,6 +237,11 @@ struct LaneBf16Vec {
         accum_pair(lo(a.z), hi(a.z), l2e2, negc2, acc);
         accum_pair(lo(a.w), hi(a.w), l2e2, negc2, acc);
     }
+    static __device__ __forceinline__ void unpack(unit a, float (&f)[8])
+    {
+        f[0] = lo(a.x); f[1] = hi(a.x); f[2] = lo(a.y); f[3] = hi(a.y);
+        f[4] = lo(a.z); f[5] = hi(a.z); f[6] = lo(a.w); f[7] = hi(a.w);
+    }
     static __device__ __forceinline__ int first_eq(unit a, float v)
     {
         const unsigned int w[4] = {a.x, a.y, a.z, a.w};
@@ -261,6 +270,7 @@ struct LaneF32Scalar {
         // one element: the second half of the pair adds 2^(-inf) = 0
         accum_pair(a, -INFINITY, l2e2, negc2, acc);
     }
+    static __device__ __forceinline__ void unpack(unit a, float (&f)[1]) { f[0] = a; }
     static __device__ __forceinline__ int first_eq(unit a, float v) { return a == v ? 0 : -1; }
 };
 
@@ -283,13 +293,15 @@ struct LaneBf16Scalar {
         // one element: the second half of the pair adds 2^(-inf) = 0
         accum_pair(a, -INFINITY, l2e2, negc2, acc);
     }
+    static __device__ __forceinline__ void unpack(unit a, float (&f)[1]) { f[0] = a; }
     static __device__ __forceinline__ int first_eq(unit a, float v) { return a == v ? 0 : -1; }
 };
 
 // ---- S1: one warp reduces one tile ---------------------------------------------------
 
+// `l2e` = log2(e) / T: the sums are of 2^(x * l2e - c) = exp(x / T) up to the reference.
 template <typename L>
-__device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0, int e1, int lane)
+__device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0, int e1, int lane, const float l2e = kLog2e)
 {
     using U = typename L::unit;
     const typename L::elem *base = row + e0;
@@ -302,7 +314,7 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
     int it_thr = -1;           // iteration of the last strict improvement
     // four sums as two packed pairs: acc0 = (s0, s1), acc1 = (s2, s3)
     unsigned long long acc0 = pack2(0.f, 0.f), acc1 = acc0;
-    const unsigned long long l2e2 = pack2(kLog2e, kLog2e);
+    const unsigned long long l2e2 = pack2(l2e, l2e);
     U v[kUnroll];
 
     auto consume = [&](const U (&v)[kUnroll], int it) {
@@ -312,7 +324,7 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
         if (bmax > m_thr) {
             m_thr = bmax;
             it_thr = it;
-            const float cn = rintf(bmax * kLog2e);
+            const float cn = rintf(bmax * l2e);
             if (cn > c_thr) {
                 const float f = pow2_nonpos(c_thr - cn);
                 const unsigned long long f2 = pack2(f, f);
@@ -353,7 +365,7 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
     float wmax = m_thr;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) wmax = fmaxf(wmax, __shfl_xor_sync(kFull, wmax, o));
-    const float cw = (wmax == -INFINITY) ? kNoRef : rintf(wmax * kLog2e);
+    const float cw = (wmax == -INFINITY) ? kNoRef : rintf(wmax * l2e);
     float s = ((s0 + s1) + (s2 + s3)) * pow2_nonpos(c_thr - cw);
     int cand = 0x7fffffff;
     if (it_thr >= 0 && m_thr == wmax) {

@@ -173,6 +173,25 @@ class Synth:
         return z.contiguous(), draft.contiguous()
 
 
+    def step_sampled(self, step: int, draft_noise: float = 0.3, draft_margin: float = 1.0):
+        """Inputs of one STOCHASTIC step: (logits, draft_logits[B, K, V], draft, r[B, K] float32).
+
+        The target logits and draft tokens are those of `step`.  The draft model's logits are
+        the target's plus N(0, draft_noise^2) (a drafter that mostly agrees), except that at
+        every position the drafter's favourite is its own draft token: that logit is raised
+        to the row's maximum plus `draft_margin`.  r is uniform on [0, 1).
+        """
+        wl, dev = self.wl, self.device
+        z, draft = self.step(step)
+        g = self._gen(4, step)
+        y = z[:, :wl.K].to(torch.float32).clone()
+        y.add_(torch.randn(y.shape, generator=g, device=dev, dtype=torch.float32), alpha=draft_noise)
+        top = y.amax(dim=2, keepdim=True) + draft_margin
+        y.scatter_(2, draft.to(torch.int64).unsqueeze(-1), top)
+        r = torch.rand(wl.B, wl.K, generator=g, device=dev, dtype=torch.float32)
+        return z, y.to(wl.torch_dtype).contiguous(), draft, r.contiguous()
+
+
 def logits_to_numpy(z: torch.Tensor):
     """Exact host copy for the oracle: float32 array (bf16 widens exactly)."""
     return z.detach().to("cpu").to(torch.float32).numpy()

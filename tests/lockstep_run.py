@@ -32,11 +32,45 @@ from paper_2604_13634_b200.synth import WORKLOADS, Synth         # noqa: E402
 OVERLAP = False
 
 
-def run(wl, tau, steps, checkpoint, prewarm_steps, seed=0):
+def compare_memory(ocm, mem, dropped_before=0):
+    """Stored pairs, counts, number of keys and of dropped occurrences (a continued run's library
+    object counts its drops from the leg's start)."""
+    d, t, c = ocm.export()
+    rd, rt, rc = mem.export()
+    assert np.array_equal(d.numpy(), rd) and np.array_equal(t.numpy(), rt), "stored pairs differ"
+    assert np.array_equal(c.numpy(), rc), "counts differ"
+    st = ocm.stats()
+    assert st["n_keys"] == mem.n_keys and st["n_dropped"] + dropped_before == mem.n_dropped
+    return st
+
+
+def save_state(path, mem, next_step, totals):
+    d, t, c = mem.export()
+    np.savez(path, d=d, t=t, c=c, n_dropped=mem.n_dropped, next_step=next_step, totals=np.asarray(totals, dtype=np.int64))
+
+
+def load_state(path, ocm, mem):
+    """Continue a run: the oracle's memory comes from the file, the library's is loaded with the same
+    triples (the previous leg ended with the two compared equal)."""
+    st = np.load(path)
+    mem.table = {(int(a), int(b)): int(c) for a, b, c in zip(st["d"], st["t"], st["c"])}
+    mem.n_dropped = int(st["n_dropped"])
+    if len(st["d"]):
+        dev = ocm.device
+        ocm.import_(torch.tensor(st["d"], dtype=torch.int32, device=dev), torch.tensor(st["t"], dtype=torch.int32, device=dev),
+                    torch.tensor(st["c"], dtype=torch.int64, device=dev).to(torch.int32))
+    return int(st["next_step"]), [int(x) for x in st["totals"]]
+
+
+def run(wl, tau, steps, checkpoint, prewarm_steps, seed=0, first_step=None, load=None, save=None):
     syn = Synth(wl, seed, "cuda")
     ocm = Ocm(wl.ocm_slots, wl.lam)
     mem = ORACLE.OCM(wl.ocm_slots, wl.lam)
     kind, n = wl.prewarm
+    resumed = None
+    if load:
+        resumed = load_state(load, ocm, mem)
+        kind = "none"
     if kind == "pairs":
         pd, pt = syn.prewarm_pairs(n)
         ocm.update(pd, pt)
@@ -48,6 +82,12 @@ def run(wl, tau, steps, checkpoint, prewarm_steps, seed=0):
         first = -min(prewarm_steps, n)
     t0 = time.time()
     near = acc = resc = checked_diag = 0
+    dropped_before = 0
+    if resumed:
+        first, (near, acc, resc, checked_diag) = resumed
+        dropped_before = mem.n_dropped          # the library counts drops from this leg's start
+    if first_step is not None and not resumed:
+        first = first_step
     for s in range(first, steps):
         z, d = syn.step(s + 10 ** 6 if s < 0 else s)
         csd_step(z, d, ocm, tau, buf)
@@ -59,11 +99,14 @@ def run(wl, tau, steps, checkpoint, prewarm_steps, seed=0):
             acc += int(ref["accept_len"].sum())
             resc += int(ref["rescued_mask"].sum())
         if checkpoint and s >= 0 and (s + 1) % checkpoint == 0:
-            T.compare_memory(ocm, mem)
-    st = T.compare_memory(ocm, mem)
+            compare_memory(ocm, mem, dropped_before)
+    st = compare_memory(ocm, mem, dropped_before)
     assert st["flags"] == 0, st
+    if save:
+        save_state(save, mem, steps, (near, acc, resc, checked_diag))
     out = dict(workload=wl.name, tau=tau, steps=steps, prewarm_steps=-first, B=wl.B, K=wl.K, V=wl.V, dtype=wl.dtype,
-               accepted=acc, rescued=resc, acceptance_rate=acc / (steps * wl.B * wl.K), near_ties=near,
+               first_step_of_this_leg=first, accepted=acc, rescued=resc,
+               acceptance_rate=acc / (steps * wl.B * wl.K), near_ties=near,
                diag_steps_checked=checked_diag, n_keys=st["n_keys"], n_dropped=st["n_dropped"],
                checkpoints=(steps // checkpoint if checkpoint else 0), seconds=round(time.time() - t0, 1),
                overlap_launch_shape=bool(OVERLAP), verdict="identical")
@@ -78,6 +121,8 @@ def main():
     ap.add_argument("--checkpoint", type=int, default=0)
     ap.add_argument("--prewarm-steps", type=int, default=10 ** 9, help="cap on step-type pre-warming")
     ap.add_argument("--taus", default="")
+    ap.add_argument("--load", default="", help="continue from a state file written by --save")
+    ap.add_argument("--save", default="", help="write the memory and the running totals here at the end")
     ap.add_argument("--overlap", action="store_true",
                     help="the launch shape the benchmark times (csd_set_overlap: one block per SM and launch)")
     args = ap.parse_args()
@@ -89,7 +134,8 @@ def main():
     wl = WORKLOADS[args.workload]
     taus = [float(x) for x in args.taus.split(",")] if args.taus else list(wl.taus)
     for tau in taus:
-        res = run(wl, tau, args.steps or wl.steps, args.checkpoint or wl.checkpoint_every, args.prewarm_steps)
+        res = run(wl, tau, args.steps or wl.steps, args.checkpoint or wl.checkpoint_every, args.prewarm_steps,
+                  load=args.load or None, save=args.save or None)
         print(json.dumps(res), flush=True)
 
 

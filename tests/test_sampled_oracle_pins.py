@@ -38,8 +38,10 @@ def pin_clocks_are_exponential(mod):
     assert not np.array_equal(e[:100], mod.race_clocks(12345, 8, 100))                  # of (seed, row, v)
     assert not np.array_equal(e[:100], mod.race_clocks(12346, 7, 100))
     assert np.array_equal(e[:1001], mod.race_clocks(12345, 7, 1001))                    # prefix-stable in V
-    # the smallest and largest clock the 24-bit grid allows
-    assert e.min() >= -math.log1p(-0.5 / 2 ** 24) and e.max() <= -math.log(0.5 / 2 ** 24)
+    # the smallest and largest clock the 23-bit grid allows, and the grid itself
+    assert e.min() >= -math.log1p(-0.5 / 2 ** 23) and e.max() <= -math.log(0.5 / 2 ** 23)
+    u = -np.expm1(-e[:1000]) * 2 ** 23 - 0.5
+    assert np.allclose(u, np.round(u), atol=1e-6)
 
 
 def pin_race_draws_from_the_weights(mod):
