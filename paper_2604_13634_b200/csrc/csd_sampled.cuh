@@ -28,7 +28,7 @@ struct RowNorm {
     float m;        // max of the raw logits
     float lse2;     // log2 of sum_v 2^(x_v * log2(e)/T): the normaliser in base-2 units
     int argmax;     // lowest index attaining m
-    int pad;
+    float skip;     // target rows: weights up to this can never win the row's draw (see race_skip_bound)
 };
 
 struct __align__(8) RacePart {
@@ -98,6 +98,13 @@ __global__ void __launch_bounds__(256) sampled_stats_kernel(const __grid_constan
     }
 }
 
+// A weight that can never win a draw.  Clocks lie in [E_min, E_max] = [-ln(1 - 2^-24), -ln(2^-24)]
+// = [5.96e-8, 16.64].  If some token is known to have weight w0 > 0, the winning key is at least
+// w0 / E_max, and a token with weight w <= 3.0e-9 * w0 has key <= w / E_min <= 0.0503 * w0
+// < w0 / E_max = 0.0601 * w0: it loses whatever the clocks are (the 19 % margin dwarfs rounding).
+// The bound depends only on the row's statistics, so skipping by it changes no result bit.
+__device__ __forceinline__ float race_skip_bound(float w0) { return w0 > 0.0f ? 3.0e-9f * w0 : 0.0f; }
+
 // ---- A2: normalisers, alpha and the stochastic test, one thread per (b, i <= K) -----------
 
 __device__ __forceinline__ RowNorm fold_row_norm(const SampledParams &p, long long row)
@@ -112,7 +119,7 @@ __device__ __forceinline__ RowNorm fold_row_norm(const SampledParams &p, long lo
     n.m = acc.m;
     n.lse2 = acc.c + log2f(acc.s);
     n.argmax = acc.idx;
-    n.pad = 0;
+    n.skip = 0.0f;
     return n;
 }
 
@@ -126,15 +133,27 @@ __global__ void sampled_decide_kernel(const __grid_constant__ SampledParams p)
     const int K = p.K;
     const long long b = j / (K + 1);
     const int i = static_cast<int>(j - b * (K + 1));
-    const RowNorm np_ = fold_row_norm(p, j);
-    p.rownorm[j] = np_;
+    RowNorm np_ = fold_row_norm(p, j);
     if (!(np_.lse2 == np_.lse2) || np_.lse2 == INFINITY || np_.m == -INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
     if (p.diag.lse_p) p.diag.lse_p[j] = np_.lse2 * 0.6931471805599453f;
-    if (i == K) return;
+    // the probability of the row's arg-max: a weight known to take part in a draw from p
+    const float p_top = exp2f(static_cast<float>(static_cast<double>(np_.m) * static_cast<double>(p.l2e_T) - static_cast<double>(np_.lse2)));
+    if (i == K) {
+        np_.skip = race_skip_bound(p_top);
+        p.rownorm[j] = np_;
+        return;
+    }
     const long long pos = b * K + i;
     const long long yrow = n + pos;
     const RowNorm nq = fold_row_norm(p, yrow);
     p.rownorm[yrow] = nq;
+    {
+        // the residual weight p - q at the target's arg-max (if positive) takes part in the residual draw
+        const float y_top = L::load_elem(sampled_row_ptr<E>(p, yrow), np_.argmax);
+        const float q_top = exp2f(static_cast<float>(static_cast<double>(y_top) * static_cast<double>(p.l2e_T) - static_cast<double>(nq.lse2)));
+        np_.skip = race_skip_bound(0.99f * (p_top - q_top));     // 1 % off for the rounding of p_top - q_top
+        p.rownorm[j] = np_;
+    }
     if (!(nq.lse2 == nq.lse2) || nq.lse2 == INFINITY || nq.m == -INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
     if (p.diag.lse_q) p.diag.lse_q[pos] = nq.lse2 * 0.6931471805599453f;
     const int d = __ldg(p.draft + pos);
@@ -196,20 +215,31 @@ __device__ __forceinline__ void race_candidate(RaceBest &best, float w, unsigned
 // without a draft row (bonus draw) w = p.
 template <typename L, bool kHasQ>
 __device__ __forceinline__ void race_vector(RaceBest &best, typename L::unit zv, typename L::unit yv, int v0, float s, float mz, float lp,
-                                            float my, float lq, unsigned int row, unsigned int k0, unsigned int k1)
+                                            float my, float lq, float skip, unsigned int row, unsigned int k0, unsigned int k1)
 {
-    float zf[L::kPer], yf[L::kPer];
+    float zf[L::kPer], yf[L::kPer], w[L::kPer];
     L::unpack(zv, zf);
     if (kHasQ) L::unpack(yv, yf);
-    uint4 rnd = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
     for (int e = 0; e < L::kPer; ++e) {
-        const int v = v0 + e;
-        if (e == 0 || (v & 3) == 0) rnd = philox4x32_10(make_uint4(static_cast<unsigned int>(v) >> 2, row, 0u, 0u), k0, k1);
-        float w = exp2f(fmaf(zf[e] - mz, s, -lp));
-        if (kHasQ) w -= exp2f(fmaf(yf[e] - my, s, -lq));
-        const unsigned int word = (v & 3) == 0 ? rnd.x : (v & 3) == 1 ? rnd.y : (v & 3) == 2 ? rnd.z : rnd.w;
-        if (w > 0.0f) race_candidate(best, w, word, v);
+        w[e] = exp2f(fmaf(zf[e] - mz, s, -lp));
+        if (kHasQ) w[e] -= exp2f(fmaf(yf[e] - my, s, -lq));
+    }
+    // one Philox block serves four consecutive indices; it is computed only if one of them can win
+    constexpr int kGroup = L::kPer < 4 ? L::kPer : 4;
+#pragma unroll
+    for (int g0 = 0; g0 < L::kPer; g0 += kGroup) {
+        bool any = false;
+#pragma unroll
+        for (int e = g0; e < g0 + kGroup; ++e) any = any || (w[e] > skip);
+        if (!any) continue;
+        const uint4 rnd = philox4x32_10(make_uint4(static_cast<unsigned int>(v0 + g0) >> 2, row, 0u, 0u), k0, k1);
+#pragma unroll
+        for (int e = g0; e < g0 + kGroup; ++e) {
+            const int v = v0 + e;
+            const unsigned int word = (v & 3) == 0 ? rnd.x : (v & 3) == 1 ? rnd.y : (v & 3) == 2 ? rnd.z : rnd.w;
+            if (w[e] > skip) race_candidate(best, w[e], word, v);
+        }
     }
 }
 
@@ -252,10 +282,10 @@ __global__ void __launch_bounds__(256) sampled_race_kernel(const __grid_constant
             const int v0 = e0 + u * L::kPer;
             const U zv = L::load(zr + e0, u);
             if (bonus) {
-                race_vector<L, false>(best, zv, zv, v0, p.l2e_T, np_.m, lp, 0.0f, 0.0f, static_cast<unsigned int>(row), p.seed_lo, p.seed_hi);
+                race_vector<L, false>(best, zv, zv, v0, p.l2e_T, np_.m, lp, 0.0f, 0.0f, np_.skip, static_cast<unsigned int>(row), p.seed_lo, p.seed_hi);
             } else {
                 const U yv = L::load(yr + e0, u);
-                race_vector<L, true>(best, zv, yv, v0, p.l2e_T, np_.m, lp, my, lq, static_cast<unsigned int>(row), p.seed_lo, p.seed_hi);
+                race_vector<L, true>(best, zv, yv, v0, p.l2e_T, np_.m, lp, my, lq, np_.skip, static_cast<unsigned int>(row), p.seed_lo, p.seed_hi);
             }
         }
 #pragma unroll
