@@ -30,6 +30,25 @@ from paper_2604_13634_b200.synth import WORKLOADS, Synth         # noqa: E402
 
 
 OVERLAP = False
+_PINNED = {}
+
+
+def _bits_through_pinned_memory(z: torch.Tensor):
+    """Same result as synth.logits_bits_numpy, but the device-to-host copy lands in a pinned buffer
+    that is kept between steps (several times faster for the 100 MB+ steps of the long runs)."""
+    z = z.detach().contiguous()
+    key = (tuple(z.shape), z.dtype)
+    if key not in _PINNED:
+        _PINNED.clear()
+        _PINNED[key] = torch.empty(z.shape, dtype=z.dtype).pin_memory()
+    host = _PINNED[key]
+    host.copy_(z, non_blocking=False)
+    if z.dtype == torch.bfloat16:
+        return host.view(torch.int16).numpy().view("uint16"), True
+    return host.numpy(), False
+
+
+T.logits_bits_numpy = _bits_through_pinned_memory
 
 
 def compare_memory(ocm, mem, dropped_before=0):
