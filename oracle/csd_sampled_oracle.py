@@ -18,21 +18,28 @@ Algorithm 1 of the paper as it is printed, at temperature T > 0, one step, all f
 
 Readings (the paper leaves these open; each is a convention of this build):
   S1  the uniforms r are INPUTS (one per position).
-  S2  a categorical draw from non-negative weights w(v) is an exponential race: the
-      winner is argmax_v w(v) / E_v with independent E_v ~ Exp(1), lowest index on
-      ties; P(v wins) = w(v) / sum w exactly.  It needs no normaliser, no prefix sum
-      and no second pass, and the integer it returns is well conditioned: it can only
-      change when two keys nearly coincide.  (An inverse-CDF draw would make the index
-      depend on rounding in a 150 000-term prefix sum.)
-  S3  E_v = -ln(1 - u_v), u_v = (j_v + 1/2) / 2^23, j_v = the top 23 bits of one
-      32-bit word (so that u_v and 1 - u_v are exact in binary32 as well) of Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy
-      as 1, 2, 3", SC'11) with key = (seed low, seed high) and counter
-      = (v >> 2, row, 0, 0), word v & 3, row = b * (K+1) + i (i = K: bonus draw).
+  S2  a categorical draw from non-negative weights w(v) is an exponential race: among
+      items with weights W and independent clocks E ~ Exp(1) the winner is
+      argmax W / E, lowest index on ties; P(item wins) = W / sum W exactly.  It needs
+      no normaliser, no prefix sum and no second pass, and the integer it returns is
+      well conditioned: it can only change when two keys nearly coincide.  (An
+      inverse-CDF draw would make the index depend on rounding in a 150 000-term
+      prefix sum.)  The race is run in two levels: first among the groups of GROUP = 8
+      consecutive tokens (weight = the sum of the group), then among the tokens of
+      the winning group: P(v) = W_g / sum W * w(v) / W_g = w(v) / sum w.  One random
+      number per eight tokens is what makes the draw cheap.
+  S3  a clock is E = -ln(1 - u), u = (j + 1/2) / 2^23, j = the top 23 bits of one
+      32-bit word (so that u and 1 - u are exact in binary32 as well) of
+      Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy as 1, 2, 3",
+      SC'11) with key = (seed low, seed high).  Clock number n of stream s of draw
+      `row` is word n & 3 of counter (n >> 2, row, s, 0); group g uses clock g of
+      stream 0, token v uses clock v of stream 1; row = b * (K+1) + i (i = K: the
+      bonus draw).
   S4  look-ups see the memory as it was when the step began; rejections are added
       afterwards in (b, i) order (as in the greedy oracle).
   S5  near-ties are reported, not decided on: |r - alpha| < 1e-5 for the acceptance
-      test; for a draw, the winner is "clear" if it still wins after every p is scaled
-      by (1 -+ 1e-5) and every q by (1 +- 1e-5) against it.  A result that depends on a
+      test; for a draw, the winner (group, then token) is "clear" if it still wins
+      after every p is scaled by (1 -+ 1e-5) and every q by (1 +- 1e-5) against it.  A result that depends on a
       near-tie is excluded from exactness by the tests.
   S6  a draft id outside [0, V) is a rejection that cannot be rescued and is not
       recorded; its alpha is 0.  PARITY UNPINNED (paper silent).
@@ -75,13 +82,16 @@ def philox4x32_10(c0, c1, c2, c3, k0, k1):
     return c0, c1, c2, c3
 
 
-def race_clocks(seed: int, row: int, V: int) -> np.ndarray:
-    """E_v ~ Exp(1) for v in [0, V) of draw `row` (S3), float64."""
-    nblk = (V + 3) // 4
-    blk = np.arange(nblk, dtype=np.uint64)
-    z = np.zeros(nblk, dtype=np.uint64)
-    w = philox4x32_10(blk, z + np.uint64(row), z, z, seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
-    words = np.stack(w, axis=1).reshape(-1)[:V]
+GROUP = 8
+
+
+def race_clocks(seed: int, row: int, stream: int, first: int, n: int) -> np.ndarray:
+    """Clocks first .. first+n-1 of stream `stream` of draw `row` (S3), float64, ~ Exp(1)."""
+    idx = np.arange(first, first + n, dtype=np.uint64)
+    blk = idx >> np.uint64(2)
+    z = np.zeros(n, dtype=np.uint64)
+    w = philox4x32_10(blk, z + np.uint64(row), z + np.uint64(stream), z, seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
+    words = np.choose((idx & np.uint64(3)).astype(np.int64), w)
     j = (words >> np.uint64(9)).astype(np.float64)
     u = (j + 0.5) / 8388608.0
     return -np.log1p(-u)
@@ -107,12 +117,36 @@ def race(weights: np.ndarray, clocks: np.ndarray, fallback: int):
     return int(np.flatnonzero(key == best)[0]), float(best)
 
 
-def draw_is_clear(p, q, clocks, winner: int) -> bool:
-    """S5: the winner keeps winning under relative perturbations of BAND on p and q."""
-    lo = max(0.0, p[winner] * (1 - BAND) - (q[winner] * (1 + BAND) if q is not None else 0.0)) / clocks[winner]
-    hi = np.maximum(0.0, p * (1 + BAND) - (q * (1 - BAND) if q is not None else 0.0)) / clocks
-    hi[winner] = 0.0
-    return bool(lo > np.max(hi))
+def _weights(p, q, sp=1.0, sq=1.0):
+    return np.maximum(0.0, p * sp - (q * sq if q is not None else 0.0))
+
+
+def _by_group(w):
+    pad = (-len(w)) % GROUP
+    return np.concatenate([w, np.zeros(pad)]).reshape(-1, GROUP)
+
+
+def draw(p, q, seed: int, row: int, fallback: int):
+    """One draw from norm(max(0, p - q)) (q None: from p) by the two-level race (S2, S3).
+
+    Returns (token, clear): `clear` is False when the winning group or the winning token would
+    change under relative perturbations of BAND on p and q (S5)."""
+    w = _by_group(_weights(p, q))
+    n_groups = w.shape[0]
+    e_g = race_clocks(seed, row, 0, 0, n_groups)
+    g, best = race(w.sum(axis=1), e_g, -1)
+    if g < 0:                                                     # S7
+        return int(fallback), True
+    e_t = race_clocks(seed, row, 1, g * GROUP, GROUP)
+    t, _ = race(w[g], e_t, 0)
+    lo = _by_group(_weights(p, q, 1 - BAND, 1 + BAND))
+    hi = _by_group(_weights(p, q, 1 + BAND, 1 - BAND))
+    hi_g = hi.sum(axis=1) / e_g
+    hi_g[g] = 0.0
+    hi_t = hi[g] / e_t
+    hi_t[t] = 0.0
+    clear = lo[g].sum() / e_g[g] > np.max(hi_g) and lo[g, t] / e_t[t] > np.max(hi_t)
+    return g * GROUP + t, bool(clear)
 
 
 # ----------------------------------------------------------------------------
@@ -150,10 +184,8 @@ def verify(z, y, draft, r, seed: int, T: float, ocm: OCM, tau: float):
             lp, _, lse_p[b, i] = log_softmax_T(z[b, i], T)
             row = b * K1 + i
             if i == K:                                              # bonus draw t ~ p_{gamma+1}
-                clocks = race_clocks(seed, row, V)
-                p = np.exp(lp)
-                bonus[b], _ = race(p, clocks, int(np.argmax(as_f64(z[b, i]))))
-                unclear[b, i] = not draw_is_clear(p, None, clocks, int(bonus[b]))
+                bonus[b], clear = draw(np.exp(lp), None, seed, row, int(np.argmax(as_f64(z[b, i]))))
+                unclear[b, i] = not clear
                 continue
             lq, _, lse_q[b, i] = log_softmax_T(y[b, i], T)
             d = int(draft[b, i])
@@ -163,10 +195,8 @@ def verify(z, y, draft, r, seed: int, T: float, ocm: OCM, tau: float):
             near_accept[b, i] = abs(r[b, i] - alpha[b, i]) < BAND
             if accepted[b, i]:
                 continue
-            p, q = np.exp(lp), np.exp(lq)
-            clocks = race_clocks(seed, row, V)
-            t_star[b, i], _ = race(np.maximum(0.0, p - q), clocks, int(np.argmax(as_f64(z[b, i]))))
-            unclear[b, i] = not draw_is_clear(p, q, clocks, int(t_star[b, i]))
+            t_star[b, i], clear = draw(np.exp(lp), np.exp(lq), seed, row, int(np.argmax(as_f64(z[b, i]))))   # residual
+            unclear[b, i] = not clear
             if 0 <= d < V:
                 score[b, i] = np.exp(float(z[b, i, d]) - float(z[b, i, t_star[b, i]]))
                 cnt[b, i] = ocm.count(d, t_star[b, i])

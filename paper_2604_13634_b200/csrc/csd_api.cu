@@ -287,17 +287,29 @@ csd_status_t run_update(csd_ocm *ocm, const int32_t *d, const int32_t *t, const 
 // ---- stochastic verification (Algorithm 1 at T > 0) ----------------------------------------
 namespace {
 
-constexpr int kSampledChunkElems = 8192;   // elements of a row reduced by a warp at a time
+constexpr int kSampledChunkMax = 8192;   // most elements of a row reduced by a warp at a time
+constexpr int kSampledChunkMin = 2048;   // least (one unrolled iteration of a warp of bf16 vectors)
+
+// Elements per tile: as large as possible while the step still has a few tiles per resident warp.
+int sampled_chunk_elems(int B, int K, int V)
+{
+    const long long rows = static_cast<long long>(B) * (2 * K + 1);
+    const long long want = static_cast<long long>(sm_count()) * 32 * 2;
+    int chunk = kSampledChunkMax;
+    while (chunk > kSampledChunkMin && rows * ((V + chunk - 1) / chunk) < want) chunk /= 2;
+    return chunk;
+}
 
 struct SampledLayout {
     size_t stat_part, rownorm, alpha, accepted, race_part, total;
-    int nchunks;
+    int nchunks, chunk_elems;
 };
 
 SampledLayout sampled_layout(int B, int K, int V)
 {
     SampledLayout w;
-    w.nchunks = (V + kSampledChunkElems - 1) / kSampledChunkElems;
+    w.chunk_elems = sampled_chunk_elems(B, K, V);
+    w.nchunks = (V + w.chunk_elems - 1) / w.chunk_elems;
     const size_t rows = static_cast<size_t>(B) * (2 * K + 1);
     const size_t draws = static_cast<size_t>(B) * (K + 1);
     size_t off = 0;
@@ -326,7 +338,7 @@ cudaError_t launch_sampled(const SampledParams &p, cudaStream_t st)
         return static_cast<unsigned int>(b < 1 ? 1 : (b > cap ? cap : b));
     };
     sampled_stats_kernel<L><<<blocks_for(rows * p.nchunks), 256, 0, st>>>(p);
-    sampled_decide_kernel<L><<<static_cast<unsigned int>((draws + 127) / 128), 128, 0, st>>>(p);
+    sampled_decide_kernel<L><<<static_cast<unsigned int>((draws + 3) / 4), 128, 0, st>>>(p);
     sampled_race_kernel<L><<<blocks_for(draws * p.nchunks), 256, 0, st>>>(p);
     sampled_finalize_kernel<L><<<static_cast<unsigned int>((p.B + 3) / 4), 128, 0, st>>>(p);
     return cudaGetLastError();
@@ -373,7 +385,7 @@ csd_status_t run_sampled(const void *logits, const void *draft_logits, csd_dtype
     p.alpha = reinterpret_cast<float *>(ws + w.alpha);
     p.accepted = reinterpret_cast<unsigned char *>(ws + w.accepted);
     p.race_part = reinterpret_cast<RacePart *>(ws + w.race_part);
-    p.chunk_elems = kSampledChunkElems;
+    p.chunk_elems = w.chunk_elems;
     p.nchunks = w.nchunks;
 
     const int eb = elt_bytes(dtype);

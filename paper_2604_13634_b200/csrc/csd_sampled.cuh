@@ -28,7 +28,8 @@ struct RowNorm {
     float m;        // max of the raw logits
     float lse2;     // log2 of sum_v 2^(x_v * log2(e)/T): the normaliser in base-2 units
     int argmax;     // lowest index attaining m
-    float skip;     // target rows: weights up to this can never win the row's draw (see race_skip_bound)
+    float zcut;     // target rows: a token whose logit is below this can never win the row's draw
+                    // (see race_skip_bound); -inf if no bound is known
 };
 
 struct __align__(8) RacePart {
@@ -100,58 +101,73 @@ __global__ void __launch_bounds__(256) sampled_stats_kernel(const __grid_constan
 
 // A weight that can never win a draw.  Clocks lie in [E_min, E_max] = [-ln(1 - 2^-24), -ln(2^-24)]
 // = [5.96e-8, 16.64].  If some token is known to have weight w0 > 0, the winning key is at least
-// w0 / E_max, and a token with weight w <= 3.0e-9 * w0 has key <= w / E_min <= 0.0503 * w0
-// < w0 / E_max = 0.0601 * w0: it loses whatever the clocks are (the 19 % margin dwarfs rounding).
-// The bound depends only on the row's statistics, so skipping by it changes no result bit.
-__device__ __forceinline__ float race_skip_bound(float w0) { return w0 > 0.0f ? 3.0e-9f * w0 : 0.0f; }
+// w0 / E_max (its group weighs at least w0), and a group of eight tokens that each weigh
+// w <= 3.7e-10 * w0 has key <= 8 w / E_min <= 0.0497 * w0 < w0 / E_max = 0.0601 * w0: it loses
+// whatever the clocks are (the 20 % margin dwarfs rounding).  The bound depends only on the row's
+// statistics, so skipping by it changes no result bit.
+__device__ __forceinline__ float race_skip_bound(float w0) { return w0 > 0.0f ? 3.7e-10f * w0 : 0.0f; }
 
-// ---- A2: normalisers, alpha and the stochastic test, one thread per (b, i <= K) -----------
+// ---- A2: normalisers, alpha and the stochastic test, one warp per (b, i <= K) --------------
 
-__device__ __forceinline__ RowNorm fold_row_norm(const SampledParams &p, long long row)
+// All lanes return the row's statistics.  Lane k pre-folds chunks k, k+32, ... in order, then a
+// fixed-shape butterfly: the result does not depend on timing.
+__device__ __forceinline__ RowNorm fold_row_norm(const SampledParams &p, long long row, int lane)
 {
     Partial acc = partial_identity();
-    for (int c = 0; c < p.nchunks; ++c) {
-        Partial x = ld_partial_cg(p.stat_part + row * p.nchunks + c);
-        // partials carry c = rint(m * log2(e)/T) of their own chunk; combine() rescales exactly
-        acc = (c == 0) ? x : combine(acc, x);
+    for (int c = lane; c < p.nchunks; c += 32) {
+        const Partial x = ld_partial_cg(p.stat_part + row * p.nchunks + c);
+        acc = (c == lane) ? x : combine(acc, x);
     }
+    acc = butterfly_fold(acc, 32, p.l2e_T);
     RowNorm n;
     n.m = acc.m;
     n.lse2 = acc.c + log2f(acc.s);
     n.argmax = acc.idx;
-    n.skip = 0.0f;
+    n.zcut = -INFINITY;
     return n;
 }
 
+// The logit below which p(v) <= race_skip_bound(w0): (z - m) * l2e_T - (lse2 - m * l2e_T) <= log2(bound),
+// lowered by 1e-3 so that rounding can only make the cut more cautious.
+__device__ __forceinline__ float race_logit_cut(const RowNorm &n, float w0, float l2e_T)
+{
+    const float bound = race_skip_bound(w0);
+    if (!(bound > 0.0f)) return -INFINITY;
+    return static_cast<float>((static_cast<double>(n.lse2) + log2(static_cast<double>(bound))) / static_cast<double>(l2e_T) - 1e-3);
+}
+
 template <typename L>
-__global__ void sampled_decide_kernel(const __grid_constant__ SampledParams p)
+__global__ void __launch_bounds__(128) sampled_decide_kernel(const __grid_constant__ SampledParams p)
 {
     using E = typename L::elem;
+    const int lane = threadIdx.x & 31;
     const long long n = sampled_rows_z(p);
-    const long long j = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const long long j = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (j >= n) return;
     const int K = p.K;
     const long long b = j / (K + 1);
     const int i = static_cast<int>(j - b * (K + 1));
-    RowNorm np_ = fold_row_norm(p, j);
+    RowNorm np_ = fold_row_norm(p, j, lane);
+    RowNorm nq = np_;
+    const long long pos = b * K + i;
+    const long long yrow = n + pos;
+    if (i < K) nq = fold_row_norm(p, yrow, lane);
+    if (lane != 0) return;
     if (!(np_.lse2 == np_.lse2) || np_.lse2 == INFINITY || np_.m == -INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
     if (p.diag.lse_p) p.diag.lse_p[j] = np_.lse2 * 0.6931471805599453f;
     // the probability of the row's arg-max: a weight known to take part in a draw from p
     const float p_top = exp2f(static_cast<float>(static_cast<double>(np_.m) * static_cast<double>(p.l2e_T) - static_cast<double>(np_.lse2)));
     if (i == K) {
-        np_.skip = race_skip_bound(p_top);
+        np_.zcut = race_logit_cut(np_, p_top, p.l2e_T);
         p.rownorm[j] = np_;
         return;
     }
-    const long long pos = b * K + i;
-    const long long yrow = n + pos;
-    const RowNorm nq = fold_row_norm(p, yrow);
     p.rownorm[yrow] = nq;
     {
         // the residual weight p - q at the target's arg-max (if positive) takes part in the residual draw
         const float y_top = L::load_elem(sampled_row_ptr<E>(p, yrow), np_.argmax);
         const float q_top = exp2f(static_cast<float>(static_cast<double>(y_top) * static_cast<double>(p.l2e_T) - static_cast<double>(nq.lse2)));
-        np_.skip = race_skip_bound(0.99f * (p_top - q_top));     // 1 % off for the rounding of p_top - q_top
+        np_.zcut = race_logit_cut(np_, 0.99f * (p_top - q_top), p.l2e_T);     // 1 % off for the rounding of p_top - q_top
         p.rownorm[j] = np_;
     }
     if (!(nq.lse2 == nq.lse2) || nq.lse2 == INFINITY || nq.m == -INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
@@ -177,6 +193,13 @@ __global__ void sampled_decide_kernel(const __grid_constant__ SampledParams p)
 }
 
 // ---- B: exponential races --------------------------------------------------------------------
+//
+// Two levels.  First among the groups of 8 consecutive tokens, weight W_g = sum of the group's
+// weights, clock number g of stream 0: this is what kernel B streams for.  Then among the 8
+// tokens of the winning group, clock number v of stream 1: eight gathers in kernel C.
+// P(v) = W_g / sum W * w(v) / W_g = w(v) / sum w, with one random number per eight tokens.
+
+constexpr int kRaceGroup = 8;
 
 __device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned int k0, unsigned int k1)
 {
@@ -191,63 +214,146 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned int k0, unsigne
     return c;
 }
 
+__device__ __forceinline__ unsigned int philox_word(const uint4 &r, unsigned int n)
+{
+    return (n & 3u) == 0u ? r.x : (n & 3u) == 1u ? r.y : (n & 3u) == 2u ? r.z : r.w;
+}
+
+// u = (j + 1/2) / 2^23 from the top 23 bits of a word: exact in binary32, and so is 1 - u.
+__device__ __forceinline__ float clock_u(unsigned int word) { return (static_cast<float>(word >> 9) + 0.5f) * 1.1920928955078125e-07f; }
+__device__ __forceinline__ float clock_of(float u) { return -log1pf(-u); }      // E = -ln(1 - u) ~ Exp(1)
+
+// What a draw needs of its two rows.  Weights are w(v) = max(0, 2^((z-mz)*s - lp) - 2^((y-my)*s - lq))
+// with lp = Lp - mz*s: the row maxima are taken out first so that the exponents of the tokens
+// that matter are small and exact; a bonus draw has no draft row and w = p.
+struct DrawCoef {
+    float s, mz, lp, my, lq, zcut;
+    bool has_q;
+};
+
+__device__ __forceinline__ DrawCoef draw_coef(const SampledParams &p, long long row, bool bonus, long long yrow)
+{
+    DrawCoef c;
+    const RowNorm np_ = p.rownorm[row];
+    c.s = p.l2e_T;
+    c.mz = np_.m;
+    c.lp = static_cast<float>(static_cast<double>(np_.lse2) - static_cast<double>(np_.m) * static_cast<double>(p.l2e_T));
+    c.zcut = np_.zcut;
+    c.has_q = !bonus;
+    c.my = 0.0f;
+    c.lq = 0.0f;
+    if (!bonus) {
+        const RowNorm nq = p.rownorm[yrow];
+        c.my = nq.m;
+        c.lq = static_cast<float>(static_cast<double>(nq.lse2) - static_cast<double>(nq.m) * static_cast<double>(p.l2e_T));
+    }
+    return c;
+}
+
+__device__ __forceinline__ float draw_weight(const DrawCoef &c, float z, float y)
+{
+    float w = ex2_approx(fmaf(z - c.mz, c.s, -c.lp));
+    if (c.has_q) w -= ex2_approx(fmaf(y - c.my, c.s, -c.lq));
+    return fmaxf(w, 0.0f);
+}
+
+// Sum of a group's weights, in a fixed order.
+__device__ __forceinline__ float group_weight(const DrawCoef &c, const float (&z)[8], const float (&y)[8])
+{
+    float w[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) w[e] = draw_weight(c, z[e], y[e]);
+    return ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
+}
+
 struct RaceBest {
     float key;
     int idx;
 };
 
-// One candidate: weight w > 0 at index v with random word `word`.  u = (j + 1/2) / 2^23 is
-// exact in binary32; E = -ln(1 - u) >= u, so a candidate with w <= best * u cannot win and
-// the logarithm is skipped for it.
-__device__ __forceinline__ void race_candidate(RaceBest &best, float w, unsigned int word, int v)
-{
-    const float u = (static_cast<float>(word >> 9) + 0.5f) * 1.1920928955078125e-07f;
-    if (!(w > best.key * u)) return;
-    const float key = w / (-log1pf(-u));
-    if (key > best.key) {       // indices ascend within a lane: strict keeps the lowest
-        best.key = key;
-        best.idx = v;
-    }
-}
+// Eight consecutive tokens of a row starting at v0 (a multiple of 8); tokens at or beyond V read
+// as -inf (weight 0).  The vector forms need the row 16-byte aligned.
+template <typename L>
+struct Group8;
 
-// w(v) = max(0, 2^((z-mz)*s - lp) - 2^((y-my)*s - lq)), lp = Lp - mz*s: the row maxima are
-// taken out first so that the exponents of the tokens that matter are small and exact;
-// without a draft row (bonus draw) w = p.
-template <typename L, bool kHasQ>
-__device__ __forceinline__ void race_vector(RaceBest &best, typename L::unit zv, typename L::unit yv, int v0, float s, float mz, float lp,
-                                            float my, float lq, float skip, unsigned int row, unsigned int k0, unsigned int k1)
-{
-    float zf[L::kPer], yf[L::kPer], w[L::kPer];
-    L::unpack(zv, zf);
-    if (kHasQ) L::unpack(yv, yf);
-#pragma unroll
-    for (int e = 0; e < L::kPer; ++e) {
-        w[e] = exp2f(fmaf(zf[e] - mz, s, -lp));
-        if (kHasQ) w[e] -= exp2f(fmaf(yf[e] - my, s, -lq));
+template <>
+struct Group8<LaneBf16Vec> {
+    static constexpr int kVec = 1;
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *row, int v0, int V, uint4 (&raw)[1]) { raw[0] = ld_stream16(row + v0); }
+    static __device__ __forceinline__ float hmax(const uint4 (&raw)[1]) { return LaneBf16Vec::hmax(raw[0]); }
+    static __device__ __forceinline__ void unpack(const uint4 (&raw)[1], float (&f)[8]) { LaneBf16Vec::unpack(raw[0], f); }
+};
+
+template <>
+struct Group8<LaneF32Vec> {
+    static constexpr int kVec = 2;
+    static __device__ __forceinline__ void load(const float *row, int v0, int V, uint4 (&raw)[2])
+    {
+        raw[0] = ld_stream16(row + v0);
+        raw[1] = v0 + 4 < V ? ld_stream16(row + v0 + 4) : LaneF32Vec::neg_inf();      // V is a multiple of 4 here
     }
-    // one Philox block serves four consecutive indices; it is computed only if one of them can win
-    constexpr int kGroup = L::kPer < 4 ? L::kPer : 4;
+    static __device__ __forceinline__ float hmax(const uint4 (&raw)[2]) { return fmaxf(LaneF32Vec::hmax(raw[0]), LaneF32Vec::hmax(raw[1])); }
+    static __device__ __forceinline__ void unpack(const uint4 (&raw)[2], float (&f)[8])
+    {
+        float a[4], b[4];
+        LaneF32Vec::unpack(raw[0], a);
+        LaneF32Vec::unpack(raw[1], b);
 #pragma unroll
-    for (int g0 = 0; g0 < L::kPer; g0 += kGroup) {
-        bool any = false;
-#pragma unroll
-        for (int e = g0; e < g0 + kGroup; ++e) any = any || (w[e] > skip);
-        if (!any) continue;
-        const uint4 rnd = philox4x32_10(make_uint4(static_cast<unsigned int>(v0 + g0) >> 2, row, 0u, 0u), k0, k1);
-#pragma unroll
-        for (int e = g0; e < g0 + kGroup; ++e) {
-            const int v = v0 + e;
-            const unsigned int word = (v & 3) == 0 ? rnd.x : (v & 3) == 1 ? rnd.y : (v & 3) == 2 ? rnd.z : rnd.w;
-            if (w[e] > skip) race_candidate(best, w[e], word, v);
+        for (int e = 0; e < 4; ++e) {
+            f[e] = a[e];
+            f[4 + e] = b[e];
         }
     }
-}
+};
+
+template <typename L>
+struct Group8Scalar {
+    static constexpr int kVec = 8;
+    using E = typename L::elem;
+    static __device__ __forceinline__ void load(const E *row, int v0, int V, float (&raw)[8])
+    {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) raw[e] = v0 + e < V ? L::load_elem(row, v0 + e) : -INFINITY;
+    }
+    static __device__ __forceinline__ float hmax(const float (&raw)[8])
+    {
+        float m = raw[0];
+#pragma unroll
+        for (int e = 1; e < 8; ++e) m = fmaxf(m, raw[e]);
+        return m;
+    }
+    static __device__ __forceinline__ void unpack(const float (&raw)[8], float (&f)[8])
+    {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = raw[e];
+    }
+};
+
+template <>
+struct Group8<LaneF32Scalar> : Group8Scalar<LaneF32Scalar> {};
+template <>
+struct Group8<LaneBf16Scalar> : Group8Scalar<LaneBf16Scalar> {};
+
+template <typename L>
+struct Group8Raw {
+    using type = uint4;
+};
+template <>
+struct Group8Raw<LaneF32Scalar> {
+    using type = float;
+};
+template <>
+struct Group8Raw<LaneBf16Scalar> {
+    using type = float;
+};
 
 template <typename L>
 __global__ void __launch_bounds__(256) sampled_race_kernel(const __grid_constant__ SampledParams p)
 {
     using E = typename L::elem;
-    using U = typename L::unit;
+    using G = Group8<L>;
+    using Raw = typename Group8Raw<L>::type;
+    constexpr int kGroups = G::kVec == 1 ? 4 : G::kVec == 2 ? 2 : 1;      // groups a lane has in flight (8 vectors)
     const int lane = threadIdx.x & 31;
     const int K = p.K;
     const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
@@ -260,32 +366,57 @@ __global__ void __launch_bounds__(256) sampled_race_kernel(const __grid_constant
         const int i = static_cast<int>(row - b * (K + 1));
         const bool bonus = i == K;
         if (!bonus && p.accepted[b * K + i]) continue;       // passed the stochastic test: no draw
-        const RowNorm np_ = p.rownorm[row];
-        const float lp = static_cast<float>(static_cast<double>(np_.lse2) - static_cast<double>(np_.m) * static_cast<double>(p.l2e_T));
-        float lq = 0.0f, my = 0.0f;
+        const long long yrow = draws + b * K + i;
+        const DrawCoef cf = draw_coef(p, row, bonus, yrow);
         const E *zr = sampled_row_ptr<E>(p, row);
-        const E *yr = zr;
-        if (!bonus) {
-            const long long yrow = draws + b * K + i;
-            const RowNorm nq = p.rownorm[yrow];
-            my = nq.m;
-            lq = static_cast<float>(static_cast<double>(nq.lse2) - static_cast<double>(nq.m) * static_cast<double>(p.l2e_T));
-            yr = sampled_row_ptr<E>(p, yrow);
-        }
-        const int e0 = c * p.chunk_elems;
-        const int e1 = min(p.V, e0 + p.chunk_elems);
-        const int nunits = (e1 - e0) / L::kPer;
+        const E *yr = bonus ? zr : sampled_row_ptr<E>(p, yrow);
+        const int g0 = c * (p.chunk_elems / kRaceGroup);
+        const int g1 = min((p.V + kRaceGroup - 1) / kRaceGroup, g0 + p.chunk_elems / kRaceGroup);
         RaceBest best;
         best.key = 0.0f;
         best.idx = 0x7fffffff;
-        for (int u = lane; u < nunits; u += 32) {
-            const int v0 = e0 + u * L::kPer;
-            const U zv = L::load(zr + e0, u);
-            if (bonus) {
-                race_vector<L, false>(best, zv, zv, v0, p.l2e_T, np_.m, lp, 0.0f, 0.0f, np_.skip, static_cast<unsigned int>(row), p.seed_lo, p.seed_hi);
-            } else {
-                const U yv = L::load(yr + e0, u);
-                race_vector<L, true>(best, zv, yv, v0, p.l2e_T, np_.m, lp, my, lq, np_.skip, static_cast<unsigned int>(row), p.seed_lo, p.seed_hi);
+        for (int gb = g0; gb < g1; gb += 32 * kGroups) {
+            Raw zraw[kGroups][G::kVec], yraw[kGroups][G::kVec];
+#pragma unroll
+            for (int k = 0; k < kGroups; ++k) {
+                const int g = gb + k * 32 + lane;
+                if (g < g1) {
+                    G::load(zr, g * kRaceGroup, p.V, zraw[k]);
+                    if (!bonus) G::load(yr, g * kRaceGroup, p.V, yraw[k]);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < kGroups; ++k) {
+                const int g = gb + k * 32 + lane;
+                // A group all of whose logits are below the row's cut cannot win: no exponentials.
+                float W = 0.0f;
+                if (g < g1 && G::hmax(zraw[k]) > cf.zcut) {
+                    float zf[8], yf[8];
+                    G::unpack(zraw[k], zf);
+                    if (!bonus) G::unpack(yraw[k], yf);
+                    W = group_weight(cf, zf, bonus ? zf : yf);
+                }
+                // One Philox block serves four consecutive groups, i.e. four consecutive lanes: the
+                // first of them computes it when any of the four has a weight, the others take its words.
+                const unsigned int need = __ballot_sync(kFull, W > 0.0f);
+                const int leader = lane & ~3;
+                uint4 rnd = make_uint4(0u, 0u, 0u, 0u);
+                if (lane == leader && ((need >> leader) & 0xfu))
+                    rnd = philox4x32_10(make_uint4(static_cast<unsigned int>(g) >> 2, static_cast<unsigned int>(row), 0u, 0u), p.seed_lo, p.seed_hi);
+                rnd.x = __shfl_sync(kFull, rnd.x, leader);
+                rnd.y = __shfl_sync(kFull, rnd.y, leader);
+                rnd.z = __shfl_sync(kFull, rnd.z, leader);
+                rnd.w = __shfl_sync(kFull, rnd.w, leader);
+                if (W > 0.0f) {
+                    const float u = clock_u(philox_word(rnd, static_cast<unsigned int>(g)));
+                    if (W > best.key * u) {                  // E >= u: otherwise the key cannot exceed the best
+                        const float key = W / clock_of(u);
+                        if (key > best.key) {                // groups ascend within a lane: strict keeps the lowest
+                            best.key = key;
+                            best.idx = g;
+                        }
+                    }
+                }
             }
         }
 #pragma unroll
@@ -308,18 +439,41 @@ __global__ void __launch_bounds__(256) sampled_race_kernel(const __grid_constant
 
 // ---- C: per batch row: the draws' winners, look-up, gate, prefix scan -----------------------
 
-__device__ __forceinline__ int race_winner(const SampledParams &p, long long row, int fallback)
+// The drawn token of draw `row`: the winning group over the row's chunks, then the race among its
+// (up to) eight tokens.  `fallback` if no group has a positive weight.
+template <typename L>
+__device__ __forceinline__ int race_winner(const SampledParams &p, long long row, bool bonus, long long yrow, int fallback)
 {
+    using E = typename L::elem;
     float key = 0.0f;
-    int idx = fallback;
+    int g = -1;
     for (int c = 0; c < p.nchunks; ++c) {
         const RacePart x = p.race_part[row * p.nchunks + c];
-        if (x.key > key) {          // chunks ascend: strict keeps the lowest index
+        if (x.key > key) {          // chunks ascend: strict keeps the lowest group
             key = x.key;
-            idx = x.idx;
+            g = x.idx;
         }
     }
-    return idx;
+    if (g < 0) return fallback;
+    const DrawCoef cf = draw_coef(p, row, bonus, yrow);
+    const E *zr = sampled_row_ptr<E>(p, row);
+    const E *yr = bonus ? zr : sampled_row_ptr<E>(p, yrow);
+    float best = 0.0f;
+    int t = g * kRaceGroup;
+    uint4 rnd = make_uint4(0u, 0u, 0u, 0u);
+    for (int e = 0; e < kRaceGroup; ++e) {
+        const int v = g * kRaceGroup + e;
+        if (v >= p.V) break;
+        if ((e & 3) == 0) rnd = philox4x32_10(make_uint4(static_cast<unsigned int>(v) >> 2, static_cast<unsigned int>(row), 1u, 0u), p.seed_lo, p.seed_hi);
+        const float w = draw_weight(cf, L::load_elem(zr, v), bonus ? 0.0f : L::load_elem(yr, v));
+        if (!(w > 0.0f)) continue;
+        const float k2 = w / clock_of(clock_u(philox_word(rnd, static_cast<unsigned int>(v))));
+        if (k2 > best) {            // tokens ascend: strict keeps the lowest
+            best = k2;
+            t = v;
+        }
+    }
+    return t;
 }
 
 template <typename L>
@@ -344,7 +498,7 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
         float score = __int_as_float(0x7fc00000);
         if (!passed) {
             const RowNorm np_ = p.rownorm[row0 + lane];
-            t = race_winner(p, row0 + lane, np_.argmax);                                    // t* ~ norm(max(0, p - q))
+            t = race_winner<L>(p, row0 + lane, false, sampled_rows_z(p) + pos, np_.argmax);    // t* ~ norm(max(0, p - q))
             if (valid) {
                 const E *zr = sampled_row_ptr<E>(p, row0 + lane);
                 const float zd = L::load_elem(zr, d);
@@ -378,10 +532,11 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
     const unsigned int m_rec = __ballot_sync(kFull, record);
     if (lane == 0) {
         int next = t_stop;
-        if (n_acc == K) next = race_winner(p, row0 + K, p.rownorm[row0 + K].argmax);       // bonus ~ p_{gamma+1}
+        const int bonus_t = race_winner<L>(p, row0 + K, true, 0, p.rownorm[row0 + K].argmax);   // bonus ~ p_{gamma+1}
+        if (n_acc == K) next = bonus_t;
         p.accept_len[b] = n_acc;
         p.next_token[b] = next;
-        if (p.diag.bonus) p.diag.bonus[b] = race_winner(p, row0 + K, p.rownorm[row0 + K].argmax);
+        if (p.diag.bonus) p.diag.bonus[b] = bonus_t;
         OcmStatsDev *st = p.ocm.stats;
         atomicAdd(&st->positions, static_cast<unsigned long long>(K));
         if (m_pass) atomicAdd(&st->matches, static_cast<unsigned long long>(__popc(m_pass)));

@@ -451,7 +451,7 @@ __device__ __forceinline__ int update_regime(const StepParams &p)
 // Butterfly fold of one value per lane inside aligned groups of `width` lanes: maximum and
 // its lowest index first, then the sums rescaled (exactly) to the group's reference.
 // Every lane of a group ends with the group's total.
-__device__ __forceinline__ Partial butterfly_fold(Partial v, int width)
+__device__ __forceinline__ Partial butterfly_fold(Partial v, int width, const float l2e = kLog2e)
 {
     float m = v.m;
     int idx = v.idx;
@@ -462,7 +462,7 @@ __device__ __forceinline__ Partial butterfly_fold(Partial v, int width)
         m = take ? om : m;
         idx = take ? oi : idx;
     }
-    const float c = (m == -INFINITY) ? kNoRef : rintf(m * kLog2e);
+    const float c = (m == -INFINITY) ? kNoRef : rintf(m * l2e);
     float s = v.s * pow2_nonpos(v.c - c);
     for (int o = 1; o < width; o <<= 1) s += __shfl_xor_sync(kFull, s, o);
     Partial r;

@@ -265,7 +265,7 @@ def oracle_sampled_row(z, y, d, r, seed, T, tau, b, K1):
     """The oracle on batch row b alone, with that row's own clock streams."""
     orig = ORACLE.race_clocks
     try:
-        ORACLE.race_clocks = lambda s, row, V: orig(s, row + b * K1, V)
+        ORACLE.race_clocks = lambda s, row, stream, first, n: orig(s, row + b * K1, stream, first, n)
         return ORACLE.verify(_f64(z[b:b + 1]), _f64(y[b:b + 1]), d[b:b + 1].cpu().numpy(), r[b:b + 1].cpu().numpy(),
                              seed, T, ORACLE.OCM(64, 2), tau)
     finally:
