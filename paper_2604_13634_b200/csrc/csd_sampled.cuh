@@ -289,8 +289,9 @@ struct Group8<LaneF32Vec> {
     static constexpr int kVec = 2;
     static __device__ __forceinline__ void load(const float *row, int v0, int V, uint4 (&raw)[2])
     {
-        raw[0] = ld_stream16(row + v0);
-        raw[1] = v0 + 4 < V ? ld_stream16(row + v0 + 4) : LaneF32Vec::neg_inf();      // V is a multiple of 4 here
+        // a lane's two vectors share a 32-byte sector: cached loads, so that the second one hits
+        raw[0] = __ldg(reinterpret_cast<const uint4 *>(row + v0));
+        raw[1] = v0 + 4 < V ? __ldg(reinterpret_cast<const uint4 *>(row + v0 + 4)) : LaneF32Vec::neg_inf();   // V is a multiple of 4 here
     }
     static __device__ __forceinline__ float hmax(const uint4 (&raw)[2]) { return fmaxf(LaneF32Vec::hmax(raw[0]), LaneF32Vec::hmax(raw[1])); }
     static __device__ __forceinline__ void unpack(const uint4 (&raw)[2], float (&f)[8])
@@ -458,19 +459,27 @@ __device__ __forceinline__ int race_winner(const SampledParams &p, long long row
     const DrawCoef cf = draw_coef(p, row, bonus, yrow);
     const E *zr = sampled_row_ptr<E>(p, row);
     const E *yr = bonus ? zr : sampled_row_ptr<E>(p, yrow);
+    float zf[kRaceGroup], yf[kRaceGroup];
+#pragma unroll
+    for (int e = 0; e < kRaceGroup; ++e) {       // all gathers in flight together
+        const int v = g * kRaceGroup + e;
+        zf[e] = v < p.V ? L::load_elem(zr, v) : -INFINITY;
+        yf[e] = (v < p.V && !bonus) ? L::load_elem(yr, v) : -INFINITY;
+    }
     float best = 0.0f;
     int t = g * kRaceGroup;
     uint4 rnd = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
     for (int e = 0; e < kRaceGroup; ++e) {
         const int v = g * kRaceGroup + e;
-        if (v >= p.V) break;
         if ((e & 3) == 0) rnd = philox4x32_10(make_uint4(static_cast<unsigned int>(v) >> 2, static_cast<unsigned int>(row), 1u, 0u), p.seed_lo, p.seed_hi);
-        const float w = draw_weight(cf, L::load_elem(zr, v), bonus ? 0.0f : L::load_elem(yr, v));
-        if (!(w > 0.0f)) continue;
-        const float k2 = w / clock_of(clock_u(philox_word(rnd, static_cast<unsigned int>(v))));
-        if (k2 > best) {            // tokens ascend: strict keeps the lowest
-            best = k2;
-            t = v;
+        const float w = draw_weight(cf, zf[e], yf[e]);
+        if (w > 0.0f) {
+            const float k2 = w / clock_of(clock_u(philox_word(rnd, static_cast<unsigned int>(v))));
+            if (k2 > best) {        // tokens ascend: strict keeps the lowest
+                best = k2;
+                t = v;
+            }
         }
     }
     return t;
@@ -494,11 +503,19 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
         d = __ldg(p.draft + pos);
         valid = static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V);
         passed = p.accepted[pos] != 0;
+    }
+    // The draws: lane i < K its residual draw t* ~ norm(max(0, p - q)) if the position failed the test,
+    // lane K the bonus draw t ~ p_{gamma+1} -- one code path, so that they run side by side.
+    const bool is_bonus = lane == K;
+    int drawn = -1;
+    if ((lane < K && !passed) || is_bonus)
+        drawn = race_winner<L>(p, row0 + lane, is_bonus, sampled_rows_z(p) + b * K + lane, p.rownorm[row0 + lane].argmax);
+    if (lane < K) {
+        const long long pos = b * K + lane;
         ok = passed;
         float score = __int_as_float(0x7fc00000);
         if (!passed) {
-            const RowNorm np_ = p.rownorm[row0 + lane];
-            t = race_winner<L>(p, row0 + lane, false, sampled_rows_z(p) + pos, np_.argmax);    // t* ~ norm(max(0, p - q))
+            t = drawn;
             if (valid) {
                 const E *zr = sampled_row_ptr<E>(p, row0 + lane);
                 const float zd = L::load_elem(zr, d);
@@ -514,6 +531,9 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
         if (p.diag.score) p.diag.score[pos] = score;
         if (p.diag.cnt) p.diag.cnt[pos] = cnt;
     }
+    int bonus_t = drawn;                        // lane K's, if there is a lane K
+    if (K == 32 && lane == 0) bonus_t = race_winner<L>(p, row0 + K, true, 0, p.rownorm[row0 + K].argmax);
+    bonus_t = __shfl_sync(kFull, bonus_t, K < 32 ? K : 0);
     const unsigned int kmask = (K == 32) ? kFull : ((1u << K) - 1u);
     const unsigned int okmask = __ballot_sync(kFull, ok) & kmask;
     const unsigned int fail = ~okmask & kmask;
@@ -532,7 +552,6 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
     const unsigned int m_rec = __ballot_sync(kFull, record);
     if (lane == 0) {
         int next = t_stop;
-        const int bonus_t = race_winner<L>(p, row0 + K, true, 0, p.rownorm[row0 + K].argmax);   // bonus ~ p_{gamma+1}
         if (n_acc == K) next = bonus_t;
         p.accept_len[b] = n_acc;
         p.next_token[b] = next;
