@@ -349,7 +349,7 @@ struct Group8Raw<LaneBf16Scalar> {
 };
 
 template <typename L>
-__global__ void __launch_bounds__(256) sampled_race_kernel(const __grid_constant__ SampledParams p)
+__global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_constant__ SampledParams p)
 {
     using E = typename L::elem;
     using G = Group8<L>;

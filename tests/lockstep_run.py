@@ -133,6 +133,42 @@ def run(wl, tau, steps, checkpoint, prewarm_steps, seed=0, first_step=None, load
     return out
 
 
+def run_sampled(wl, tau, steps, T_, lam, seed=0):
+    """The stochastic step (Algorithm 1 at temperature T_) in lock-step with its oracle.  A batch row
+    whose result hangs on a near-tie the oracle flags is counted as excused and the memories are
+    re-synchronised; any other difference raises."""
+    import test_gpu_sampled_parity as S
+    from paper_2604_13634_b200 import SampledBuffers, csd_step_sampled
+    syn = Synth(wl, seed, "cuda")
+    ocm, mem = Ocm(wl.ocm_slots, lam), S.ORACLE.OCM(wl.ocm_slots, lam)
+    buf = SampledBuffers(wl.B, wl.K, wl.V, wl.torch_dtype)
+    t0 = time.time()
+    excused = passed = resc = acc = flagged = 0
+    for s in range(steps):
+        z, y, d, r = syn.step_sampled(s)
+        csd_step_sampled(z, y, d, r, 7919 * seed + s, T_, ocm, tau, buf)
+        ref = S.oracle_sampled(z, y, d, r, 7919 * seed + s, T_, mem, tau)
+        e = S.compare(buf, ref)
+        excused += e
+        if e:
+            S.resync(ocm, mem)
+        flagged += int(ref["near_accept"].sum()) + int(ref["unclear_draw"].sum())
+        passed += int(ref["accepted"].sum())
+        resc += int(ref["rescued_mask"].sum())
+        acc += int(ref["accept_len"].sum())
+        if (s + 1) % 100 == 0:
+            S.compare_memory(ocm, mem)
+    st = S.compare_memory(ocm, mem)
+    assert st["flags"] == 0, st
+    out = dict(workload=wl.name, mode="stochastic", temperature=T_, tau=tau, lam=lam, steps=steps, B=wl.B, K=wl.K, V=wl.V,
+               dtype=wl.dtype, passed_acceptance_test=passed, rescued=resc, accepted=acc,
+               acceptance_rate=acc / (steps * wl.B * wl.K), near_ties_flagged_by_oracle=flagged,
+               batch_rows_excused=excused, n_keys=st["n_keys"], seconds=round(time.time() - t0, 1),
+               verdict="identical apart from the excused rows")
+    ocm.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", required=True)
@@ -144,7 +180,15 @@ def main():
     ap.add_argument("--save", default="", help="write the memory and the running totals here at the end")
     ap.add_argument("--overlap", action="store_true",
                     help="the launch shape the benchmark times (csd_set_overlap: one block per SM and launch)")
+    ap.add_argument("--sampled", type=float, default=0.0,
+                    help="run the stochastic step at this temperature instead of the greedy one")
+    ap.add_argument("--lam", type=int, default=2, help="frequency threshold of the --sampled run")
     args = ap.parse_args()
+    if args.sampled > 0:
+        wl = WORKLOADS[args.workload]
+        for tau in ([float(x) for x in args.taus.split(",")] if args.taus else list(wl.taus)):
+            print(json.dumps(run_sampled(wl, tau, args.steps or wl.steps, args.sampled, args.lam)), flush=True)
+        return
     if args.overlap:
         from paper_2604_13634_b200 import csd_set_overlap
         global OVERLAP
