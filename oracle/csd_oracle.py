@@ -154,7 +154,8 @@ def verify(z: np.ndarray, draft: np.ndarray, ocm: OCM, tau: float, stats=None):
       bad_draft            number of draft ids outside [0, V)
     The memory is NOT modified; see `step`.
     """
-    z = np.asarray(z)
+    if not hasattr(z, "shape"):
+        z = np.asarray(z)          # anything with .shape and [b, i, v] indexing will do (e.g. a lazy decoder)
     B, K1, V = z.shape
     K = K1 - 1
     draft = np.asarray(draft).reshape(B, K)

@@ -24,15 +24,27 @@ pytestmark = pytest.mark.gpu
 RTOL = 1e-5
 
 
-def _np_logits(z):
+class _Bf16Decoded:
+    """bf16 bit patterns that decode on access: the oracle step only gathers single logits once the row
+    statistics come from the C routine, so widening a 100 MB tensor every step would be wasted."""
+
+    def __init__(self, bits):
+        self.bits = bits
+        self.shape = bits.shape
+
+    def __getitem__(self, idx):
+        return ORACLE.bf16_bits_to_f64(np.asarray(self.bits[idx])).reshape(np.shape(self.bits[idx]))
+
+
+def _np_logits(z, lazy=False):
     arr, is_bits = logits_bits_numpy(z)
     if is_bits:
-        return ORACLE.bf16_bits_to_f64(arr).astype(np.float32), arr, True
+        return (_Bf16Decoded(arr) if lazy else ORACLE.bf16_bits_to_f64(arr).astype(np.float32)), arr, True
     return arr, arr, False
 
 
 def oracle_step(z, draft, mem, tau, update=True, use_c=True):
-    vals, raw, is_bits = _np_logits(z)
+    vals, raw, is_bits = _np_logits(z, lazy=use_c and z.is_contiguous())
     stats = None
     if use_c and z.is_contiguous():
         stats = row_stats_c.row_stats_batch(raw, is_bf16_bits=is_bits)
