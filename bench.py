@@ -401,6 +401,7 @@ def run_sampled(args, wl, tau):
     pkg.lib()
     device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
     torch.cuda.set_device(device)
+    pkg.csd_set_overlap(not args.no_overlap)     # a step's statistics kernel may run beside the previous step's tail
     T = args.temperature
     syn = Synth(wl, 0, device)
     step_bytes = (wl.rows + wl.B * wl.K) * wl.V * wl.elt_bytes

@@ -269,7 +269,8 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
 }
 
-csd_status_t run_update(csd_ocm *ocm, const int32_t *d, const int32_t *t, const uint32_t *w, int64_t n, void *stream)
+csd_status_t run_update(csd_ocm *ocm, const int32_t *d, const int32_t *t, const uint32_t *w, int64_t n, void *stream,
+                        bool programmatic = false)
 {
     if (!ocm || n < 0 || (n > 0 && (!d || !t))) return CSD_ERR_INVALID_ARG;
     if (n == 0) return CSD_OK;
@@ -277,8 +278,23 @@ csd_status_t run_update(csd_ocm *ocm, const int32_t *d, const int32_t *t, const 
     long long blocks = (n + 1023) / 1024;
     const long long cap = static_cast<long long>(sm_count()) * 2;
     if (blocks > cap) blocks = cap;
-    ocm_update_kernel<<<static_cast<unsigned int>(blocks), 1024, 0, static_cast<cudaStream_t>(stream)>>>(
-        view_of(ocm), d, t, w, n);
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned int>(blocks));
+    cfg.blockDim = dim3(1024);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    if (programmatic) {     // behind the kernel that writes d / t: the update kernel waits for it itself
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    const long long n_ll = n;
+    if (cudaLaunchKernelEx(&cfg, ocm_update_kernel, view_of(ocm), d, t, w, n_ll) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
     return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
 }
 
@@ -337,11 +353,29 @@ cudaError_t launch_sampled(const SampledParams &p, cudaStream_t st)
         long long b = (tiles + 7) / 8;            // 8 warps per block
         return static_cast<unsigned int>(b < 1 ? 1 : (b > cap ? cap : b));
     };
-    sampled_stats_kernel<L><<<blocks_for(rows * p.nchunks), 256, 0, st>>>(p);
-    sampled_decide_kernel<L><<<static_cast<unsigned int>((draws + 3) / 4), 128, 0, st>>>(p);
-    sampled_race_kernel<L><<<blocks_for(draws * p.nchunks), 256, 0, st>>>(p);
-    sampled_finalize_kernel<L><<<static_cast<unsigned int>((p.B + 3) / 4), 128, 0, st>>>(p);
-    return cudaGetLastError();
+    auto launch = [&](auto kernel, unsigned int grid, unsigned int block, bool programmatic) {
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(block);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        if (programmatic) {
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+        }
+        return cudaLaunchKernelEx(&cfg, kernel, p);
+    };
+    // The statistics kernel touches only inputs and its own partials before it waits, so it may run
+    // beside the previous kernels on the stream when the caller has allowed step overlap; the other
+    // three depend on their predecessor alone and wait for it first thing.
+    cudaError_t err = launch(sampled_stats_kernel<L>, blocks_for(rows * p.nchunks), 256, g_overlap_steps != 0);
+    if (err == cudaSuccess) err = launch(sampled_decide_kernel<L>, static_cast<unsigned int>((draws + 3) / 4), 128, true);
+    if (err == cudaSuccess) err = launch(sampled_race_kernel<L>, blocks_for(draws * p.nchunks), 256, true);
+    if (err == cudaSuccess) err = launch(sampled_finalize_kernel<L>, static_cast<unsigned int>((p.B + 3) / 4), 128, true);
+    return err;
 }
 
 csd_status_t run_sampled(const void *logits, const void *draft_logits, csd_dtype_t dtype, int B, int K, int V,
@@ -404,7 +438,7 @@ csd_status_t run_sampled(const void *logits, const void *draft_logits, csd_dtype
         (void)cudaGetLastError();
         return CSD_ERR_CUDA;
     }
-    if (do_update) return run_update(ocm, rej_draft, rej_target, nullptr, static_cast<int64_t>(B) * K, stream);
+    if (do_update) return run_update(ocm, rej_draft, rej_target, nullptr, static_cast<int64_t>(B) * K, stream, true);
     return CSD_OK;
 }
 

@@ -9,7 +9,12 @@
 // A race is one more streaming arg-max: no normaliser, no prefix sums, no second pass over
 // the winner's neighbourhood, and every tile of a row can run independently.
 //
-// Four launches, stream-ordered:
+// Four launches.  Each is launched programmatically behind the one before (its blocks become
+// resident while that one drains); B, C and the decision kernel wait for their predecessor before
+// anything else and only then let their successor in, so at most two of them are resident.  Kernel A
+// reads only the step's inputs and writes only the chunk statistics, which nobody else writes and
+// only this step's decision kernel reads: with step overlap switched on it streams while the previous
+// step's last kernels finish, and waits for them at its end.
 //   A  sampled_stats_kernel    every row of z and y once: max and sum exp(x/T) per chunk
 //   A2 sampled_decide_kernel   per position: normalisers, alpha, the stochastic test
 //   B  sampled_race_kernel     rows that failed the test (z and y again) and the bonus rows:
@@ -89,6 +94,7 @@ __global__ void __launch_bounds__(256) sampled_stats_kernel(const __grid_constan
     const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
     const long long rows = sampled_rows_z(p) + static_cast<long long>(p.B) * p.K;
     const long long tiles = rows * p.nchunks;
+    pdl_launch_dependents();
     for (long long tile = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < tiles; tile += warps) {
         const long long row = tile / p.nchunks;
         const int c = static_cast<int>(tile - row * p.nchunks);
@@ -97,6 +103,7 @@ __global__ void __launch_bounds__(256) sampled_stats_kernel(const __grid_constan
         const Partial r = warp_tile<L>(sampled_row_ptr<E>(p, row), e0, e1, lane, p.l2e_T);
         if (lane == 0) st_partial_cg(p.stat_part + tile, r);
     }
+    pdl_wait();       // this kernel's completion then implies that of everything before it on the stream
 }
 
 // A weight that can never win a draw.  Clocks lie in [E_min, E_max] = [-ln(1 - 2^-24), -ln(2^-24)]
@@ -143,6 +150,8 @@ __global__ void __launch_bounds__(128) sampled_decide_kernel(const __grid_consta
     const int lane = threadIdx.x & 31;
     const long long n = sampled_rows_z(p);
     const long long j = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    pdl_wait();
+    pdl_launch_dependents();
     if (j >= n) return;
     const int K = p.K;
     const long long b = j / (K + 1);
@@ -360,6 +369,8 @@ __global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_const
     const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
     const long long draws = sampled_rows_z(p);
     const long long tiles = draws * p.nchunks;
+    pdl_wait();
+    pdl_launch_dependents();
     for (long long tile = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < tiles; tile += warps) {
         const long long row = tile / p.nchunks;
         const int c = static_cast<int>(tile - row * p.nchunks);
@@ -492,6 +503,8 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
     const int lane = threadIdx.x & 31;
     const int K = p.K;
     const long long b = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    pdl_wait();
+    pdl_launch_dependents();
     if (b >= p.B) return;
     const long long row0 = b * (K + 1);
 
