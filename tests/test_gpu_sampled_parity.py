@@ -270,3 +270,66 @@ def oracle_sampled_row(z, y, d, r, seed, T, tau, b, K1):
                              seed, T, ORACLE.OCM(64, 2), tau)
     finally:
         ORACLE.race_clocks = orig
+
+
+def test_overlapped_and_replayed_steps_match_plain_launches():
+    """Back-to-back stochastic steps with step overlap on (the statistics kernel of a step runs beside the
+    tail of the step before), eagerly and as a replayed CUDA graph, against plain launches; the plain
+    run's last step is pinned to the oracle."""
+    from paper_2604_13634_b200 import csd_set_overlap
+    wl = dataclasses.replace(WORKLOADS["batched_serving"], B=8)
+    syn = Synth(wl, 2, "cuda")
+    inputs = [syn.step_sampled(s) for s in range(3)]
+    reps = 12
+
+    def run(overlap, graph):
+        try:
+            csd_set_overlap(overlap)
+            ocm = Ocm(4096, 2)
+            bufs = [SampledBuffers(wl.B, wl.K, wl.V, wl.torch_dtype) for _ in inputs]
+            for b in bufs[1:]:                                   # one workspace for all, as a serving loop has
+                b.workspace, b.ws_bytes = bufs[0].workspace, bufs[0].ws_bytes
+
+            def ring():
+                for i, ((z, y, d, r), buf) in enumerate(zip(inputs, bufs)):
+                    csd_step_sampled(z, y, d, r, 500 + i, 0.3, ocm, 0.3, buf)
+            if graph:
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    ring()
+                torch.cuda.current_stream().wait_stream(side)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    ring()
+                for _ in range(reps - 1):
+                    g.replay()
+            else:
+                for _ in range(reps):
+                    ring()
+            torch.cuda.synchronize()
+            out = ([[t.clone() for t in (b.accept_len, b.next_token, b.rescued_mask, b.rej_draft, b.rej_target,
+                                         b.diag["t_star"], b.diag["accepted"], b.diag["cnt"], b.diag["alpha"])] for b in bufs],
+                   ocm.export(), ocm.stats())
+            ocm.close()
+            return out
+        finally:
+            csd_set_overlap(False)
+
+    ref_out, ref_exp, ref_st = run(False, False)
+    assert ref_st["steps"] == reps * len(inputs) and ref_st["flags"] == 0 and ref_st["rescues"] > 0
+    for overlap, graph in ((True, False), (True, True), (False, True)):
+        out, exp, st = run(overlap, graph)
+        assert st == ref_st, (overlap, graph)
+        assert all(torch.equal(p, q) for p, q in zip(exp, ref_exp)), (overlap, graph)
+        for x, y in zip(out, ref_out):
+            assert all(torch.equal(p, q) for p, q in zip(x, y)), (overlap, graph)     # the same launches: bit-identical
+    mem = ORACLE.OCM(4096, 2)
+    for rep in range(reps):
+        for i, (z, y, d, r) in enumerate(inputs):
+            ref = oracle_sampled(z, y, d, r, 500 + i, 0.3, mem, 0.3)
+    if not (ref["near_accept"].any() or ref["unclear_draw"].any()):
+        assert np.array_equal(ref_out[-1][0].cpu().numpy(), ref["accept_len"])
+        assert np.array_equal(ref_out[-1][5].cpu().numpy(), ref["t_star"])
+    rd, rt, rc = mem.export()
+    assert np.array_equal(ref_exp[0].numpy(), rd) and np.array_equal(ref_exp[2].numpy(), rc)
