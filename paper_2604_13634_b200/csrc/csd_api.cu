@@ -157,10 +157,10 @@ Shape pick_shape(int B, int K, int V, csd_dtype_t dt, bool overlap)
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-    size_t seq_off, half_bytes, partials_off, hint_off, b_ticket_off, g_ticket_off, total;   // *_off within a half
+    size_t seq_off, copy_bytes, partials_off, hint_off, b_ticket_off, g_ticket_off, total;   // *_off within a copy
 };
 
-// header {launch sequence, blocks counted in, launches completed} followed by two halves,
+// header {launch sequence, blocks counted in, launches completed} followed by kScratchRing copies of the scratch,
 // each {partials | slot hints | per-batch-row tickets | global ticket}
 WorkspaceLayout ws_layout(int B, int K, const Shape &s)
 {
@@ -170,8 +170,8 @@ WorkspaceLayout ws_layout(int B, int K, const Shape &s)
     w.hint_off = align_up(static_cast<size_t>(B) * (K + 1) * s.slots_per_row * sizeof(Partial), 256);
     w.b_ticket_off = align_up(w.hint_off + static_cast<size_t>(B) * K * sizeof(int), 256);
     w.g_ticket_off = align_up(w.b_ticket_off + static_cast<size_t>(B) * sizeof(unsigned int), 16);
-    w.half_bytes = align_up(w.g_ticket_off + 16, 256);
-    w.total = 256 + kScratchRing * w.half_bytes;
+    w.copy_bytes = align_up(w.g_ticket_off + 16, 256);
+    w.total = 256 + kScratchRing * w.copy_bytes;
     return w;
 }
 
@@ -217,9 +217,9 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.rej_d = rej_draft; p.rej_t = rej_target;
     if (diag) p.diag = *diag;
     char *ws = static_cast<char *>(workspace);
-    if (w.half_bytes > 0xffffffffull) return CSD_ERR_UNSUPPORTED;
+    if (w.copy_bytes > 0xffffffffull) return CSD_ERR_UNSUPPORTED;
     p.scratch = ws + 256;
-    p.copy_bytes = static_cast<unsigned int>(w.half_bytes);
+    p.copy_bytes = static_cast<unsigned int>(w.copy_bytes);
     p.hint_off = static_cast<unsigned int>(w.hint_off);
     p.b_ticket_off = static_cast<unsigned int>(w.b_ticket_off);
     p.g_ticket_off = static_cast<unsigned int>(w.g_ticket_off);

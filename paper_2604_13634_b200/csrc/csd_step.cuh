@@ -546,7 +546,7 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
     const ScratchCopy sc = scratch_of(p, seq);
     fold_rows(p, sc, b, lane, rs);
 
-    // Everything above read only this launch's inputs and its own half of the scratch.
+    // Everything above read only this launch's inputs and its own copy of the scratch.
     // From here on the previous launch must be complete: the memory, its statistics and
     // the output buffers come into play.
     wait_completed(p, seq);
