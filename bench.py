@@ -389,8 +389,8 @@ def run_ours(args, wl, tau):
 def run_sampled(args, wl, tau):
     """csd_step_sampled (statistics, decision, races, finalisation, memory update: five
     launches per step) over a ring of resident inputs.  Algorithmic bytes per step: every row of
-    the target and draft logits once, the two rows of every position that fails the acceptance
-    test once more, and the bonus rows once more."""
+    the target and draft logits once, the two rows of every position whose residual draw a row
+    needs once more, and the bonus row of every fully accepted batch row once more."""
     import torch
 
     import paper_2604_13634_b200 as pkg
@@ -413,12 +413,8 @@ def run_sampled(args, wl, tau):
     if kind == "pairs":
         ocm.update(*syn.prewarm_pairs(n))
     diag_buf = pkg.SampledBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, device=device, diag=True)
-    failed = []
-    for i, (z, y, d, r) in enumerate(ring):                 # also warms the memory up
-        pkg.csd_step_sampled(z, y, d, r, i, T, ocm, tau, diag_buf)
-        failed.append(int((diag_buf.diag["accepted"] == 0).sum().item()))
-    rows_per_step = wl.rows + wl.B * wl.K + 2 * (sum(failed) / len(failed)) + wl.B
-    algo_bytes = rows_per_step * wl.V * wl.elt_bytes
+    for i, (z, y, d, r) in enumerate(ring):                 # warms the memory up
+        pkg.csd_step_sampled(z, y, d, r, 1000 + i, T, ocm, tau, diag_buf)
     buf = pkg.SampledBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, device=device, diag=False)
 
     def step(i):
@@ -449,6 +445,18 @@ def run_sampled(args, wl, tau):
     b.synchronize()
     clocks = sampler.stop()
     sec = a.elapsed_time(b) * 1e-3
+    # how many draws a step makes depends on the memory (rescues let rows go on): counted on one more pass
+    # over the ring with the memory as the timed region left it
+    failed, draws, bonus = [], [], []
+    for i, (z, y, d, r) in enumerate(ring):
+        pkg.csd_step_sampled(z, y, d, r, 1000 + i, T, ocm, tau, diag_buf)
+        failed.append(int((diag_buf.diag["accepted"] == 0).sum().item()))
+        draws.append(int((diag_buf.diag["t_star"] >= 0).sum().item()))
+        bonus.append(int((diag_buf.diag["bonus"] >= 0).sum().item()))
+    mean = lambda v: sum(v) / len(v)
+    # every row of z and y once; z and y again for each residual draw made; z again for each bonus draw made
+    rows_per_step = wl.rows + wl.B * wl.K + 2 * mean(draws) + mean(bonus)
+    algo_bytes = rows_per_step * wl.V * wl.elt_bytes
     peak, peak_kind = measured_peak()
     achieved = algo_bytes * steps / sec / 1e9
     st = ocm.stats()
@@ -459,13 +467,14 @@ def run_sampled(args, wl, tau):
                 "mode": f"stochastic verification (Algorithm 1 at T={T}): acceptance test, residual and bonus draws",
                 "draft_logits": "target logits + N(0, 0.3^2), the draft token raised to the row maximum + 1",
                 "l2_policy": f"ring of {ring_len} distinct step inputs ({ring_len * step_bytes / 1e6:.0f} MB, > 2x L2)",
-                "launch": "CUDA graph of %d steps (5 launches each) replayed" % graph_steps,
-                "failed_positions_per_step": sum(failed) / len(failed)}),
+                "launch": "CUDA graph of %d steps (7 launches each) replayed" % graph_steps,
+                "failed_positions_per_step": mean(failed), "residual_draws_per_step": mean(draws),
+                "bonus_draws_per_step": mean(bonus)}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": None, "peak_source": f"of {peak_kind}",
                          "kernel": "sampled_stats_kernel + sampled_race_kernel (whole step)",
                          "bytes_per_launch": algo_bytes},
-            "gpu_launches": 5 * steps, "clocks": clocks,
+            "gpu_launches": 7 * steps, "clocks": clocks,
             "ocm": {k: st[k] for k in ("n_keys", "n_dropped", "steps", "matches", "rescues", "rejections", "flags")}}
     if not args.no_cpu_baseline:
         import dataclasses

@@ -241,25 +241,27 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
  *     ties) with E_v = -ln(1 - u_v), u_v = (j + 1/2) / 2^23, j = the top 23 bits of word
  *     (v & 3) of Philox4x32-10 (Salmon et al., SC'11) under key (seed low, seed high) and
  *     counter (v >> 2, b*(K+1)+i, 0, 0); i = K is the bonus draw.  P(v) = w(v) / sum w.
- * Every position that fails the acceptance test gets its t* (diag.t_star), reached or not.
+ * Draws are made only where a row can need them: for its first failed position, for the later failed
+ * positions if that one was rescued, and the bonus draw if every position went through; diag.t_star and
+ * diag.bonus are -1 where no draw was made (never at a position the row reaches).
  * Look-ups see the memory as it is when the call starts; a draft id outside [0,V) fails
  * the test, cannot be rescued and is not recorded.
  *
  * draft_logits: y[B, K, V], same dtype as logits, strides in elements, V contiguous.
  * temperature > 0; tau as for csd_verify.  workspace: csd_sampled_workspace_bytes bytes,
  * 16-byte aligned, no initialisation needed.  diag: NULL or a HOST struct of optional
- * device arrays.  Four kernel launches (statistics, decision, races, finalisation);
- * csd_step_sampled appends the memory update of the recorded pairs in (b,i) order.
+ * device arrays.  Six kernel launches (statistics, decision, two rounds of races and
+ * finalisation); csd_step_sampled appends the memory update of the recorded pairs in (b,i) order.
  * Errors as csd_verify; also INVALID_ARG for temperature <= 0 or NaN.  Asynchronous. */
 typedef struct {
     float    *alpha;     /* [B,K]   min(1, p(d)/q(d))                                        */
     uint8_t  *accepted;  /* [B,K]   1 where r <= alpha                                       */
-    int32_t  *t_star;    /* [B,K]   residual draw where the test failed, -1 where it passed  */
+    int32_t  *t_star;    /* [B,K]   residual draw where one was made (see above), else -1     */
     float    *lse_p;     /* [B,K+1] ln sum_v exp(z_v / T)                                    */
     float    *lse_q;     /* [B,K]   ln sum_v exp(y_v / T)                                    */
     float    *score;     /* [B,K]   exp(z_d - z_t*) where the test failed (NaN elsewhere)    */
     uint32_t *cnt;       /* [B,K]   memory count of (d, t*) at the start of the step         */
-    int32_t  *bonus;     /* [B]     the draw from p_K                                        */
+    int32_t  *bonus;     /* [B]     the draw from p_K where one was made, else -1            */
 } csd_sampled_diag_t;
 
 size_t csd_sampled_workspace_bytes(int B, int K, int V, csd_dtype_t dtype);

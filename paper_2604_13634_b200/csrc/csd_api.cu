@@ -317,8 +317,8 @@ int sampled_chunk_elems(int B, int K, int V)
 }
 
 struct SampledLayout {
-    size_t stat_part, rownorm, alpha, accepted, race_part, total;
-    int nchunks, chunk_elems;
+    size_t stat_part, rownorm, alpha, accepted, race_part, row_state, total;
+    int nchunks, chunk_elems, race_nchunks;
 };
 
 SampledLayout sampled_layout(int B, int K, int V)
@@ -326,6 +326,7 @@ SampledLayout sampled_layout(int B, int K, int V)
     SampledLayout w;
     w.chunk_elems = sampled_chunk_elems(B, K, V);
     w.nchunks = (V + w.chunk_elems - 1) / w.chunk_elems;
+    w.race_nchunks = (V + kSampledChunkMin - 1) / kSampledChunkMin;
     const size_t rows = static_cast<size_t>(B) * (2 * K + 1);
     const size_t draws = static_cast<size_t>(B) * (K + 1);
     size_t off = 0;
@@ -338,7 +339,8 @@ SampledLayout sampled_layout(int B, int K, int V)
     w.rownorm = take(rows * sizeof(RowNorm));
     w.alpha = take(static_cast<size_t>(B) * K * sizeof(float));
     w.accepted = take(static_cast<size_t>(B) * K);
-    w.race_part = take(draws * w.nchunks * sizeof(RacePart));
+    w.race_part = take(draws * w.race_nchunks * sizeof(RacePart));
+    w.row_state = take(static_cast<size_t>(B));
     w.total = off;
     return w;
 }
@@ -353,7 +355,7 @@ cudaError_t launch_sampled(const SampledParams &p, cudaStream_t st)
         long long b = (tiles + 7) / 8;            // 8 warps per block
         return static_cast<unsigned int>(b < 1 ? 1 : (b > cap ? cap : b));
     };
-    auto launch = [&](auto kernel, unsigned int grid, unsigned int block, bool programmatic) {
+    auto launch = [&](auto kernel, unsigned int grid, unsigned int block, bool programmatic, auto... extra) {
         cudaLaunchConfig_t cfg;
         std::memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = dim3(grid);
@@ -366,15 +368,20 @@ cudaError_t launch_sampled(const SampledParams &p, cudaStream_t st)
             cfg.attrs = attr;
             cfg.numAttrs = 1;
         }
-        return cudaLaunchKernelEx(&cfg, kernel, p);
+        return cudaLaunchKernelEx(&cfg, kernel, p, extra...);
     };
     // The statistics kernel touches only inputs and its own partials before it waits, so it may run
     // beside the previous kernels on the stream when the caller has allowed step overlap; the other
     // three depend on their predecessor alone and wait for it first thing.
     cudaError_t err = launch(sampled_stats_kernel<L>, blocks_for(rows * p.nchunks), 256, g_overlap_steps != 0);
     if (err == cudaSuccess) err = launch(sampled_decide_kernel<L>, static_cast<unsigned int>((draws + 3) / 4), 128, true);
-    if (err == cudaSuccess) err = launch(sampled_race_kernel<L>, blocks_for(draws * p.nchunks), 256, true);
-    if (err == cudaSuccess) err = launch(sampled_finalize_kernel<L>, static_cast<unsigned int>((p.B + 3) / 4), 128, true);
+    // two rounds of draws: each row's first failed position (or its bonus row), then what the rows whose
+    // first failure was rescued still need; a round's race launch is sized for the draws it can have
+    const unsigned int fin_blocks = static_cast<unsigned int>((p.B + 3) / 4);
+    if (err == cudaSuccess) err = launch(sampled_race_kernel<L>, blocks_for(static_cast<long long>(p.B) * p.race_nchunks), 256, true, 1);
+    if (err == cudaSuccess) err = launch(sampled_finalize_kernel<L>, fin_blocks, 128, true, 1);
+    if (err == cudaSuccess) err = launch(sampled_race_kernel<L>, blocks_for(draws * p.race_nchunks), 256, true, 2);
+    if (err == cudaSuccess) err = launch(sampled_finalize_kernel<L>, fin_blocks, 128, true, 2);
     return err;
 }
 
@@ -419,8 +426,11 @@ csd_status_t run_sampled(const void *logits, const void *draft_logits, csd_dtype
     p.alpha = reinterpret_cast<float *>(ws + w.alpha);
     p.accepted = reinterpret_cast<unsigned char *>(ws + w.accepted);
     p.race_part = reinterpret_cast<RacePart *>(ws + w.race_part);
+    p.row_state = reinterpret_cast<unsigned char *>(ws + w.row_state);
     p.chunk_elems = w.chunk_elems;
     p.nchunks = w.nchunks;
+    p.race_chunk_elems = kSampledChunkMin;
+    p.race_nchunks = w.race_nchunks;
 
     const int eb = elt_bytes(dtype);
     const int per_vec = 16 / eb;

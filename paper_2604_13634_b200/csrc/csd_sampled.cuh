@@ -9,7 +9,13 @@
 // A race is one more streaming arg-max: no normaliser, no prefix sums, no second pass over
 // the winner's neighbourhood, and every tile of a row can run independently.
 //
-// Four launches.  Each is launched programmatically behind the one before (its blocks become
+// Algorithm 1 stops a row at its first un-rescued rejection, so most residual draws of a step are never
+// needed: a row's FIRST failed position always is, the later ones only if that one was rescued.  The
+// draws therefore run in two rounds: round 1 races each row's first failed position (or its bonus row if
+// every position passed) and finalises every row that stops there; round 2 races the remaining failed
+// positions and the bonus row of the rows whose first failure was rescued, and finalises those.
+//
+// Six launches (A, A2, B1, C1, B2, C2) plus the memory's update kernel.  Each is launched programmatically behind the one before (its blocks become
 // resident while that one drains); B, C and the decision kernel wait for their predecessor before
 // anything else and only then let their successor in, so at most two of them are resident.  Kernel A
 // reads only the step's inputs and writes only the chunk statistics, which nobody else writes and
@@ -17,8 +23,8 @@
 // step's last kernels finish, and waits for them at its end.
 //   A  sampled_stats_kernel    every row of z and y once: max and sum exp(x/T) per chunk
 //   A2 sampled_decide_kernel   per position: normalisers, alpha, the stochastic test
-//   B  sampled_race_kernel     rows that failed the test (z and y again) and the bonus rows:
-//                              best key per chunk
+//   B  sampled_race_kernel     the round's draws (z and y rows again; bonus rows: z only): best group
+//                              key per chunk
 //   C  sampled_finalize_kernel per batch row: t*, look-up, gate, prefix scan, outputs
 // followed by the memory's own update kernel on the recorded pairs.
 #pragma once
@@ -63,8 +69,10 @@ struct SampledParams {
     RowNorm *rownorm;         // [B*(K+1) + B*K]: target rows first, then draft rows
     float *alpha;             // [B*K]
     unsigned char *accepted;  // [B*K]
-    RacePart *race_part;      // [B*(K+1) * nchunks]
-    int chunk_elems, nchunks;
+    RacePart *race_part;      // [B*(K+1) * race_nchunks]
+    unsigned char *row_state; // [B] 1 while a batch row still needs the second round of draws
+    int chunk_elems, nchunks;             // tiles of the statistics kernel
+    int race_chunk_elems, race_nchunks;   // tiles of the race kernel: smaller, a round has few rows to spread
 };
 
 __device__ __forceinline__ long long sampled_rows_z(const SampledParams &p) { return static_cast<long long>(p.B) * (p.K + 1); }
@@ -358,7 +366,7 @@ struct Group8Raw<LaneBf16Scalar> {
 };
 
 template <typename L>
-__global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_constant__ SampledParams p)
+__global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_constant__ SampledParams p, const int round)
 {
     using E = typename L::elem;
     using G = Group8<L>;
@@ -368,22 +376,28 @@ __global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_const
     const int K = p.K;
     const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
     const long long draws = sampled_rows_z(p);
-    const long long tiles = draws * p.nchunks;
+    // round 1 has one draw per batch row (tiles run over batch rows), round 2 up to K per pending row
+    const long long tiles = (round == 1 ? static_cast<long long>(p.B) : draws) * p.race_nchunks;
     pdl_wait();
     pdl_launch_dependents();
     for (long long tile = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < tiles; tile += warps) {
-        const long long row = tile / p.nchunks;
-        const int c = static_cast<int>(tile - row * p.nchunks);
-        const long long b = row / (K + 1);
-        const int i = static_cast<int>(row - b * (K + 1));
+        const long long unit = tile / p.race_nchunks;
+        const int c = static_cast<int>(tile - unit * p.race_nchunks);
+        const long long b = round == 1 ? unit : unit / (K + 1);
+        if (round == 2 && p.row_state[b] == 0) continue;            // finalised in round 1
+        // f0 = the batch row's first failed position, K if none
+        const unsigned int failed = __ballot_sync(kFull, lane < K && p.accepted[b * K + lane] == 0);
+        const int f0 = failed ? __ffs(failed) - 1 : K;
+        const int i = round == 1 ? f0 : static_cast<int>(unit - b * (K + 1));
         const bool bonus = i == K;
-        if (!bonus && p.accepted[b * K + i]) continue;       // passed the stochastic test: no draw
+        if (round == 2 && !(i > f0 && (bonus || ((failed >> i) & 1u)))) continue;
+        const long long row = b * (K + 1) + i;
         const long long yrow = draws + b * K + i;
         const DrawCoef cf = draw_coef(p, row, bonus, yrow);
         const E *zr = sampled_row_ptr<E>(p, row);
         const E *yr = bonus ? zr : sampled_row_ptr<E>(p, yrow);
-        const int g0 = c * (p.chunk_elems / kRaceGroup);
-        const int g1 = min((p.V + kRaceGroup - 1) / kRaceGroup, g0 + p.chunk_elems / kRaceGroup);
+        const int g0 = c * (p.race_chunk_elems / kRaceGroup);
+        const int g1 = min((p.V + kRaceGroup - 1) / kRaceGroup, g0 + p.race_chunk_elems / kRaceGroup);
         RaceBest best;
         best.key = 0.0f;
         best.idx = 0x7fffffff;
@@ -444,7 +458,7 @@ __global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_const
             RacePart out;
             out.key = best.key;
             out.idx = best.idx;
-            p.race_part[tile] = out;
+            p.race_part[row * p.race_nchunks + c] = out;
         }
     }
 }
@@ -459,8 +473,8 @@ __device__ __forceinline__ int race_winner(const SampledParams &p, long long row
     using E = typename L::elem;
     float key = 0.0f;
     int g = -1;
-    for (int c = 0; c < p.nchunks; ++c) {
-        const RacePart x = p.race_part[row * p.nchunks + c];
+    for (int c = 0; c < p.race_nchunks; ++c) {
+        const RacePart x = p.race_part[row * p.race_nchunks + c];
         if (x.key > key) {          // chunks ascend: strict keeps the lowest group
             key = x.key;
             g = x.idx;
@@ -497,7 +511,7 @@ __device__ __forceinline__ int race_winner(const SampledParams &p, long long row
 }
 
 template <typename L>
-__global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_constant__ SampledParams p)
+__global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_constant__ SampledParams p, const int round)
 {
     using E = typename L::elem;
     const int lane = threadIdx.x & 31;
@@ -506,6 +520,7 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
     pdl_wait();
     pdl_launch_dependents();
     if (b >= p.B) return;
+    if (round == 2 && p.row_state[b] == 0) return;       // finalised in round 1
     const long long row0 = b * (K + 1);
 
     bool passed = false, valid = false, ok = false;
@@ -517,17 +532,20 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
         valid = static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V);
         passed = p.accepted[pos] != 0;
     }
-    // The draws: lane i < K its residual draw t* ~ norm(max(0, p - q)) if the position failed the test,
+    const unsigned int failed = __ballot_sync(kFull, lane < K && !passed);
+    const int f0 = failed ? __ffs(failed) - 1 : K;        // the row's first failed position
+    // The draws that exist so far: round 1 has made the one of position f0 (the bonus draw if f0 = K),
+    // round 2 all the others of this row.  Lane i < K takes its residual draw t* ~ norm(max(0, p - q)),
     // lane K the bonus draw t ~ p_{gamma+1} -- one code path, so that they run side by side.
     const bool is_bonus = lane == K;
+    const bool have = round == 1 ? lane == f0 : ((lane < K && !passed) || is_bonus);
     int drawn = -1;
-    if ((lane < K && !passed) || is_bonus)
+    if (have && lane <= K)
         drawn = race_winner<L>(p, row0 + lane, is_bonus, sampled_rows_z(p) + b * K + lane, p.rownorm[row0 + lane].argmax);
+    float score = __int_as_float(0x7fc00000);
     if (lane < K) {
-        const long long pos = b * K + lane;
         ok = passed;
-        float score = __int_as_float(0x7fc00000);
-        if (!passed) {
+        if (!passed && have) {
             t = drawn;
             if (valid) {
                 const E *zr = sampled_row_ptr<E>(p, row0 + lane);
@@ -540,12 +558,21 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
                 score = expf(zd - zt);
             }
         }
+    }
+    if (round == 1) {
+        // first failure rescued: the row goes on, and needs the draws of round 2
+        const bool pending = f0 < K && __shfl_sync(kFull, ok, f0);
+        if (lane == 0) p.row_state[b] = pending ? 1 : 0;
+        if (pending) return;
+    }
+    if (lane < K) {
+        const long long pos = b * K + lane;
         if (p.diag.t_star) p.diag.t_star[pos] = t;
         if (p.diag.score) p.diag.score[pos] = score;
         if (p.diag.cnt) p.diag.cnt[pos] = cnt;
     }
-    int bonus_t = drawn;                        // lane K's, if there is a lane K
-    if (K == 32 && lane == 0) bonus_t = race_winner<L>(p, row0 + K, true, 0, p.rownorm[row0 + K].argmax);
+    int bonus_t = K < 32 ? drawn : -1;          // lane K's, if there is a lane K and the draw was made
+    if (K == 32 && lane == 0 && (round == 2 || f0 == K)) bonus_t = race_winner<L>(p, row0 + K, true, 0, p.rownorm[row0 + K].argmax);
     bonus_t = __shfl_sync(kFull, bonus_t, K < 32 ? K : 0);
     const unsigned int kmask = (K == 32) ? kFull : ((1u << K) - 1u);
     const unsigned int okmask = __ballot_sync(kFull, ok) & kmask;

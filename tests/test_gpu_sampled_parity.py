@@ -53,10 +53,20 @@ def compare(buf: SampledBuffers, ref):
     assert acc_ok.all(), "acceptance test differs away from r == alpha"
     same_acc = dg["accepted"].astype(bool) == ref["accepted"]
     unclear = ref["unclear_draw"]
-    draw_same = (dg["t_star"] == ref["t_star"]) | ~same_acc
+    # The library makes only the draws a row can need (the first failed position, the others if that one was
+    # rescued, the bonus draw if every position went through): t_star = -1 / bonus = -1 where none was made.
+    # Every failed position the row REACHES must have its draw; wherever one was made it must be the oracle's.
+    made = dg["t_star"] >= 0
+    pos = np.arange(K)[None, :]
+    reached_failed = ~ref["accepted"] & (pos <= ref["accept_len"][:, None]) & same_acc
+    rows_clear = ~(ref["near_accept"].any(axis=1) | unclear.any(axis=1))
+    assert (made | ~reached_failed | ~rows_clear[:, None]).all(), "a reached failed position has no draw"
+    draw_same = (dg["t_star"] == ref["t_star"]) | ~same_acc | ~made
     assert (draw_same | unclear[:, :K]).all(), "a residual draw differs although its race is clear"
-    assert ((dg["bonus"] == ref["bonus"]) | unclear[:, K]).all(), "a bonus draw differs although its race is clear"
-    settled = same_acc & (dg["t_star"] == ref["t_star"])
+    bonus_made = dg["bonus"] >= 0
+    assert (bonus_made | (ref["accept_len"] < K) | ~rows_clear).all(), "a fully accepted row has no bonus draw"
+    assert ((dg["bonus"] == ref["bonus"]) | ~bonus_made | unclear[:, K]).all(), "a bonus draw differs although its race is clear"
+    settled = same_acc & made & (dg["t_star"] == ref["t_star"])
     rej = settled & ~ref["accepted"]
     assert np.array_equal(dg["cnt"][rej].astype(np.int64) & 0xFFFFFFFF, ref["cnt"][rej]), "cnt"
     valid = rej & ~np.isnan(ref["score"])
@@ -256,7 +266,8 @@ def test_large_batch_shape_on_sampled_rows():
         if clear:
             for k, v in got.items():
                 assert np.array_equal(v, ref[k][0]), (b, k)
-            assert np.array_equal(buf.diag["t_star"][b].cpu().numpy(), ref["t_star"][0])
+            got = buf.diag["t_star"][b].cpu().numpy()
+            assert ((got == ref["t_star"][0]) | (got < 0)).all()              # draws are made on demand
         close("alpha", buf.diag["alpha"][b].cpu().numpy(), ref["alpha"][0], atol=1e-12)
     ocm.close()
 
@@ -330,6 +341,7 @@ def test_overlapped_and_replayed_steps_match_plain_launches():
             ref = oracle_sampled(z, y, d, r, 500 + i, 0.3, mem, 0.3)
     if not (ref["near_accept"].any() or ref["unclear_draw"].any()):
         assert np.array_equal(ref_out[-1][0].cpu().numpy(), ref["accept_len"])
-        assert np.array_equal(ref_out[-1][5].cpu().numpy(), ref["t_star"])
+        got = ref_out[-1][5].cpu().numpy()
+        assert ((got == ref["t_star"]) | (got < 0)).all()                     # draws are made on demand
     rd, rt, rc = mem.export()
     assert np.array_equal(ref_exp[0].numpy(), rd) and np.array_equal(ref_exp[2].numpy(), rc)
