@@ -317,7 +317,7 @@ int sampled_chunk_elems(int B, int K, int V)
 }
 
 struct SampledLayout {
-    size_t stat_part, rownorm, alpha, accepted, race_part, row_state, total;
+    size_t stat_part, rownorm, alpha, accepted, race_best, row_state, total;
     int nchunks, chunk_elems, race_nchunks;
 };
 
@@ -339,7 +339,7 @@ SampledLayout sampled_layout(int B, int K, int V)
     w.rownorm = take(rows * sizeof(RowNorm));
     w.alpha = take(static_cast<size_t>(B) * K * sizeof(float));
     w.accepted = take(static_cast<size_t>(B) * K);
-    w.race_part = take(draws * w.race_nchunks * sizeof(RacePart));
+    w.race_best = take(draws * sizeof(unsigned long long));
     w.row_state = take(static_cast<size_t>(B));
     w.total = off;
     return w;
@@ -425,7 +425,7 @@ csd_status_t run_sampled(const void *logits, const void *draft_logits, csd_dtype
     p.rownorm = reinterpret_cast<RowNorm *>(ws + w.rownorm);
     p.alpha = reinterpret_cast<float *>(ws + w.alpha);
     p.accepted = reinterpret_cast<unsigned char *>(ws + w.accepted);
-    p.race_part = reinterpret_cast<RacePart *>(ws + w.race_part);
+    p.race_best = reinterpret_cast<unsigned long long *>(ws + w.race_best);
     p.row_state = reinterpret_cast<unsigned char *>(ws + w.row_state);
     p.chunk_elems = w.chunk_elems;
     p.nchunks = w.nchunks;

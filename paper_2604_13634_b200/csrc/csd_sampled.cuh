@@ -43,10 +43,14 @@ struct RowNorm {
                     // (see race_skip_bound); -inf if no bound is known
 };
 
-struct __align__(8) RacePart {
-    float key;      // best w/E of the chunk (0 if none)
-    int idx;        // its index (lowest on ties), 0x7fffffff if none
-};
+// The best group of a draw so far, as one word that atomicMax can maintain: the key's bits above (keys
+// are positive floats, whose bit patterns order like their values), ~group below (so that of two equal
+// keys the lower group wins).  0 = no group with a positive weight yet.  The maximum does not depend on
+// the order in which the tiles arrive.
+__device__ __forceinline__ unsigned long long race_pack(float key, int group)
+{
+    return (static_cast<unsigned long long>(__float_as_uint(key)) << 32) | (0xffffffffu - static_cast<unsigned int>(group));
+}
 
 struct SampledParams {
     const void *z, *y;
@@ -69,7 +73,7 @@ struct SampledParams {
     RowNorm *rownorm;         // [B*(K+1) + B*K]: target rows first, then draft rows
     float *alpha;             // [B*K]
     unsigned char *accepted;  // [B*K]
-    RacePart *race_part;      // [B*(K+1) * race_nchunks]
+    unsigned long long *race_best;   // [B*(K+1)] see race_pack; cleared by the decision kernel
     unsigned char *row_state; // [B] 1 while a batch row still needs the second round of draws
     int chunk_elems, nchunks;             // tiles of the statistics kernel
     int race_chunk_elems, race_nchunks;   // tiles of the race kernel: smaller, a round has few rows to spread
@@ -170,6 +174,7 @@ __global__ void __launch_bounds__(128) sampled_decide_kernel(const __grid_consta
     const long long yrow = n + pos;
     if (i < K) nq = fold_row_norm(p, yrow, lane);
     if (lane != 0) return;
+    p.race_best[j] = 0ull;
     if (!(np_.lse2 == np_.lse2) || np_.lse2 == INFINITY || np_.m == -INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
     if (p.diag.lse_p) p.diag.lse_p[j] = np_.lse2 * 0.6931471805599453f;
     // the probability of the row's arg-max: a weight known to take part in a draw from p
@@ -454,12 +459,7 @@ __global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_const
                 best.idx = oi;
             }
         }
-        if (lane == 0) {
-            RacePart out;
-            out.key = best.key;
-            out.idx = best.idx;
-            p.race_part[row * p.race_nchunks + c] = out;
-        }
+        if (lane == 0 && best.key > 0.0f) atomicMax(p.race_best + row, race_pack(best.key, best.idx));
     }
 }
 
@@ -471,16 +471,9 @@ template <typename L>
 __device__ __forceinline__ int race_winner(const SampledParams &p, long long row, bool bonus, long long yrow, int fallback)
 {
     using E = typename L::elem;
-    float key = 0.0f;
-    int g = -1;
-    for (int c = 0; c < p.race_nchunks; ++c) {
-        const RacePart x = p.race_part[row * p.race_nchunks + c];
-        if (x.key > key) {          // chunks ascend: strict keeps the lowest group
-            key = x.key;
-            g = x.idx;
-        }
-    }
-    if (g < 0) return fallback;
+    const unsigned long long top = __ldcg(p.race_best + row);
+    if (top == 0ull) return fallback;
+    const int g = static_cast<int>(0xffffffffu - static_cast<unsigned int>(top & 0xffffffffull));
     const DrawCoef cf = draw_coef(p, row, bonus, yrow);
     const E *zr = sampled_row_ptr<E>(p, row);
     const E *yr = bonus ? zr : sampled_row_ptr<E>(p, yrow);
