@@ -320,11 +320,11 @@ __global__ void __launch_bounds__(1024) ocm_update_kernel(OcmView tb, const int 
 {
     __shared__ CanonScratch sc;
     __shared__ bool last;
-    // When launched programmatically behind the kernel that writes rd / rt, wait for it; and let a
-    // kernel launched programmatically behind this one begin (it waits in turn before it touches the
-    // table).  Both are no-ops for ordinary launches.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Let a kernel launched programmatically behind this one begin (it waits in turn before it touches
+    // the table), and, when launched programmatically behind the kernel that writes rd / rt, wait for
+    // that one.  Both are no-ops for ordinary launches.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const unsigned long long nk0 = __ldcg(&tb.stats->n_keys_start);
     if (nk0 + static_cast<unsigned long long>(n) <= tb.key_limit) {
         const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;

@@ -15,12 +15,14 @@
 // every position passed) and finalises every row that stops there; round 2 races the remaining failed
 // positions and the bonus row of the rows whose first failure was rescued, and finalises those.
 //
-// Six launches (A, A2, B1, C1, B2, C2) plus the memory's update kernel.  Each is launched programmatically behind the one before (its blocks become
-// resident while that one drains); B, C and the decision kernel wait for their predecessor before
-// anything else and only then let their successor in, so at most two of them are resident.  Kernel A
-// reads only the step's inputs and writes only the chunk statistics, which nobody else writes and
-// only this step's decision kernel reads: with step overlap switched on it streams while the previous
-// step's last kernels finish, and waits for them at its end.
+// Six launches (A, A2, B1, C1, B2, C2) plus the memory's update kernel.  Each is launched programmatically
+// behind the one before and waits for it (griddepcontrol.wait) before it reads or writes anything that
+// others share.  B, C and the update kernel let their successor in before they wait, the decision kernel
+// only when it exits.  Kernel A reads only the step's inputs and writes only the chunk statistics, which
+// nobody else writes and only this step's decision kernel reads: with step overlap switched on, the
+// statistics kernel of step n+1 therefore streams from the moment step n's decision kernel has finished,
+// beside that step's races, finalisations and update, and waits for them at its end -- so that its own
+// completion, which the next decision kernel waits for, implies theirs.
 //   A  sampled_stats_kernel    every row of z and y once: max and sum exp(x/T) per chunk
 //   A2 sampled_decide_kernel   per position: normalisers, alpha, the stochastic test
 //   B  sampled_race_kernel     the round's draws (z and y rows again; bonus rows: z only): best group
@@ -163,7 +165,8 @@ __global__ void __launch_bounds__(128) sampled_decide_kernel(const __grid_consta
     const long long n = sampled_rows_z(p);
     const long long j = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
     pdl_wait();
-    pdl_launch_dependents();
+    // no early trigger here: the kernels behind this one let their own successors in at once, down to the
+    // next step's statistics kernel, which overwrites the chunk statistics this kernel is reading
     if (j >= n) return;
     const int K = p.K;
     const long long b = j / (K + 1);
@@ -383,8 +386,8 @@ __global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_const
     const long long draws = sampled_rows_z(p);
     // round 1 has one draw per batch row (tiles run over batch rows), round 2 up to K per pending row
     const long long tiles = (round == 1 ? static_cast<long long>(p.B) : draws) * p.race_nchunks;
-    pdl_wait();
     pdl_launch_dependents();
+    pdl_wait();
     for (long long tile = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < tiles; tile += warps) {
         const long long unit = tile / p.race_nchunks;
         const int c = static_cast<int>(tile - unit * p.race_nchunks);
@@ -510,8 +513,8 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
     const int lane = threadIdx.x & 31;
     const int K = p.K;
     const long long b = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    pdl_wait();
     pdl_launch_dependents();
+    pdl_wait();
     if (b >= p.B) return;
     if (round == 2 && p.row_state[b] == 0) return;       // finalised in round 1
     const long long row0 = b * (K + 1);
