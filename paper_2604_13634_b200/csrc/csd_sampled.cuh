@@ -4,10 +4,12 @@
 //     all accepted: bonus token ~ p_{gamma+1}
 // with p = softmax(z/T), q = softmax(y/T).
 //
-// A categorical draw is an exponential race: argmax_v w(v) / E_v, E_v = -ln(1 - u_v),
-// u_v from one word of Philox4x32-10 keyed by the call's seed, counter (v >> 2, row, 0, 0).
-// A race is one more streaming arg-max: no normaliser, no prefix sums, no second pass over
-// the winner's neighbourhood, and every tile of a row can run independently.
+// A categorical draw is an exponential race: the winner among items with weights W and clocks
+// E ~ Exp(1) is argmax W / E; clocks are E = -ln(1 - u), u from one word of Philox4x32-10 keyed by
+// the call's seed (clock n of stream s of a draw: word n & 3 of counter (n >> 2, row, s, 0)).  It runs
+// in two levels: among the groups of eight consecutive tokens (stream 0), then among the winning
+// group's tokens (stream 1).  A race is one more streaming arg-max: no normaliser, no prefix sums, and
+// every tile of a row can run independently.
 //
 // Algorithm 1 stops a row at its first un-rescued rejection, so most residual draws of a step are never
 // needed: a row's FIRST failed position always is, the later ones only if that one was rescued.  The
@@ -20,13 +22,14 @@
 // others share.  B, C and the update kernel let their successor in before they wait, the decision kernel
 // only when it exits.  Kernel A reads only the step's inputs and writes only the chunk statistics, which
 // nobody else writes and only this step's decision kernel reads: with step overlap switched on, the
-// statistics kernel of step n+1 therefore streams from the moment step n's decision kernel has finished,
-// beside that step's races, finalisations and update, and waits for them at its end -- so that its own
-// completion, which the next decision kernel waits for, implies theirs.
+// statistics kernel of step n+1 may therefore stream as soon as step n's decision kernel has finished
+// and step n's later kernels are all resident (in practice: beside its second round and its update),
+// and waits for them at its end -- so that its own completion, which the next decision kernel waits
+// for, implies theirs.
 //   A  sampled_stats_kernel    every row of z and y once: max and sum exp(x/T) per chunk
 //   A2 sampled_decide_kernel   per position: normalisers, alpha, the stochastic test
 //   B  sampled_race_kernel     the round's draws (z and y rows again; bonus rows: z only): best group
-//                              key per chunk
+//                              key per tile, atomicMax into one word per draw
 //   C  sampled_finalize_kernel per batch row: t*, look-up, gate, prefix scan, outputs
 // followed by the memory's own update kernel on the recorded pairs.
 #pragma once
