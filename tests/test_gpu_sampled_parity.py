@@ -123,6 +123,7 @@ SHAPES = [
     (1, 1, 8, torch.bfloat16, 1.0), (2, 3, 4099, torch.float32, 1.0),          # V % 4 != 0: element-wise path
     (2, 3, 4099, torch.bfloat16, 0.3), (4, 32, 3000, torch.bfloat16, 0.6),     # K at the limit
     (5, 2, 70001, torch.float32, 0.4), (2, 2, 1024 * 33 + 8, torch.bfloat16, 1.0), (1, 7, 262144, torch.float32, 0.25),
+    (300, 3, 100, torch.float32, 0.8), (64, 2, 1000, torch.bfloat16, 0.5),     # many short rows: one tile per row
 ]
 
 
