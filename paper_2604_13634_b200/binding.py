@@ -211,6 +211,27 @@ class Ocm:
         order = torch.argsort(d * (1 << 32) + t)
         return d[order], t[order], c[order]
 
+    def save(self, path: str, stream=None):
+        """Write the stored (draft, target, count) triples, lambda and the slot count to an .npz file:
+        the table of Sec. 4.2 as it is handed from the calibration phase to deployment."""
+        import numpy as np
+        d, t, c = self.export(stream)
+        st = self.stats(stream)
+        np.savez(path, draft=d.numpy().astype(np.int32), target=t.numpy().astype(np.int32),
+                 count=c.numpy().astype(np.uint32), lam=np.uint32(st["lambda"]), n_slots=np.uint64(self.n_slots))
+
+    @classmethod
+    def load(cls, path: str, device: int = 0, n_slots: int = 0, stream=None) -> "Ocm":
+        """A new memory holding the triples of a file written by `save` (n_slots = 0: as saved)."""
+        import numpy as np
+        f = np.load(path)
+        ocm = cls(int(n_slots or f["n_slots"]), int(f["lam"]), device)
+        if len(f["draft"]):
+            dev = ocm.device
+            ocm.import_(torch.from_numpy(f["draft"].astype(np.int32)).to(dev), torch.from_numpy(f["target"].astype(np.int32)).to(dev),
+                        torch.from_numpy(f["count"].astype(np.int64)).to(dev).to(torch.int32), stream)
+        return ocm
+
     def stats(self, stream=None) -> dict:
         s = Stats()
         _check(lib().csd_ocm_stats(self.handle, byref(s), _stream_ptr(stream)), "csd_ocm_stats")

@@ -344,6 +344,28 @@ def test_update_kernel_regimes_and_import_export():
         ocm.close(); other.close()
 
 
+def test_memory_survives_a_file(tmp_path):
+    """Calibration hands its table to deployment through a file (Sec. 4.2, Phase 1): save, load, same triples,
+    same lambda; a smaller table admits the saved pairs in sorted order up to its own limit."""
+    g = torch.Generator(device="cuda").manual_seed(11)
+    ocm = Ocm(4096, 3)
+    d = torch.randint(0, 50, (5000,), generator=g, device="cuda", dtype=torch.int32)
+    t = torch.randint(0, 50, (5000,), generator=g, device="cuda", dtype=torch.int32)
+    ocm.update(d, t)
+    path = str(tmp_path / "table.npz")
+    ocm.save(path)
+    back = Ocm.load(path)
+    assert all(torch.equal(a, b) for a, b in zip(ocm.export(), back.export()))
+    assert back.stats()["lambda"] == 3 and back.n_slots == 4096
+    small = Ocm.load(path, n_slots=256)
+    sd, st_, sc = small.export()
+    fd, ft, fc = ocm.export()
+    assert small.stats()["n_keys"] == 128 and small.stats()["n_dropped"] == len(fd) - 128
+    assert torch.equal(sd, fd[:128]) and torch.equal(st_, ft[:128]) and torch.equal(sc, fc[:128])
+    for o in (ocm, back, small):
+        o.close()
+
+
 def test_host_entry_point_matches_device_entry_point():
     wl = dataclasses.replace(WORKLOADS["batched_serving"], B=6)
     syn = Synth(wl, 2, "cuda")
