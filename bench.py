@@ -387,8 +387,8 @@ def run_ours(args, wl, tau):
 # --mode sampled: the stochastic verification step (Algorithm 1 at T > 0), a separate line
 # ---------------------------------------------------------------------------------------
 def run_sampled(args, wl, tau):
-    """csd_step_sampled (statistics, decision, races, finalisation, memory update: five
-    launches per step) over a ring of resident inputs.  Algorithmic bytes per step: every row of
+    """csd_step_sampled (statistics, decision, two rounds of races and finalisation, memory update:
+    seven launches per step) over a ring of resident inputs.  Algorithmic bytes per step: every row of
     the target and draft logits once, the two rows of every position whose residual draw a row
     needs once more, and the bonus row of every fully accepted batch row once more."""
     import torch
