@@ -285,12 +285,29 @@ __device__ __forceinline__ float draw_weight(const DrawCoef &c, float z, float y
     return fmaxf(w, 0.0f);
 }
 
-// Sum of a group's weights, in a fixed order.
+// Sum of a group's weights, in a fixed order.  The affine part runs on packed pairs (one instruction
+// for two tokens; each half rounds exactly like the scalar operation in draw_weight).
 __device__ __forceinline__ float group_weight(const DrawCoef &c, const float (&z)[8], const float (&y)[8])
 {
+    const unsigned long long s2 = pack2(c.s, c.s);
+    const unsigned long long nmz = pack2(-c.mz, -c.mz), nlp = pack2(-c.lp, -c.lp);
+    const unsigned long long nmy = pack2(-c.my, -c.my), nlq = pack2(-c.lq, -c.lq);
     float w[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) w[e] = draw_weight(c, z[e], y[e]);
+    for (int e = 0; e < 8; e += 2) {
+        float a0, a1;
+        unpack2(fma2(add2(pack2(z[e], z[e + 1]), nmz), s2, nlp), a0, a1);
+        w[e] = ex2_approx(a0);
+        w[e + 1] = ex2_approx(a1);
+        if (c.has_q) {
+            float b0, b1;
+            unpack2(fma2(add2(pack2(y[e], y[e + 1]), nmy), s2, nlq), b0, b1);
+            w[e] -= ex2_approx(b0);
+            w[e + 1] -= ex2_approx(b1);
+        }
+        w[e] = fmaxf(w[e], 0.0f);
+        w[e + 1] = fmaxf(w[e + 1], 0.0f);
+    }
     return ((w[0] + w[1]) + (w[2] + w[3])) + ((w[4] + w[5]) + (w[6] + w[7]));
 }
 
