@@ -174,10 +174,20 @@ __global__ void __launch_bounds__(128) sampled_decide_kernel(const __grid_consta
     const int K = p.K;
     const long long b = j / (K + 1);
     const int i = static_cast<int>(j - b * (K + 1));
-    RowNorm np_ = fold_row_norm(p, j, lane);
-    RowNorm nq = np_;
     const long long pos = b * K + i;
     const long long yrow = n + pos;
+    // the draft token and its two logits do not depend on the folds: requested first
+    int d = -1;
+    float zd = 0.0f, yd = 0.0f;
+    if (i < K) {
+        d = __ldg(p.draft + pos);
+        if (static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V)) {
+            zd = L::load_elem(sampled_row_ptr<E>(p, j), d);
+            yd = L::load_elem(sampled_row_ptr<E>(p, yrow), d);
+        }
+    }
+    RowNorm np_ = fold_row_norm(p, j, lane);
+    RowNorm nq = np_;
     if (i < K) nq = fold_row_norm(p, yrow, lane);
     if (lane != 0) return;
     p.race_best[j] = 0ull;
@@ -200,12 +210,9 @@ __global__ void __launch_bounds__(128) sampled_decide_kernel(const __grid_consta
     }
     if (!(nq.lse2 == nq.lse2) || nq.lse2 == INFINITY || nq.m == -INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
     if (p.diag.lse_q) p.diag.lse_q[pos] = nq.lse2 * 0.6931471805599453f;
-    const int d = __ldg(p.draft + pos);
     float alpha = 0.0f;
     bool ok = false;
     if (static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V)) {
-        const float zd = L::load_elem(sampled_row_ptr<E>(p, j), d);
-        const float yd = L::load_elem(sampled_row_ptr<E>(p, yrow), d);
         // log2 p(d) - log2 q(d) in double (one per position); alpha = min(1, p(d)/q(d))      (Eq. 2)
         const double lr = (static_cast<double>(zd) - static_cast<double>(yd)) * static_cast<double>(p.l2e_T) -
                           (static_cast<double>(np_.lse2) - static_cast<double>(nq.lse2));
