@@ -24,7 +24,10 @@
  *     that the host can see is refused before anything is launched.  Conditions
  *     only the device can see (a NaN logit, a draft id outside [0,V), a full
  *     table) set sticky flags / counters readable with csd_ocm_stats; the device
- *     never traps and never waits on another block.
+ *     never traps.  Within a launch no block waits for another (arrival counters
+ *     only).  With csd_set_overlap on, the warps that finalise a batch row wait for
+ *     the PREVIOUS launch on the stream: a bounded poll (2^14 loads) of a completion
+ *     word, then the hardware's wait for that grid to retire, which always ends.
  *   - Determinism: for fixed (B,K,V,dtype) every output, including the sums s,
  *     is bit-reproducible from run to run.
  */
@@ -237,10 +240,16 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
  *
  * The paper does not say how the draws are made; this library's reading:
  *   - the uniforms r of the acceptance test are an INPUT ([B,K] float, in [0,1));
- *   - a draw from weights w(v) is an exponential race, argmax_v w(v) / E_v (lowest index on
- *     ties) with E_v = -ln(1 - u_v), u_v = (j + 1/2) / 2^23, j = the top 23 bits of word
- *     (v & 3) of Philox4x32-10 (Salmon et al., SC'11) under key (seed low, seed high) and
- *     counter (v >> 2, b*(K+1)+i, 0, 0); i = K is the bonus draw.  P(v) = w(v) / sum w.
+ *   - a draw from weights w(v) is an exponential race, argmax w / E (lowest index on ties),
+ *     run in TWO levels: first among the groups of 8 consecutive tokens (group g = tokens
+ *     8g .. 8g+7, tokens at or beyond V weigh 0, group weight W_g = the sum of its tokens'
+ *     weights), then among the 8 tokens of the winning group.  P(v) = W_g / sum W * w(v) / W_g
+ *     = w(v) / sum w.  Clocks: E = -ln(1 - u), u = (j + 1/2) / 2^23, j = the top 23 bits of a
+ *     32-bit word of Philox4x32-10 (Salmon et al., SC'11) under key (seed low, seed high);
+ *     clock number n of stream s of the draw of row = b*(K+1)+i (i = K: the bonus draw) is word
+ *     (n & 3) of counter (n >> 2, row, s, 0).  Group g uses clock g of stream 0; token v of the
+ *     winning group uses clock v of stream 1.  The group size and the clock grid are part of
+ *     this contract: a caller can reproduce every drawn token from (seed, b, i) and the logits.
  * Draws are made only where a row can need them: for its first failed position, for the later failed
  * positions if that one was rescued, and the bonus draw if every position went through; diag.t_star and
  * diag.bonus are -1 where no draw was made (never at a position the row reaches).

@@ -24,10 +24,14 @@ Readings (the paper leaves these open; each is a convention of this build):
       no normaliser, no prefix sum and no second pass, and the integer it returns is
       well conditioned: it can only change when two keys nearly coincide.  (An
       inverse-CDF draw would make the index depend on rounding in a 150 000-term
-      prefix sum.)  The race is run in two levels: first among the groups of GROUP = 8
+      prefix sum.)  `draw_plain` is that race as the textbooks state it: one level,
+      one clock per token, arg-max over the whole vocabulary.  `draw`, the one the
+      step uses, runs it in two levels: first among the groups of GROUP = 8
       consecutive tokens (weight = the sum of the group), then among the tokens of
-      the winning group: P(v) = W_g / sum W * w(v) / W_g = w(v) / sum w.  One random
-      number per eight tokens is what makes the draw cheap.
+      the winning group: P(v) = W_g / sum W * w(v) / W_g = w(v) / sum w.  The two are
+      different maps from a seed to a token and the same sampler; the tests pin them
+      to each other and to w / sum w as distributions.  GROUP and the clock grid of
+      S3 are frozen: they are part of the seed-to-token contract of the C header.
   S3  a clock is E = -ln(1 - u), u = (j + 1/2) / 2^23, j = the top 23 bits of one
       32-bit word (so that u and 1 - u are exact in binary32 as well) of
       Philox4x32-10 (Salmon et al., "Parallel random numbers: as easy as 1, 2, 3",
@@ -147,6 +151,22 @@ def draw(p, q, seed: int, row: int, fallback: int):
     hi_t[t] = 0.0
     clear = lo[g].sum() / e_g[g] > np.max(hi_g) and lo[g, t] / e_t[t] > np.max(hi_t)
     return g * GROUP + t, bool(clear)
+
+
+PLAIN_STREAM = 2      # the clocks of draw_plain: a stream of their own, one clock per token
+
+
+def draw_plain(p, q, seed: int, row: int, fallback: int) -> int:
+    """One draw from norm(max(0, p - q)) (q None: from p) by the ONE-level exponential race (S2):
+    argmax_v w(v) / E_v over the whole vocabulary, lowest index on ties, clock v of stream
+    PLAIN_STREAM of the draw's row; `fallback` if every weight is zero (S7).
+
+    The reference statement of the categorical draws of Algorithm 1 (t* ~ norm(max(0, p - q)) and
+    t ~ p_{gamma+1}).  `verify` does not call it: it exists so that the two-level `draw` can be
+    pinned to the plain definition as a sampler of the same distribution."""
+    w = _weights(p, q)
+    t, _ = race(w, race_clocks(seed, row, PLAIN_STREAM, 0, len(w)), -1)
+    return int(fallback) if t < 0 else t
 
 
 # ----------------------------------------------------------------------------

@@ -242,7 +242,31 @@ def pin_unclear_draws_are_flagged(mod):
     assert t == 0 and not clear
 
 
-PINS = [pin_philox_known_answers, pin_alpha_and_normalisers, pin_update_semantics, pin_unclear_draws_are_flagged,
+def pin_plain_draw_is_the_textbook_race(mod):
+    """draw_plain written out: arg-max of w / E over all tokens, one clock per token of its own stream."""
+    rng = np.random.default_rng(8)
+    p = rng.random(37); p /= p.sum()
+    q = rng.random(37); q /= q.sum()
+    for row in range(50):
+        e = mod.race_clocks(5, row, mod.PLAIN_STREAM, 0, 37)
+        assert mod.draw_plain(p, None, 5, row, 0) == int(np.argmax(p / e))
+        w = np.maximum(0.0, p - q)
+        assert mod.draw_plain(p, q, 5, row, 0) == int(np.argmax(w / e)) and w[mod.draw_plain(p, q, 5, row, 0)] > 0
+    assert mod.draw_plain(p, p, 5, 0, fallback=7) == 7                    # S7
+    # a short statistical check of both samplers against each other (the long one is its own test)
+    w = np.array([0.0, 3.0, 1.0, 0.0, 6.0, 2.0e-3, 1.0, 1.0,  0.5, 0.0, 0.0, 4.0, 0.0, 0.0, 0.0, 2.5,  0.0, 5.0, 1.0])
+    pr = w / w.sum()
+    n = 6000
+    a = np.zeros(19); b = np.zeros(19)
+    for s in range(n):
+        a[mod.draw(pr, None, 17, s, 0)[0]] += 1
+        b[mod.draw_plain(pr, None, 17, s, 0)] += 1
+    sd = np.sqrt(pr * (1 - pr) / n)
+    assert np.all(np.abs(a / n - pr) < 4 * sd + 1e-9) and np.all(np.abs(b / n - pr) < 4 * sd + 1e-9)
+    assert np.all(np.abs(a - b) / n < 4 * np.sqrt(2) * sd + 1e-9)
+
+
+PINS = [pin_philox_known_answers, pin_plain_draw_is_the_textbook_race, pin_alpha_and_normalisers, pin_update_semantics, pin_unclear_draws_are_flagged,
         pin_gate_is_temperature_free_and_may_exceed_one, pin_greedy_limit, pin_clocks_are_exponential,
         pin_race_draws_from_the_weights, pin_lossless_without_rescue]
 
@@ -274,6 +298,13 @@ MUTANTS = [
      "            if is_freq and is_safe:\n                rescued[b, i] = 1\n                continue\n            rej_d[b, i] = d\n            rej_t[b, i] = tt"),
     ("frequency test strict", "is_freq = cnt[b, i] >= ocm.lam", "is_freq = cnt[b, i] > ocm.lam"),
     ("bonus row shares the clocks of row 0", "row = b * K1 + i", "row = b * K1 + (0 if i == K else i)"),
+    ("group size differs between the two levels", "return g * GROUP + t, bool(clear)", "return g * (GROUP // 2) + t, bool(clear)"),
+    ("second level races half a group", "e_t = race_clocks(seed, row, 1, g * GROUP, GROUP)\n    t, _ = race(w[g], e_t, 0)",
+     "e_t = race_clocks(seed, row, 1, g * GROUP, GROUP)\n    t, _ = race(w[g][:GROUP // 2], e_t[:GROUP // 2], 0)"),
+    ("first level groups by four", "def _by_group(w):\n    pad = (-len(w)) % GROUP\n    return np.concatenate([w, np.zeros(pad)]).reshape(-1, GROUP)",
+     "def _by_group(w):\n    pad = (-len(w)) % 4\n    return np.concatenate([w, np.zeros(pad)]).reshape(-1, 4)"),
+    ("plain draw ignores the draft distribution", "    w = _weights(p, q)\n    t, _ = race(w, race_clocks(seed, row, PLAIN_STREAM", "    w = _weights(p, None)\n    t, _ = race(w, race_clocks(seed, row, PLAIN_STREAM"),
+    ("plain draw shares one clock per group", "race_clocks(seed, row, PLAIN_STREAM, 0, len(w)), -1)", "np.repeat(race_clocks(seed, row, PLAIN_STREAM, 0, len(w)), GROUP)[:len(w)], -1)"),
     ("normaliser without max shift", "lse = m + np.log(np.sum(np.exp(x - m)))", "lse = np.log(np.sum(np.exp(x - m)))"),
 ]
 
@@ -300,3 +331,78 @@ def test_planted_mistakes(name, old, new):
             caught.append(pin.__name__)
             break
     assert caught, f"no pin notices the planted mistake: {name}"
+
+
+# ---------------------------------------------------------------------------------------
+# the two-level draw and the plain one-level draw are the same sampler (100 000 draws each)
+# ---------------------------------------------------------------------------------------
+N_DRAWS = 100_000
+
+
+def _case_distributions(V, form):
+    rng = np.random.default_rng(1000 + V)
+    p = 0.2 + rng.random(V)
+    p[rng.random(V) < 0.1] = 0.0                 # tokens that can never be drawn
+    p[V - 1] = 1.0                               # the ragged last group takes part (19 and 1000 are not multiples of 8)
+    p /= p.sum()
+    if form == "bonus":                          # t ~ p_{gamma+1}
+        return p, None
+    q = 0.2 + rng.random(V)                      # t* ~ norm(max(0, p - q))
+    q[V - 1] = 0.0
+    q /= q.sum()
+    return p, q
+
+
+def _count_draws(job):
+    kind, V, form, lo, hi = job
+    p, q = _case_distributions(V, form)
+    counts = np.zeros(V, dtype=np.int64)
+    for row in range(lo, hi):
+        t = ORACLE.draw(p, q, 2024, row, 0)[0] if kind == "two_level" else ORACLE.draw_plain(p, q, 2024, row, 0)
+        counts[t] += 1
+    return kind, counts
+
+
+@pytest.mark.parametrize("form", ["residual", "bonus"])
+@pytest.mark.parametrize("V", [19, 64, 1000])
+def test_two_level_draw_and_plain_draw_sample_the_same_distribution(V, form):
+    """Algorithm 1 asks for t* ~ norm(max(0, p - q)) and t ~ p_{gamma+1}.  draw_plain is the textbook
+    exponential race for that; draw is the two-level form the step uses.  Over 100 000 draws each, every
+    token's frequency is within 4 sigma of w / sum w for both (see the note at the check), the chi-square
+    statistics stay below their mean + 5 sd, and so does the two-sample statistic between them."""
+    import concurrent.futures as cf
+    import multiprocessing as mp
+    workers = max(1, min(8, os.cpu_count() or 1))
+    step = -(-N_DRAWS // (4 * workers))
+    jobs = [(kind, V, form, lo, min(N_DRAWS, lo + step)) for kind in ("two_level", "plain") for lo in range(0, N_DRAWS, step)]
+    counts = {"two_level": np.zeros(V, dtype=np.int64), "plain": np.zeros(V, dtype=np.int64)}
+    with cf.ProcessPoolExecutor(workers, mp_context=mp.get_context("spawn")) as pool:
+        for kind, c in pool.map(_count_draws, jobs):
+            counts[kind] += c
+    p, q = _case_distributions(V, form)
+    w = np.maximum(0.0, p - (q if q is not None else 0.0))
+    pr = w / w.sum()
+    n = N_DRAWS
+    sd = np.sqrt(pr * (1 - pr) / n)
+    live = pr > 0
+    assert live.sum() >= V // 3 and pr[V - 1] > 0
+    for kind, c in counts.items():
+        assert c.sum() == n and np.all(c[~live] == 0), kind
+        zs = np.abs(c / n - pr)[live] / sd[live]
+        # 4 sigma per token; among the ~900 live tokens of the largest case 4 sigma excursions are no longer
+        # rare (one in ten runs), so there a single token may go up to 5 sigma
+        assert np.all(zs < 4.0) or (V > 64 and np.sum(zs >= 4.0) == 1 and zs.max() < 5.0), (kind, np.sort(zs)[-3:])
+    # chi-square with the rare tokens pooled (expected count < 10)
+    rare = live & (pr * n < 10)
+    bins = [np.flatnonzero(live & ~rare)] if not rare.any() else [np.flatnonzero(live & ~rare), np.flatnonzero(rare)]
+    def pooled(x):
+        return np.concatenate([x[bins[0]]] + [[x[b].sum()] for b in bins[1:]])
+    e = pooled(pr * n)
+    k = len(e)
+    bound = (k - 1) + 5 * math.sqrt(2 * (k - 1))
+    for kind, c in counts.items():
+        chi = float(np.sum((pooled(c.astype(np.float64)) - e) ** 2 / e))
+        assert chi < bound, (kind, chi, bound)
+    a, b = pooled(counts["two_level"].astype(np.float64)), pooled(counts["plain"].astype(np.float64))
+    chi2 = float(np.sum((a - b) ** 2 / (a + b + 1e-300)))
+    assert chi2 < bound, (chi2, bound)
