@@ -133,7 +133,7 @@ class OracleRunner:
     def __init__(self, wl, tau, rows_b):
         import dataclasses
         from oracle import csd_oracle, row_stats_c
-        from paper_2604_13634_b200.synth import Synth, logits_bits_numpy
+        from synth_inputs import Synth, logits_bits_numpy
         self.o, self.rs = csd_oracle, row_stats_c
         self.wl = dataclasses.replace(wl, B=rows_b)
         self.tau = tau
@@ -208,10 +208,12 @@ def run_reference(args, wl, tau):
 # the GPU leg
 # ---------------------------------------------------------------------------------------
 class Bench:
+    """One workload's resident inputs, memory and buffers, and the launch plans that replay them."""
+
     def __init__(self, wl, tau, device, seed=0):
         import torch
         import paper_2604_13634_b200 as pkg
-        from paper_2604_13634_b200.synth import Synth
+        from synth_inputs import Synth
         self.torch, self.pkg, self.wl, self.tau = torch, pkg, wl, tau
         self.device = device
         l2 = torch.cuda.get_device_properties(device).L2_cache_size
@@ -228,38 +230,53 @@ class Bench:
                 z, d = self.ring[s % self.ring_len]
                 pkg.csd_step(z, d, self.ocm, tau, self.buf)
         torch.cuda.synchronize(device)
-        self.graph = None
+        self.plan = None          # [(graph, replays)], together exactly the planned number of steps
+        self.plan_steps = 0
+        self.plan_label = "eager"
 
     def step(self, i):
         z, d = self.ring[i % self.ring_len]
         self.pkg.csd_step(z, d, self.ocm, self.tau, self.buf)
 
-    def capture(self, min_steps=48):
-        """A CUDA graph of whole passes over the ring, at least `min_steps` steps long (the
-        launches are captured, not changed).  Consecutive steps overlap only inside one graph
-        launch, so a short graph would spend a large share of its time on its own start and
-        drain."""
+    def _graph_of(self, n):
         torch = self.torch
-        self.graph_steps = self.ring_len * max(1, math.ceil(min_steps / self.ring_len))
         side = torch.cuda.Stream(self.device)
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
-            self.step(0)
+            self.step(0)              # outside the capture: first-use set-up (a workspace clear) must not be captured
         torch.cuda.current_stream().wait_stream(side)
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
-            for i in range(self.graph_steps):
+            for i in range(n):
                 self.step(i)
-        self.graph = g
+        return g
+
+    def plan_steps_exactly(self, steps, graph_steps=48):
+        """CUDA graphs that together enqueue EXACTLY `steps` steps: as many replays of one graph of about
+        `graph_steps` steps as fit (consecutive steps overlap only inside one graph launch, so a short graph
+        spends a large share of its time on its own start and drain), plus one shorter graph for the rest."""
+        replays = max(1, steps // max(1, graph_steps))
+        per = steps // replays
+        rest = steps - per * replays
+        self.plan = [(self._graph_of(per), replays)]
+        self.plan_label = f"CUDA graph of {per} steps replayed {replays}x"
+        if rest:
+            self.plan.append((self._graph_of(rest), 1))
+            self.plan_label += f" + one graph of {rest} steps"
+        self.plan_steps = steps
 
     def run(self, steps):
-        """Enqueue `steps` steps: whole-graph replays, then the remainder eagerly."""
-        if self.graph is not None:
-            while steps >= self.graph_steps:
-                self.graph.replay()
-                steps -= self.graph_steps
+        """Enqueue `steps` steps through the plan (which must have been made for that count), else eagerly."""
+        if self.plan is not None and steps == self.plan_steps:
+            for g, n in self.plan:
+                for _ in range(n):
+                    g.replay()
+            return
         for i in range(steps):
             self.step(i)
+
+    def launch_label(self, steps):
+        return self.plan_label if (self.plan is not None and steps == self.plan_steps) else "eager"
 
     def timed(self, steps):
         torch = self.torch
@@ -271,11 +288,51 @@ class Bench:
         return a.elapsed_time(b) * 1e-3
 
 
+def repeats_for(region_s, floor=7, target_s=0.25, cap=201):
+    """How often the timed region is repeated: at least `floor` times, more while the whole stays near
+    `target_s` (a region of a few milliseconds alone would see one clock sample)."""
+    if region_s <= 0:
+        return floor
+    return int(max(floor, min(cap, math.ceil(target_s / region_s))))
+
+
+def read_stream_gbs(device):
+    """Context for the roofline: a read-only stream (torch.sum over 2 GiB of fp32, best of 5) next to the
+    read+write copy that MEASURED_PEAKS.json holds."""
+    import torch
+    x = torch.empty(1 << 29, dtype=torch.float32, device=device).normal_()
+    best = 0.0
+    for _ in range(6):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        x.sum()
+        b.record()
+        b.synchronize()
+        best = max(best, x.numel() * 4 / (a.elapsed_time(b) * 1e-3) / 1e9)
+    del x
+    torch.cuda.empty_cache()
+    return best
+
+
+def standalone_us(pkg, bench, steps=96):
+    """Latency of a step that runs alone: overlap off (stream-ordered launches, the 4-blocks-per-SM shape),
+    a graph of `steps` steps over the ring, median of 7 replays."""
+    import torch
+    pkg.csd_set_overlap(False)
+    try:
+        bench.plan_steps_exactly(steps, steps)
+        bench.run(steps)
+        torch.cuda.synchronize(bench.device)
+        return 1e6 * statistics.median(bench.timed(steps) for _ in range(7)) / steps
+    finally:
+        bench.plan = None
+
+
 def time_e2e(wl, tau, device, steps):
     """csd_step_host: pinned host inputs, copies inside the timed region."""
     import torch
     import paper_2604_13634_b200 as pkg
-    from paper_2604_13634_b200.synth import Synth
+    from synth_inputs import Synth
     syn = Synth(wl, 0, device)
     host = []
     for s in range(2):
@@ -318,27 +375,38 @@ def run_ours(args, wl, tau):
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
 
-    pkg.csd_set_overlap(not args.no_overlap)
+    overlap = not args.no_overlap
+    pkg.csd_set_overlap(overlap)
     pkg.csd_set_tuning(args.chunk_bytes, args.ctas_per_sm, args.block_threads)
     bench = Bench(wl, tau, device, seed=rank)
-    use_graph = not args.eager
-    if use_graph:
-        bench.capture(args.graph_steps)
+    if not args.eager:
+        bench.plan_steps_exactly(args.steps, args.graph_steps)
     warm = max(args.warmup, 3)
-    bench.run(warm)
+    for i in range(warm):                 # warm-up steps are launched one by one
+        bench.step(i)
+    bench.run(args.steps)                 # and the plan itself once
     torch.cuda.synchronize(device)
 
-    sampler = ClockSampler(local)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize(device)
+    # the timed region (exactly --steps steps, barrier + synchronize on both sides, max over ranks) is
+    # taken several times back to back; the line reports the median region
+    probe = bench.timed(args.steps)
+    repeats = args.repeats if args.repeats > 0 else repeats_for(probe)
+    sampler = ClockSampler(local, period_s=0.005)
     sampler.start()
-    sec = bench.timed(args.steps)
-    torch.cuda.synchronize(device)
+    regions = []
+    for _ in range(repeats):
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+        sec_r = bench.timed(args.steps)
+        torch.cuda.synchronize(device)
+        if world > 1:
+            dist.barrier()
+        sec_r, positions = reduce_over_ranks(sec_r, wl.B * wl.K * args.steps, dist if world > 1 else None, device)
+        regions.append(sec_r)
     clocks = sampler.stop()
-    if world > 1:
-        dist.barrier()
-    sec, positions = reduce_over_ranks(sec, wl.B * wl.K * args.steps, dist if world > 1 else None, device)
+    sec = statistics.median(regions)
+    launch = bench.launch_label(args.steps)
 
     st = bench.ocm.stats()
     e2e = time_e2e(wl, tau, device, steps=max(3, min(args.steps, args.e2e_steps)))
@@ -354,31 +422,51 @@ def run_ours(args, wl, tau):
             "metric": METRIC, "value": positions / sec, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": warm, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "repeats": repeats, "value_min": positions / max(regions), "value_max": positions / min(regions),
+            "region_ms": {"median": 1e3 * sec, "min": 1e3 * min(regions), "max": 1e3 * max(regions)},
             "config": workload_config(wl, tau, {
                 "steps_per_s": args.steps * world / sec, "parallelism": f"replicas x{world}",
                 "l2_policy": f"ring of {bench.ring_len} distinct step inputs "
                              f"({bench.ring_len * wl.logit_bytes / 1e6:.0f} MB, > 2x L2)",
-                "launch": ("CUDA graph of %d steps replayed" % bench.graph_steps) if use_graph else "eager",
-                "step_overlap": "off" if args.no_overlap else
+                "launch": launch,
+                "timing": f"the region of exactly {args.steps} steps timed {repeats} times back to back; value = median",
+                "step_overlap": "off" if not overlap else
                                 "programmatic dependent launch, one block per SM and launch: a step streams its "
                                 "logits while the steps before it finish",
                 "kernel_shape": shape}),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "peak_source": f"of {peak_kind}",
+                         "peak_kind": "read+write copy; this kernel only reads, so a fraction slightly above 1 is possible",
                          "kernel": "csd_step_kernel", "bytes_per_launch": wl.logit_bytes,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "e2e": e2e, "gpu_launches": args.steps, "clocks": clocks,
             "ocm": {k: st[k] for k in ("n_keys", "n_dropped", "steps", "matches", "rescues", "rejections", "flags")},
         }
+        if world == 1 and not args.lean:
+            line["roofline"]["read_stream_GBs_torch_sum"] = read_stream_gbs(device)
+            us = standalone_us(pkg, bench)
+            line["roofline"]["single_step"] = {
+                "us_per_step": us, "achieved": wl.logit_bytes / us / 1e3, "frac": wl.logit_bytes / us / 1e3 / peak,
+                "what": "a step that runs alone: overlap off, stream-ordered launches, 4 blocks per SM"}
+            pkg.csd_set_overlap(overlap)
         if not args.no_cpu_baseline and world == 1:
             r = time_oracle(wl, tau)
             line["cpu_baseline"] = {"value": r["positions_per_s"], "unit": UNIT, "cores": r["cores"], "kind": "oracle",
                                     "sample": f"{r['steps']} oracle steps over {r['rows_b']} of the workload's {wl.B} "
                                               f"batch rows (CPU-generated inputs, same recipe) in {r['seconds']:.1f} s"}
-        if args.extras and world == 1:
-            line["other_workloads"] = run_extras(device, wl.name, peak)
+        bench.ocm.close()
+        del bench
+        torch.cuda.empty_cache()
+        if world == 1 and not args.lean:
+            names = ("batched_serving", "large_batch", "ocm_contention") + (("single_stream", "tiny") if args.extras else ())
+            line["other_workloads"] = run_extras(device, wl.name, peak, names, overlap)
+            try:
+                line["sampled"] = measure_sampled(args, wl, tau, device, graph_steps=16, min_steps=48, count_draws=True)
+            except Exception as e:             # the greedy line stands on its own
+                line["sampled"] = {"error": repr(e)}
         print(json.dumps(line), flush=True)
-    bench.ocm.close()
+    else:
+        bench.ocm.close()
     if world > 1:
         dist.destroy_process_group()
 
@@ -386,22 +474,16 @@ def run_ours(args, wl, tau):
 # ---------------------------------------------------------------------------------------
 # --mode sampled: the stochastic verification step (Algorithm 1 at T > 0), a separate line
 # ---------------------------------------------------------------------------------------
-def run_sampled(args, wl, tau):
-    """csd_step_sampled (statistics, decision, two rounds of races and finalisation, memory update:
-    seven launches per step) over a ring of resident inputs.  Algorithmic bytes per step: every row of
-    the target and draft logits once, the two rows of every position whose residual draw a row
-    needs once more, and the bonus row of every fully accepted batch row once more."""
+def measure_sampled(args, wl, tau, device, graph_steps, min_steps, count_draws=True):
+    """csd_step_sampled (statistics + decision, races + finalisation, memory update) over a ring of resident
+    inputs.  Algorithmic bytes per step: every row of the target and draft logits once, the two rows of
+    every position whose residual draw a row needs once more, and the bonus row of every fully accepted
+    batch row once more."""
     import torch
 
     import paper_2604_13634_b200 as pkg
-    from paper_2604_13634_b200.synth import Synth
+    from synth_inputs import Synth
 
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
-    pkg.lib()
-    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
-    torch.cuda.set_device(device)
-    pkg.csd_set_overlap(not args.no_overlap)     # a step's statistics kernel may run beside the previous step's tail
     T = args.temperature
     syn = Synth(wl, 0, device)
     step_bytes = (wl.rows + wl.B * wl.K) * wl.V * wl.elt_bytes
@@ -421,7 +503,7 @@ def run_sampled(args, wl, tau):
         z, y, d, r = ring[i % ring_len]
         pkg.csd_step_sampled(z, y, d, r, 1000 + i % ring_len, T, ocm, tau, buf)
 
-    graph_steps = ring_len * max(1, math.ceil(args.graph_steps / ring_len))
+    graph_steps = ring_len * max(1, math.ceil(graph_steps / ring_len))
     side = torch.cuda.Stream(device)
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
@@ -431,20 +513,23 @@ def run_sampled(args, wl, tau):
     with torch.cuda.graph(g):
         for i in range(graph_steps):
             step(i)
-    steps = max(graph_steps, args.steps - args.steps % graph_steps)
+    steps = max(graph_steps, min_steps - min_steps % graph_steps)
     for _ in range(max(1, math.ceil(max(args.warmup, 3) / graph_steps))):
         g.replay()
     torch.cuda.synchronize(device)
-    sampler = ClockSampler(device.index)
+    sampler = ClockSampler(device.index, period_s=0.005)
     sampler.start()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for _ in range(steps // graph_steps):
-        g.replay()
-    b.record()
-    b.synchronize()
+    regions = []
+    for _ in range(7):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps // graph_steps):
+            g.replay()
+        b.record()
+        b.synchronize()
+        regions.append(a.elapsed_time(b) * 1e-3)
     clocks = sampler.stop()
-    sec = a.elapsed_time(b) * 1e-3
+    sec = statistics.median(regions)
     # how many draws a step makes depends on the memory (rescues let rows go on): counted on one more pass
     # over the ring with the memory as the timed region left it
     failed, draws, bonus = [], [], []
@@ -460,26 +545,52 @@ def run_sampled(args, wl, tau):
     peak, peak_kind = measured_peak()
     achieved = algo_bytes * steps / sec / 1e9
     st = ocm.stats()
-    line = {"metric": METRIC, "value": wl.B * wl.K * steps / sec, "unit": UNIT, "n_gpus": 1, "steps": steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * sec / steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+    ocm.close()
+    launches = pkg.sampled_launches_per_step()
+    return {"positions_per_s": wl.B * wl.K * steps / sec, "us_per_step": 1e6 * sec / steps, "steps": steps, "repeats": 7,
+            "temperature": T, "achieved_GBs": achieved, "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+            "algorithmic_bytes_per_step": algo_bytes, "failed_positions_per_step": mean(failed),
+            "residual_draws_per_step": mean(draws), "bonus_draws_per_step": mean(bonus),
+            "launches_per_step": launches, "launch": f"CUDA graph of {graph_steps} steps replayed",
+            "ring_len": ring_len, "step_bytes": step_bytes, "clocks": clocks,
+            "ocm": {k: st[k] for k in ("n_keys", "n_dropped", "steps", "matches", "rescues", "rejections", "flags")}}
+
+
+def run_sampled(args, wl, tau):
+    """--mode sampled: the stochastic verification step (Algorithm 1 at T > 0) as a bench line of its own."""
+    import torch
+
+    import paper_2604_13634_b200 as pkg
+    from synth_inputs import Synth
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    pkg.lib()
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    pkg.csd_set_overlap(not args.no_overlap)     # a step's statistics kernel may run beside the previous step's tail
+    m = measure_sampled(args, wl, tau, device, graph_steps=args.graph_steps, min_steps=args.steps)
+    T = args.temperature
+    line = {"metric": METRIC, "value": m["positions_per_s"], "unit": UNIT, "n_gpus": 1, "steps": m["steps"],
+            "warmup": max(args.warmup, 3), "ms_per_step": m["us_per_step"] * 1e-3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "repeats": m["repeats"],
             "config": workload_config(wl, tau, {
                 "mode": f"stochastic verification (Algorithm 1 at T={T}): acceptance test, residual and bonus draws",
                 "draft_logits": "target logits + N(0, 0.3^2), the draft token raised to the row maximum + 1",
-                "l2_policy": f"ring of {ring_len} distinct step inputs ({ring_len * step_bytes / 1e6:.0f} MB, > 2x L2)",
-                "launch": "CUDA graph of %d steps (7 launches each) replayed" % graph_steps,
-                "failed_positions_per_step": mean(failed), "residual_draws_per_step": mean(draws),
-                "bonus_draws_per_step": mean(bonus)}),
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_source": f"of {peak_kind}",
+                "l2_policy": f"ring of {m['ring_len']} distinct step inputs ({m['ring_len'] * m['step_bytes'] / 1e6:.0f} MB, > 2x L2)",
+                "launch": m["launch"] + f" ({m['launches_per_step']} launches per step)",
+                "failed_positions_per_step": m["failed_positions_per_step"],
+                "residual_draws_per_step": m["residual_draws_per_step"],
+                "bonus_draws_per_step": m["bonus_draws_per_step"]}),
+            "roofline": {"bound": "hbm", "achieved": m["achieved_GBs"], "peak": measured_peak()[0], "unit": "GB/s",
+                         "frac": m["frac"], "traffic": None, "peak_source": m["peak_source"],
                          "kernel": "sampled_stats_kernel + sampled_race_kernel (whole step)",
-                         "bytes_per_launch": algo_bytes},
-            "gpu_launches": 7 * steps, "clocks": clocks,
-            "ocm": {k: st[k] for k in ("n_keys", "n_dropped", "steps", "matches", "rescues", "rejections", "flags")}}
+                         "bytes_per_launch": m["algorithmic_bytes_per_step"]},
+            "gpu_launches": m["launches_per_step"] * m["steps"], "clocks": m["clocks"], "ocm": m["ocm"]}
     if not args.no_cpu_baseline:
         import dataclasses
         from oracle import csd_sampled_oracle as so
-        from paper_2604_13634_b200.synth import logits_to_numpy
+        from synth_inputs import logits_to_numpy
         rows_b = min(wl.B, 2)
         small = dataclasses.replace(wl, B=rows_b)
         z, y, d, r = Synth(small, 0, "cpu").step_sampled(0)
@@ -494,31 +605,38 @@ def run_sampled(args, wl, tau):
         line["cpu_baseline"] = {"value": rows_b * wl.K * n / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
                                 "sample": f"{n} oracle steps over {rows_b} of the workload's {wl.B} batch rows in {secs:.1f} s"}
     print(json.dumps(line), flush=True)
-    ocm.close()
 
 
-def run_extras(device, skip, peak):
-    """Short device-resident runs of the other workloads (extra keys, not bench lines)."""
+def run_extras(device, skip, peak, names, overlap):
+    """Short device-resident runs of the other workloads (extra keys, not bench lines): the pipelined loop
+    (about a quarter of a second, median of 7 regions) and the latency of a step that runs alone."""
     import torch
-    from paper_2604_13634_b200.synth import WORKLOADS
+    import paper_2604_13634_b200 as pkg
+    from synth_inputs import WORKLOADS
     out = {}
-    for name in ("batched_serving", "large_batch", "ocm_contention", "single_stream", "tiny"):
+    for name in names:
         if name == skip:
             continue
         wl = WORKLOADS[name]
+        pkg.csd_set_overlap(overlap)
         b = Bench(wl, wl.taus[0], device)
-        b.capture()
-        b.run(50)
+        steps = 960 if wl.logit_bytes > 100e6 else 1920
+        b.plan_steps_exactly(steps, 48)
+        b.run(steps)
         torch.cuda.synchronize(device)
-        steps = 4000 if wl.logit_bytes > 100e6 else 20000
-        steps -= steps % b.graph_steps
-        sec = b.timed(steps)
+        sec = statistics.median(b.timed(steps) for _ in range(7))
+        launch = b.launch_label(steps)
+        alone = standalone_us(pkg, b)
         out[name] = {"positions_per_s": wl.B * wl.K * steps / sec, "us_per_step": 1e6 * sec / steps,
                      "achieved_GBs": wl.logit_bytes * steps / sec / 1e9,
-                     "frac_of_measured_peak": wl.logit_bytes * steps / sec / 1e9 / peak, "steps": steps}
+                     "frac_of_measured_peak": wl.logit_bytes * steps / sec / 1e9 / peak, "steps": steps, "repeats": 7,
+                     "launch": launch, "logit_bytes_per_step": wl.logit_bytes,
+                     "single_step": {"us_per_step": alone, "achieved_GBs": wl.logit_bytes / alone / 1e3,
+                                     "frac_of_measured_peak": wl.logit_bytes / alone / 1e3 / peak}}
         b.ocm.close()
         del b
         torch.cuda.empty_cache()
+    pkg.csd_set_overlap(overlap)
     return out
 
 
@@ -539,13 +657,16 @@ def main():
     ap.add_argument("--graph-steps", type=int, default=48, help="least number of steps captured into the replayed graph")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--extras", action="store_true", help="also time the other workloads (extra keys, same line)")
+    ap.add_argument("--extras", action="store_true", help="also time the two B = 1 workloads (extra keys, same line)")
+    ap.add_argument("--lean", action="store_true", help="only the headline measurement: no other workloads, no stand-alone "
+                                                         "latency, no stochastic sub-record")
+    ap.add_argument("--repeats", type=int, default=0, help="how often the timed region is taken (0 = automatic, at least 7)")
     ap.add_argument("--mode", default="greedy", choices=["greedy", "sampled"],
                     help="sampled: the stochastic verification step (its own JSON line; 1 GPU)")
     ap.add_argument("--temperature", type=float, default=0.3, help="T of --mode sampled")
     args = ap.parse_args()
 
-    from paper_2604_13634_b200.synth import WORKLOADS
+    from synth_inputs import WORKLOADS
     wl = WORKLOADS[args.workload]
     tau = wl.taus[0] if args.tau is None else args.tau
     if args.impl == "reference":

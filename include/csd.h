@@ -62,6 +62,11 @@ typedef enum { CSD_F32 = 0, CSD_BF16 = 1 } csd_dtype_t;
 #define CSD_FLAG_BAD_DRAFT      0x2u  /* a draft id outside [0, V) was seen                            */
 #define CSD_FLAG_PROBE_EXHAUSTED 0x4u /* a hash probe visited every slot (cannot happen below capacity) */
 #define CSD_FLAG_COUNT_SATURATED 0x8u /* a count reached 2^32 - 1                                      */
+#define CSD_FLAG_INTERNAL       0x10u /* an index check inside the library failed: a bug of the library,
+                                         the step's results are unreliable (csd_stats_t.debug_site says
+                                         which check).  The access was skipped; nothing trapped.  One
+                                         check (a partial-result slot) is always compiled in; a library
+                                         built with -DCSD_DEBUG checks every index it computes.        */
 
 /* Optional per-position diagnostics.  Any member may be NULL.  Row arrays have
  * B*(K+1) entries, position arrays B*K, both row-major.  Values are defined for
@@ -90,6 +95,8 @@ typedef struct {
     uint64_t rejections;    /* pairs handed to the memory update                     */
     uint32_t lambda;        /* frequency threshold in force                          */
     uint32_t flags;         /* CSD_FLAG_* (sticky until csd_ocm_reset)               */
+    uint32_t debug_site;    /* first failed index check (0 = none), see CSD_FLAG_INTERNAL */
+    uint32_t reserved;
 } csd_stats_t;
 
 /* ---- Online Correction Memory (Sec. 4.2): frequency table of ordered pairs ----

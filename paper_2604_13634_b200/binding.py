@@ -15,11 +15,12 @@ from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int64,
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libcsd.so")
+# CSD_DEBUG=1 in the environment selects the bounds-checked build of the same sources
+LIB_PATH = os.path.join(_HERE, "libcsd_debug.so" if os.environ.get("CSD_DEBUG", "0") not in ("", "0") else "libcsd.so")
 
 CSD_F32, CSD_BF16 = 0, 1
 CSD_MAX_K = 32
-FLAG_NAN_LOGIT, FLAG_BAD_DRAFT, FLAG_PROBE_EXHAUSTED, FLAG_COUNT_SATURATED = 1, 2, 4, 8
+FLAG_NAN_LOGIT, FLAG_BAD_DRAFT, FLAG_PROBE_EXHAUSTED, FLAG_COUNT_SATURATED, FLAG_INTERNAL = 1, 2, 4, 8, 16
 
 EXPORTS = [
     "csd_ocm_create", "csd_ocm_reset", "csd_ocm_destroy", "csd_ocm_set_lambda",
@@ -44,7 +45,8 @@ class SampledDiag(Structure):
 
 class Stats(Structure):
     _fields_ = [(n, c_uint64) for n in ("n_slots", "key_limit", "n_keys", "n_dropped", "steps", "positions",
-                                         "matches", "rescues", "rejections")] + [("lambda_", c_uint32), ("flags", c_uint32)]
+                                         "matches", "rescues", "rejections")] + [("lambda_", c_uint32), ("flags", c_uint32),
+                                                                                 ("debug_site", c_uint32), ("reserved", c_uint32)]
 
     def as_dict(self):
         d = {n: int(getattr(self, n)) for n, _ in self._fields_}
@@ -386,3 +388,8 @@ def csd_step_sampled(logits, draft_logits, draft, r_accept, seed: int, temperatu
                      buf: SampledBuffers, stream=None):
     """csd_verify_sampled followed by the memory update with the step's recorded pairs."""
     _sampled_call("csd_step_sampled", logits, draft_logits, draft, r_accept, seed, temperature, ocm, tau, buf, stream)
+
+
+def sampled_launches_per_step() -> int:
+    """Kernel launches one csd_step_sampled call makes (for launch counts in reports)."""
+    return 7

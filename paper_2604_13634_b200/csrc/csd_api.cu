@@ -78,6 +78,64 @@ bool chain_follows(void *stream, const void *ws, const void *ocm, const void *ou
     return false;
 }
 
+// ---- which layout a workspace currently holds -----------------------------------------------
+// The scratch layout inside a workspace depends on the launch shape (grid, partial slots per
+// row), and so on csd_set_overlap / csd_set_tuning as well as on (B, K, V, dtype).  A workspace
+// whose counters were left by steps of another layout must be cleared before a step of this
+// layout touches it: its tickets would otherwise start from stale words and no row would ever
+// be finalised.  The host remembers, per workspace address, the layout of the last step issued
+// on it; a step that finds another layout (or no record) enqueues a clear first.
+struct WorkspaceRecord {
+    const void *ws;
+    size_t bytes;               // bytes the recorded layout covers
+    unsigned long long sig[3];  // layout signature
+    unsigned long long age;
+};
+constexpr int kWorkspaceRecords = 64;
+WorkspaceRecord g_ws_records[kWorkspaceRecords];
+int g_ws_used = 0;
+unsigned long long g_ws_clock = 0;
+
+// True if `ws` is known to hold exactly this layout; records it otherwise (caller clears).
+bool workspace_holds(const void *ws, size_t bytes, const unsigned long long (&sig)[3])
+{
+    std::lock_guard<std::mutex> lock(g_chain_mutex);
+    ++g_ws_clock;
+    int victim = 0;
+    for (int i = 0; i < g_ws_used; ++i) {
+        WorkspaceRecord &r = g_ws_records[i];
+        if (r.ws == ws) {
+            const bool same = r.bytes == bytes && r.sig[0] == sig[0] && r.sig[1] == sig[1] && r.sig[2] == sig[2];
+            r.bytes = bytes;
+            r.sig[0] = sig[0]; r.sig[1] = sig[1]; r.sig[2] = sig[2];
+            r.age = g_ws_clock;
+            return same;
+        }
+        if (r.age < g_ws_records[victim].age) victim = i;
+    }
+    if (g_ws_used < kWorkspaceRecords) victim = g_ws_used++;
+    WorkspaceRecord &r = g_ws_records[victim];
+    r.ws = ws;
+    r.bytes = bytes;
+    r.sig[0] = sig[0]; r.sig[1] = sig[1]; r.sig[2] = sig[2];
+    r.age = g_ws_clock;
+    return false;
+}
+
+// Forget every record that overlaps [ws, ws + bytes): the range was cleared or is about to be reused.
+void workspace_forget(const void *ws, size_t bytes)
+{
+    std::lock_guard<std::mutex> lock(g_chain_mutex);
+    const char *lo = static_cast<const char *>(ws), *hi = lo + bytes;
+    for (int i = 0; i < g_ws_used;) {
+        const char *a = static_cast<const char *>(g_ws_records[i].ws);
+        if (a < hi && a + g_ws_records[i].bytes > lo)
+            g_ws_records[i] = g_ws_records[--g_ws_used];
+        else
+            ++i;
+    }
+}
+
 int sm_count()
 {
     static int cached = 0;
@@ -189,7 +247,8 @@ OcmView view_of(const csd_ocm *o)
 csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b, int64_t stride_k,
                       const int32_t *draft, const csd_ocm *ocm, float tau, int32_t *accept_len, int32_t *next_token,
                       uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
-                      void *workspace, size_t workspace_bytes, void *stream, bool do_update, bool may_chain = true)
+                      void *workspace, size_t workspace_bytes, void *stream, bool do_update, bool may_chain = true,
+                      bool may_overlap = true, bool track_layout = true)
 {
     if (!logits || !draft || !ocm || !accept_len || !next_token || !rescued_mask || !rej_draft || !rej_target || !workspace)
         return CSD_ERR_INVALID_ARG;
@@ -232,6 +291,21 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.chunk_units = s.chunk_units;
     p.total_units = s.total_units;
     p.narrow = (s.total_units + 1) * (static_cast<long long>(s.grid) + 1) < (1ll << 32) ? 1 : 0;
+    if (track_layout) {
+        const unsigned long long sig[3] = {
+            (static_cast<unsigned long long>(static_cast<unsigned int>(B)) << 32) | static_cast<unsigned int>(K),
+            (static_cast<unsigned long long>(static_cast<unsigned int>(s.grid)) << 32) | static_cast<unsigned int>(s.slots_per_row),
+            (static_cast<unsigned long long>(w.copy_bytes) << 8) | static_cast<unsigned int>(dtype)};
+        if (!workspace_holds(workspace, w.total, sig)) {
+            // first step of this layout on this workspace: start from cleared counters
+            chain_break();
+            if (cudaMemsetAsync(workspace, 0, w.total, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+                (void)cudaGetLastError();
+                workspace_forget(workspace, w.total);
+                return CSD_ERR_CUDA;
+            }
+        }
+    }
     const bool follows = chain_follows(stream, workspace, ocm, accept_len, B, K, V, static_cast<int>(dtype));
     p.chain_by_flag = (may_chain && follows) ? 1 : 0;
 
@@ -245,7 +319,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     cfg.blockDim = dim3(s.block);
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
-    if (g_overlap_steps) {
+    if (g_overlap_steps && may_overlap) {
         // let this launch begin while the previous kernel on the stream drains; the kernel
         // itself waits for that kernel before its first write
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -264,6 +338,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     if (err != cudaSuccess) {
         (void)cudaGetLastError();
         chain_break();
+        workspace_forget(workspace, w.total);
         return CSD_ERR_CUDA;
     }
     return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
@@ -533,6 +608,7 @@ csd_status_t csd_workspace_init(void *workspace, size_t workspace_bytes, void *s
 {
     if (!workspace || workspace_bytes == 0) return CSD_ERR_INVALID_ARG;
     chain_break();
+    workspace_forget(workspace, workspace_bytes);
     if (cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
         (void)cudaGetLastError();
         return CSD_ERR_CUDA;
@@ -612,6 +688,7 @@ namespace {
 constexpr int kMaxDevices = 64;
 void *g_static_scratch_ptr[kMaxDevices];   // device address of g_static_scratch, per device
 bool g_static_scratch_known[kMaxDevices];
+std::mutex g_static_scratch_mutex;
 }  // namespace
 
 csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b,
@@ -630,17 +707,22 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
         return CSD_ERR_CUDA;
     }
     if (dev != ocm->device) return CSD_ERR_INVALID_ARG;   // the memory's device must be the current one
-    if (!g_static_scratch_known[dev]) {
-        // once per device, with that device current (first call: not under stream capture)
-        void *ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
-            (void)cudaGetLastError();
-            return CSD_ERR_CUDA;
+    void *scratch = nullptr;
+    {
+        // once per device, with that device current (first call: not under stream capture); two host
+        // threads may make their first call together
+        std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+        if (!g_static_scratch_known[dev]) {
+            void *ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+                (void)cudaGetLastError();
+                return CSD_ERR_CUDA;
+            }
+            g_static_scratch_ptr[dev] = ptr;
+            g_static_scratch_known[dev] = true;
         }
-        g_static_scratch_ptr[dev] = ptr;
-        g_static_scratch_known[dev] = true;
+        scratch = g_static_scratch_ptr[dev];
     }
-    void *scratch = g_static_scratch_ptr[dev];
     // The array keeps whatever the last call (possibly of another shape) left in it, and the
     // kernel needs its counters and sequence words to start at zero: clear the part in use.
     if (cudaMemsetAsync(scratch, 0, need, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
@@ -648,7 +730,8 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
         return CSD_ERR_CUDA;
     }
     return run_step(logits, dtype, B, K, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
-                    rej_draft, rej_target, diag, scratch, need, stream, false, false);
+                    rej_draft, rej_target, diag, scratch, need, stream, false, /*may_chain=*/false,
+                    /*may_overlap=*/false, /*track_layout=*/false);   // cleared just above, whatever it held
 }
 
 size_t csd_sampled_workspace_bytes(int B, int K, int V, csd_dtype_t dtype)
@@ -711,11 +794,12 @@ csd_status_t csd_step_host(const void *logits_host, csd_dtype_t dtype, int B, in
         return CSD_ERR_CUDA;
     }
     const csd_status_t rc =
-        csd_step(dev + s.logits, dtype, B, K, V, static_cast<int64_t>(K + 1) * V, V,
+        run_step(dev + s.logits, dtype, B, K, V, static_cast<int64_t>(K + 1) * V, V,
                  reinterpret_cast<const int32_t *>(dev + s.draft), ocm, tau, reinterpret_cast<int32_t *>(dev + s.accept),
                  reinterpret_cast<int32_t *>(dev + s.next), reinterpret_cast<uint8_t *>(dev + s.rescued),
                  reinterpret_cast<int32_t *>(dev + s.rej_d), reinterpret_cast<int32_t *>(dev + s.rej_t), nullptr,
-                 dev + s.ws, s.ws_bytes, stream);
+                 dev + s.ws, s.ws_bytes, stream, /*do_update=*/true, /*may_chain=*/true,
+                 /*may_overlap=*/true, /*track_layout=*/false);
     if (rc != CSD_OK) return rc;
     ok = ok && cudaMemcpyAsync(accept_len_host, dev + s.accept, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(next_token_host, dev + s.next, static_cast<size_t>(B) * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
@@ -773,6 +857,8 @@ csd_status_t csd_ocm_stats(const csd_ocm_t *ocm, csd_stats_t *host_out, void *st
     host_out->rejections = s.rejections;
     host_out->lambda = ocm->lambda;
     host_out->flags = s.flags;
+    host_out->debug_site = s.debug_site;
+    host_out->reserved = 0;
     return CSD_OK;
 }
 

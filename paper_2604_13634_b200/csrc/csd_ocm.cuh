@@ -37,7 +37,24 @@ struct OcmStatsDev {
     unsigned int flags;
     unsigned int ticket;              // arrival counter of multi-block update launches
     unsigned long long export_count;  // cursor of csd_ocm_export
+    unsigned int debug_site;          // first failed index check (0 = none)
+    unsigned int pad;
 };
+
+// Index checks.  A failed check sets a sticky flag, remembers which check it was and makes the
+// caller skip the access; nothing traps.  CSD_CHECKED is for the one check that every build
+// keeps; CSD_INDEX_OK compiles to `true` unless the library is built with -DCSD_DEBUG.
+__device__ __noinline__ void index_check_failed(OcmStatsDev *stats, unsigned int site)
+{
+    atomicOr(&stats->flags, 0x10u);
+    atomicCAS(&stats->debug_site, 0u, site);
+}
+#define CSD_CHECKED(cond, stats, site) ((cond) ? true : (csd::index_check_failed((stats), (site)), false))
+#ifdef CSD_DEBUG
+#define CSD_INDEX_OK(cond, stats, site) CSD_CHECKED(cond, stats, site)
+#else
+#define CSD_INDEX_OK(cond, stats, site) (true)
+#endif
 
 struct OcmView {
     OcmSlot *slots;

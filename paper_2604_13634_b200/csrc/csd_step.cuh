@@ -38,9 +38,9 @@
 // Consecutive steps (programmatic dependent launch, opt-in)
 //   * A launch may begin as soon as every block of the previous launch on the stream has
 //     started.  The scratch exists kScratchRing times and launches take the copies in
-//     turn, by a sequence number kept in the workspace itself (every block draws it with
-//     one atomic; the block that draws last advances it; only then can the next launch
-//     begin, so all blocks of a launch see the same number).  Streaming, publication,
+//     turn, by a sequence number kept in the workspace itself (one word counts the blocks
+//     of all launches; a block's count divided by the grid size is its launch's number,
+//     and the next launch begins only after every block of this one has counted in).  Streaming, publication,
 //     tickets and the per-row fold of step n therefore run while steps n-1, n-2, ... are
 //     still finishing.
 //   * What does depend on step n-1 is the memory (its update) and the output buffers.
@@ -82,7 +82,7 @@ struct StepParams {
     //   global ticket [1]                                                         at g_ticket_off
     char *scratch;
     unsigned int copy_bytes, hint_off, b_ticket_off, g_ticket_off;
-    unsigned long long *launch_seq;  // (sequence number of the launch now starting << 32) | blocks counted in
+    unsigned long long *launch_seq;  // blocks counted in by all launches on this workspace since it was cleared
     unsigned int *completed;         // launches completed on this workspace
     int n_spans;             // G: blocks that own a span of the unit space
     int unit_elems;          // elements per 512-byte unit
@@ -500,7 +500,8 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, const ScratchCopy
             const int row = r0 + q * rows_per_pass + sub;
             v[q] = partial_identity();
             if (row < K1) {
-                const int np = rs.parts[row];
+                int np = rs.parts[row];
+                if (!CSD_INDEX_OK(np >= 1 && np <= S, p.ocm.stats, 3u)) np = 0;
                 for (int k = k0; k < np; k += width) {       // one trip unless a row has > 32 parts
                     const Partial x = ld_partial_cg(part + (size_t)row * S + k);
                     v[q] = (k == k0) ? x : combine(v[q], x);
@@ -651,6 +652,7 @@ __device__ void apply_step_update(const StepParams &p, const ScratchCopy &sc, in
         for (int q = 0; q < 16; ++q) {
             if (h[q] >= 0) {
                 const unsigned long long s = static_cast<unsigned long long>(h[q] & ~kHintCareful);
+                if (!CSD_INDEX_OK(s <= p.ocm.mask, p.ocm.stats, 4u)) continue;
                 if (h[q] & kHintCareful)
                     ocm_add(p.ocm, s, 1u);
                 else
@@ -686,7 +688,9 @@ __device__ void publish_parts(const StepParams &p, BlockState &bs, int first_row
     if (lane < nseg) {
         const int row = first_row + lane;
         const int slot = static_cast<int>(blockIdx.x) - owner_of(p, static_cast<long long>(row) * U);
-        if (slot < p.slots_per_row) st_partial_cg(sc.partials + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
+        // the host sized slots_per_row from the same split: a slot beyond it would be a bug, and is reported
+        if (CSD_CHECKED(slot >= 0 && slot < p.slots_per_row && row < p.B * K1, p.ocm.stats, 1u))
+            st_partial_cg(sc.partials + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
         my_b = row / K1;
     }
     __threadfence();
@@ -703,7 +707,7 @@ __device__ void publish_parts(const StepParams &p, BlockState &bs, int first_row
         }
     }
     const unsigned int todo = __ballot_sync(kFull, completes);
-    if (completes) bs.todo_b[__popc(todo & ((1u << lane) - 1u))] = my_b;
+    if (completes && CSD_INDEX_OK(my_b >= 0 && my_b < p.B, p.ocm.stats, 2u)) bs.todo_b[__popc(todo & ((1u << lane) - 1u))] = my_b;
     if (lane == 0) bs.n_todo = __popc(todo);
     __threadfence();      // the other blocks' partials of those rows, before this block's warps read them
 }
@@ -756,11 +760,12 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
-    // Launch sequence number, one atomic: the word holds (sequence << 32 | blocks counted
-    // in).  Every block counts itself in and learns the sequence from the same answer;
-    // the block that is last to do so moves the word on to the next launch.  That launch
-    // can begin only after every block of this one has released it, which a block does
-    // after counting itself in -- so all blocks of a launch see the same number.
+    // Launch sequence number, one atomic: the word counts the blocks of every launch on this
+    // workspace since it was cleared, and every launch between two clears has the same grid
+    // (the host clears a workspace before a step of another layout uses it), so a block's
+    // launch number is its count divided by the grid size.  The next launch can begin only
+    // after every block of this one has released it, which a block does after its own count
+    // has come back -- so the counts of two launches never interleave.
     // The block's LAST warp does this, so that the round trip of the (contended) atomic
     // delays neither the other warps' start nor the set-up of the shared tables; it joins
     // the streaming afterwards.
@@ -806,11 +811,9 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             named_barrier_sync(1, 32 * (nwarps - 1));   // the streaming warps start without the last warp
         }
         if (first_window && seq_warp) {
-            if (lane == 0) {
-                if (static_cast<unsigned int>(seq_old) == gridDim.x - 1)
-                    atomicAdd(p.launch_seq, (1ull << 32) - static_cast<unsigned long long>(gridDim.x));
-                bs.seq = static_cast<unsigned int>(seq_old >> 32);
-            }
+            if (lane == 0)
+                bs.seq = (seq_old >> 32) == 0ull ? static_cast<unsigned int>(seq_old) / gridDim.x
+                                                 : static_cast<unsigned int>(seq_old / gridDim.x);
             __syncwarp();
             pdl_launch_dependents();
             bool block_complete = false;
@@ -853,6 +856,10 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             const int e0 = u0 * p.unit_elems;
             const long long e1l = static_cast<long long>(u1) * p.unit_elems;
             const int e1 = e1l < p.V ? static_cast<int>(e1l) : p.V;
+            if (!CSD_INDEX_OK(row < static_cast<long long>(p.B) * K1 && seg >= 0 && seg < nseg && nseg <= kMaxSegs &&
+                                  q < static_cast<unsigned int>(kMaxChunks) && e0 >= 0 && e0 < e1 && seg_first + seg_n <= kMaxChunks,
+                              p.ocm.stats, 5u))
+                continue;
             const Partial r = warp_tile<L>(rp, e0, e1, lane);
 
             // ---- deliver it; the warp bringing a row part's last chunk folds that part ----
@@ -884,7 +891,7 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
         // ---- the batch rows this block completed are shared out over its warps: S2..S6 ----
         __syncthreads();
         const int fin_warps = nwarps < kFinalizeWarps ? nwarps : kFinalizeWarps;
-        if (warp < fin_warps)
+        if (warp < fin_warps && CSD_INDEX_OK(bs.n_todo >= 0 && bs.n_todo <= kMaxSegs, p.ocm.stats, 6u))
             for (int j = warp; j < bs.n_todo; j += fin_warps)
                 finalize_and_update<L>(p, bs.seq, bs.todo_b[j], lane, row_scratch[warp], canon);
         g = w_end;

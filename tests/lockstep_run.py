@@ -26,7 +26,7 @@ sys.path.insert(0, os.path.join(ROOT, "tests"))
 import test_gpu_parity as T                                     # noqa: E402
 from oracle import csd_oracle as ORACLE                          # noqa: E402
 from paper_2604_13634_b200 import Ocm, StepBuffers, csd_step     # noqa: E402
-from paper_2604_13634_b200.synth import WORKLOADS, Synth         # noqa: E402
+from synth_inputs import WORKLOADS, Synth         # noqa: E402
 
 
 OVERLAP = False
@@ -34,7 +34,7 @@ _PINNED = {}
 
 
 def _bits_through_pinned_memory(z: torch.Tensor):
-    """Same result as synth.logits_bits_numpy, but the device-to-host copy lands in a pinned buffer
+    """Same result as synth_inputs.logits_bits_numpy, but the device-to-host copy lands in a pinned buffer
     that is kept between steps (several times faster for the 100 MB+ steps of the long runs)."""
     z = z.detach().contiguous()
     key = (tuple(z.shape), z.dtype)

@@ -8,6 +8,7 @@ gate is decided exactly on both sides they are expected to agree as well.
 """
 
 import dataclasses
+import os
 
 import numpy as np
 import pytest
@@ -17,7 +18,7 @@ from oracle import csd_oracle as ORACLE
 from oracle import row_stats_c
 from paper_2604_13634_b200 import (CSD_BF16, CSD_F32, HostStep, Ocm, StepBuffers, csd_launch_shape, csd_set_tuning,
                                    csd_step, csd_verify)
-from paper_2604_13634_b200.synth import WORKLOADS, Synth, logits_bits_numpy
+from synth_inputs import WORKLOADS, Synth, logits_bits_numpy
 
 pytestmark = pytest.mark.gpu
 
@@ -485,6 +486,70 @@ def test_overlapped_launches_match():
     assert np.array_equal(ref_out[-1][2].cpu().numpy(), ref["rescued_mask"])
     rd, rt, rc = mem.export()
     assert np.array_equal(ref_exp[0].numpy(), rd) and np.array_equal(ref_exp[2].numpy(), rc)
+
+
+def test_launch_shape_changes_on_a_live_workspace():
+    """csd_set_overlap and csd_set_tuning change the layout of the scratch inside a workspace.  A
+    workspace that has seen steps of one layout is cleared by the library before a step of another
+    layout uses it, so switching on a live workspace gives the same results as a fresh one."""
+    from paper_2604_13634_b200 import csd_set_overlap
+    wl = WORKLOADS["batched_serving"]
+    syn = Synth(wl, 6, "cuda")
+    ocm = Ocm(wl.ocm_slots, 1)
+    mem = ORACLE.OCM(wl.ocm_slots, 1)
+    buf = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True)
+    settings = [(False, (0, 0, 0)), (True, (0, 0, 0)), (False, (0, 0, 0)), (False, (8192, 2, 128)), (True, (0, 0, 0)),
+                (True, (4096, 3, 256)), (False, (0, 0, 0))]
+    try:
+        for s, (overlap, tuning) in enumerate(settings):
+            csd_set_overlap(overlap)
+            csd_set_tuning(*tuning)
+            for rep in range(3):
+                z, d = syn.step(2 * s + rep % 2)
+                csd_step(z, d, ocm, 0.3, buf)
+                compare(buf, oracle_step(z, d, mem, 0.3))
+        st = compare_memory(ocm, mem)
+        assert st["flags"] == 0 and st["steps"] == 3 * len(settings)
+    finally:
+        csd_set_overlap(False)
+        csd_set_tuning(0, 0, 0)
+    ocm.close()
+
+
+def test_bounds_checked_build_runs_the_small_shapes_clean():
+    """The same sources built with -DCSD_DEBUG compare every index they compute with its bound (a failed
+    check skips the access and raises CSD_FLAG_INTERNAL; nothing traps).  The small-shape parity tests
+    run once more against that build, in a process of their own, and the flag must stay clear."""
+    import os
+    import subprocess
+    import sys
+    from paper_2604_13634_b200 import build
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    assert os.path.exists(build.LIB_DEBUG), "libcsd_debug.so has not been built"
+    env = dict(os.environ, CSD_DEBUG="1")
+    sel = ("test_elementwise_parity_small or test_many_short_rows_per_warp or test_contention_fills_the_table "
+           "or test_strided_and_misaligned_views or test_internal_flag_is_clear")
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-k", sel,
+                        os.path.join(root, "tests", "test_gpu_parity.py"), os.path.join(root, "tests", "test_gpu_sampled_parity.py")],
+                       cwd=root, env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:]
+
+
+def test_internal_flag_is_clear():
+    """A step on each dtype and path; the library's own index checks (all of them in the CSD_DEBUG build,
+    the partial-slot check in every build) must not have fired."""
+    from paper_2604_13634_b200 import binding
+    for (B, K, V, dtype) in ((7, 5, 33000, torch.float32), (9, 3, 40001, torch.bfloat16), (300, 2, 700, torch.bfloat16)):
+        z, d = _random_inputs(B, K, V, dtype, seed=5)
+        ocm = Ocm(1 << 12, 1)
+        buf = StepBuffers(B, K, V, dtype)
+        for _ in range(3):
+            csd_step(z, d, ocm, 0.01, buf)
+        st = ocm.stats()
+        assert st["flags"] & binding.FLAG_INTERNAL == 0 and st["debug_site"] == 0, st
+        ocm.close()
+    want = "libcsd_debug.so" if os.environ.get("CSD_DEBUG", "0") not in ("", "0") else "libcsd.so"
+    assert binding.LIB_PATH.endswith(want)
 
 
 def test_long_rows():

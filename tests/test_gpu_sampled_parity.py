@@ -17,7 +17,7 @@ import torch
 from oracle import csd_sampled_oracle as ORACLE
 from oracle.csd_oracle import bf16_bits_to_f64
 from paper_2604_13634_b200 import CSD_BF16, CSD_F32, Ocm, SampledBuffers, csd_step_sampled, csd_verify_sampled
-from paper_2604_13634_b200.synth import WORKLOADS, Synth, logits_bits_numpy
+from synth_inputs import WORKLOADS, Synth, logits_bits_numpy
 
 pytestmark = pytest.mark.gpu
 RTOL = 1e-5

@@ -19,7 +19,7 @@ def _worker(rank, world, port, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     import bench
-    from paper_2604_13634_b200.synth import WORKLOADS, Synth
+    from synth_inputs import WORKLOADS, Synth
     import dataclasses
     # each rank is an independent replica with its own seeded batch
     wl = dataclasses.replace(WORKLOADS["tiny"], V=512)

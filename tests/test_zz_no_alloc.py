@@ -15,7 +15,7 @@ import pytest
 import torch
 
 from paper_2604_13634_b200 import Ocm, StepBuffers, binding, csd_step, csd_verify
-from paper_2604_13634_b200.synth import WORKLOADS, Synth
+from synth_inputs import WORKLOADS, Synth
 import dataclasses
 
 pytestmark = pytest.mark.gpu
@@ -61,6 +61,26 @@ def test_static_scratch_entry_point_matches_csd_verify():
                     assert torch.equal(a, b)
                 assert int(ref_buf.rescued_mask.sum()) + int((ref_buf.accept_len > 0).sum()) > 0
             ocm.close()
+
+
+def test_static_scratch_entry_point_takes_no_device_memory():
+    """What the entry point is for: the free device memory reported by the driver is the same before
+    and after a series of calls (inputs, outputs and the memory object were allocated beforehand)."""
+    L = binding.lib()
+    wl = dataclasses.replace(WORKLOADS["batched_serving"], B=8)
+    syn = Synth(wl, seed=3, device="cuda")
+    ocm = Ocm(4096, lam=1)
+    buf = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True)
+    z, d = syn.step(0)
+    _call_static(L, z, d, ocm, 0.3, buf)          # the first call on a device looks up the array's address
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(5):
+        _call_static(L, z, d, ocm, 0.3, buf)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    ocm.close()
 
 
 def test_static_scratch_refuses_what_does_not_fit():
