@@ -32,6 +32,12 @@ Conventions the paper leaves open (each one is a reading of this build):
       not recorded.  PARITY UNPINNED (paper is silent).
   R6  the gate of Eq. 3 is decided in logit space: (z_d - z_t*) in float64
       against float32(ln(float32 tau)); equality passes.
+  R7  ageing (opt-in; an alternative to "frozen when full" under R3): `age()`
+      halves every count, rounding down, and removes the pairs that reach zero,
+      which frees their room for new pairs.  It depends on nothing but the
+      stored set, so it is independent of order, layout and timing.  PARITY
+      UNPINNED: Sec. 4.2 says the memory keeps evolving online and names no
+      forgetting rule.
 """
 
 from __future__ import annotations
@@ -120,6 +126,16 @@ class OCM:
                 self.table[key] = min(w, COUNT_MAX)
             else:
                 self.n_dropped += 1
+
+    def age(self):
+        """Halve every count (floor) and forget the pairs that reach zero (R7)."""
+        self.table = {k: c // 2 for k, c in self.table.items() if c // 2 > 0}
+
+    def merge(self, other: "OCM"):
+        """Add another memory's counts to this one: its pairs in sorted order, each with its count as
+        the weight, under the same admission rule as any update (R3, R4)."""
+        d, t, c = other.export()
+        self.update(zip(d.tolist(), t.tolist()), weights=c.tolist())
 
     def export(self):
         """Sorted (draft, target, count) triples."""

@@ -420,72 +420,100 @@ def test_many_short_rows_per_warp():
 def test_overlapped_launches_match():
     """Hundreds of back-to-back steps launched with programmatic stream serialization (the
     setting the benchmark times), eagerly and as a replayed CUDA graph, give the same
-    results as plain launches; the plain run is pinned to the oracle.  With one set of
-    output buffers per ring entry consecutive launches differ in their outputs, so each
-    waits for its predecessor to retire; with a single set they chain on the completion
-    count in the workspace (the path the benchmark takes)."""
+    results as plain launches, and the plain run equals the oracle at EVERY step (accepted
+    lengths, next tokens, masks, rejection lists, arg-max, counts).  With one set of output
+    buffers per step consecutive launches differ in their outputs, so each waits for its
+    predecessor to retire, and every step's outputs survive to be compared; with a single
+    set they chain on the completion count in the workspace (the path the benchmark takes)
+    and the last step, the memory and the statistics are compared."""
     from paper_2604_13634_b200 import csd_set_overlap
     wl = WORKLOADS["batched_serving"]
     syn = Synth(wl, 4, "cuda")
     inputs = [syn.step(s) for s in range(5)]         # an odd ring: replays follow each other out of phase
     reps = 41
+    n_steps = reps * len(inputs)
 
     def run(overlap, graph, one_buffer):
         try:
             csd_set_overlap(overlap)
             ocm = Ocm(wl.ocm_slots, 2)
-            bufs = [StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True) for _ in inputs]
-            if one_buffer:
-                bufs = [bufs[0]] * len(inputs)
             ws = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype)         # one shared workspace, as the benchmark has
+            if one_buffer:
+                bufs = [StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True)] * n_steps
+            else:
+                bufs = [StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True) for _ in range(n_steps)]
             for b in bufs:
                 b.workspace, b.ws_bytes = ws.workspace, ws.ws_bytes
 
-            def ring():
-                for (z, d), buf in zip(inputs, bufs):
-                    csd_step(z, d, ocm, 0.3, buf)
-            if graph:
+            def steps(lo, hi):
+                for s in range(lo, hi):
+                    z, d = inputs[s % len(inputs)]
+                    csd_step(z, d, ocm, 0.3, bufs[s])
+            if graph and one_buffer:                 # one ring pass captured, replayed (reps - 1) times
                 side = torch.cuda.Stream()
                 side.wait_stream(torch.cuda.current_stream())
                 with torch.cuda.stream(side):
-                    ring()
+                    steps(0, len(inputs))
                 torch.cuda.current_stream().wait_stream(side)
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
-                    ring()
-                for _ in range(reps - 1):        # the capture itself runs nothing
+                    steps(0, len(inputs))
+                for _ in range(reps - 1):
                     g.replay()
+            elif graph:                               # the first pass eagerly, all the rest as ONE graph
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    steps(0, len(inputs))
+                torch.cuda.current_stream().wait_stream(side)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    steps(len(inputs), n_steps)
+                g.replay()
             else:
-                for _ in range(reps):
-                    ring()
+                steps(0, n_steps)
             torch.cuda.synchronize()
+            keep = bufs[-len(inputs):] if one_buffer else bufs
             out = ([(b.accept_len.clone(), b.next_token.clone(), b.rescued_mask.clone(), b.rej_draft.clone(),
                      b.rej_target.clone(), b.diag["t"].clone(), b.diag["cnt"].clone(), b.diag["s"].clone())
-                    for b in bufs], ocm.export(), ocm.stats())
+                    for b in keep], ocm.export(), ocm.stats())
             ocm.close()
             return out
         finally:
             csd_set_overlap(False)
 
+    plain = {}
     for one_buffer in (False, True):
         ref_out, ref_exp, ref_st = run(False, False, one_buffer)
-        assert ref_st["steps"] == reps * len(inputs) and ref_st["flags"] == 0
+        plain[one_buffer] = (ref_out, ref_exp)
+        assert ref_st["steps"] == n_steps and ref_st["flags"] == 0
         for overlap, graph in ((True, False), (True, True), (False, True)):
             out, exp, st = run(overlap, graph, one_buffer)
             assert st == ref_st, (overlap, graph, one_buffer, st, ref_st)
             assert all(torch.equal(p, q) for p, q in zip(exp, ref_exp)), (overlap, graph, one_buffer)
+            assert len(out) == len(ref_out)
             for x, y in zip(out, ref_out):
                 assert all(torch.equal(p, q) for p, q in zip(x[:-1], y[:-1])), (overlap, graph, one_buffer)
                 # the launch shape, and with it the summation tree, depends on the overlap setting
                 assert torch.allclose(x[-1], y[-1], rtol=1e-5, atol=0), (overlap, graph, one_buffer)
+    # the plain run against the oracle: every step of the per-step run, the last step of the single-buffer run
     mem = ORACLE.OCM(wl.ocm_slots, 2)
-    for rep in range(reps):
-        for z, d in inputs:
-            ref = oracle_step(z, d, mem, 0.3)
-    assert np.array_equal(ref_out[-1][0].cpu().numpy(), ref["accept_len"])
-    assert np.array_equal(ref_out[-1][2].cpu().numpy(), ref["rescued_mask"])
+    per_step, _ = plain[False]
+    last_pass, _ = plain[True]
+    for s in range(n_steps):
+        z, d = inputs[s % len(inputs)]
+        ref = oracle_step(z, d, mem, 0.3)
+        got = per_step[s]
+        for k, name in enumerate(("accept_len", "next_token", "rescued_mask", "rej_draft", "rej_target", "t")):
+            assert np.array_equal(got[k].cpu().numpy(), ref[name]), (s, name)
+        assert np.array_equal(got[6].cpu().numpy().astype(np.int64) & 0xFFFFFFFF, ref["cnt"]), (s, "cnt")
+        if s == n_steps - 1:                      # a single set of buffers keeps the last step only
+            got = last_pass[-1]
+            for k, name in enumerate(("accept_len", "next_token", "rescued_mask", "rej_draft", "rej_target", "t")):
+                assert np.array_equal(got[k].cpu().numpy(), ref[name]), (s, name, "single buffer")
     rd, rt, rc = mem.export()
-    assert np.array_equal(ref_exp[0].numpy(), rd) and np.array_equal(ref_exp[2].numpy(), rc)
+    for _, exp in plain.values():
+        assert np.array_equal(exp[0].numpy(), rd) and np.array_equal(exp[1].numpy(), rt) and np.array_equal(exp[2].numpy(), rc)
 
 
 def test_launch_shape_changes_on_a_live_workspace():

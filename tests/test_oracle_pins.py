@@ -407,7 +407,48 @@ def pin_near_tie_flag(o):
     assert not o.verify(z, np.array([[1]]), o.OCM(64, 0), 0.3)["near_tie"][0, 0]
 
 
-PINS = [pin_row_stats_closed_forms, pin_row_stats_library, pin_lowest_index_on_ties, pin_eq3_identity,
+def pin_ageing_and_merge(o):
+    """R7 and the weighted merge: hand traces and the properties that make them order-independent."""
+    mem = o.OCM(8, 2)                                   # limit: 4 pairs
+    mem.update([(1, 2)] * 5 + [(3, 4)] * 2 + [(5, 6)] + [(7, 8)] * 4)
+    assert mem.table == {(1, 2): 5, (3, 4): 2, (5, 6): 1, (7, 8): 4}
+    mem.update([(9, 9)])                                # full: dropped
+    assert mem.n_dropped == 1 and (9, 9) not in mem.table
+    mem.age()
+    assert mem.table == {(1, 2): 2, (3, 4): 1, (7, 8): 2}          # floor halves; the single occurrence is forgotten
+    assert mem.n_dropped == 1                            # ageing is not dropping
+    mem.update([(9, 9)])                                # the freed room admits a new pair
+    assert mem.table[(9, 9)] == 1 and mem.n_keys == 4
+    mem.age(); mem.age()
+    assert mem.table == {} and mem.n_keys == 0
+    # ageing a saturated count, and twice halving = quartering (floor of floor = floor)
+    mem.update([(1, 1)], weights=[o.COUNT_MAX]); mem.update([(1, 1)], weights=[5])
+    assert mem.table[(1, 1)] == o.COUNT_MAX
+    mem.age()
+    assert mem.table[(1, 1)] == (2 ** 32 - 1) // 2
+    rng = np.random.default_rng(4)
+    a = o.OCM(128, 1); b = o.OCM(128, 1)
+    pairs = [(int(x), int(y)) for x, y in rng.integers(0, 6, size=(300, 2))]
+    a.update(pairs)
+    b.update(pairs[::-1])                               # another arrival order, same multiset, room for all
+    a.age(); b.age()
+    assert a.table == b.table and all(c == pairs.count(k) // 2 for k, c in a.table.items())
+    assert all(pairs.count(k) < 2 for k in set(pairs) - set(a.table))
+    # merge: counts of common pairs add, new pairs enter in sorted order while there is room
+    x = o.OCM(8, 1); y = o.OCM(64, 1)
+    x.update([(1, 1)] * 3 + [(2, 2)] * 2)
+    y.update([(2, 2)] * 4 + [(0, 5)] + [(3, 3)] * 2 + [(9, 9)] * 7 + [(8, 8)])
+    x.merge(y)
+    assert x.table == {(1, 1): 3, (2, 2): 6, (0, 5): 1, (3, 3): 2} and x.n_dropped == 2    # the entries (8,8) and (9,9) found no room: one dropped occurrence each
+    assert y.table[(9, 9)] == 7                          # the source is left alone
+    big = o.OCM(64, 1); big.update([(1, 1)] * 3 + [(2, 2)] * 2); big.merge(y)
+    assert big.table == {(1, 1): 3, (2, 2): 6, (0, 5): 1, (3, 3): 2, (9, 9): 7, (8, 8): 1} and big.n_dropped == 0
+    z = o.OCM(64, 1); z.update([(4, 4)], weights=[o.COUNT_MAX - 1]); w = o.OCM(64, 1); w.update([(4, 4)] * 3)
+    z.merge(w)
+    assert z.table[(4, 4)] == o.COUNT_MAX                # saturates
+
+
+PINS = [pin_ageing_and_merge, pin_row_stats_closed_forms, pin_row_stats_library, pin_lowest_index_on_ties, pin_eq3_identity,
         pin_threshold, pin_empty_memory_is_strict_matching, pin_ablation_reductions, pin_monotone,
         pin_fig1_worked_example, pin_update_traces, pin_bruteforce_vs_sequential,
         pin_repeated_pair_in_one_row, pin_capacity_policy, pin_bad_draft, pin_cross_row_snapshot,
@@ -445,6 +486,11 @@ MUTANTS = [
     ("no saturation", "min(self.table[key] + w, COUNT_MAX)", "(self.table[key] + w)"),
     ("bad draft recorded", "            if not (0 <= d < V):                 # R5\n                bad += 1\n                n = i\n                break\n",
      "            if not (0 <= d < V):                 # R5\n                bad += 1\n                rej_d[b, i] = d\n                rej_t[b, i] = tt\n                n = i\n                break\n"),
+    ("ageing rounds up", "self.table = {k: c // 2 for k, c in self.table.items() if c // 2 > 0}", "self.table = {k: (c + 1) // 2 for k, c in self.table.items() if (c + 1) // 2 > 0}"),
+    ("ageing keeps the zeros", "self.table = {k: c // 2 for k, c in self.table.items() if c // 2 > 0}", "self.table = {k: c // 2 for k, c in self.table.items()}"),
+    ("ageing forgets the ones but does not halve", "self.table = {k: c // 2 for k, c in self.table.items() if c // 2 > 0}", "self.table = {k: c for k, c in self.table.items() if c // 2 > 0}"),
+    ("merge ignores the counts", "self.update(zip(d.tolist(), t.tolist()), weights=c.tolist())", "self.update(zip(d.tolist(), t.tolist()))"),
+    ("merge swaps draft and target", "self.update(zip(d.tolist(), t.tolist()), weights=c.tolist())", "self.update(zip(t.tolist(), d.tolist()), weights=c.tolist())"),
     ("rescue mask set on match", "            if d == tt:                          # exact match: accepted\n                continue",
      "            if d == tt:                          # exact match: accepted\n                rescued[b, i] = 1\n                continue"),
 ]
