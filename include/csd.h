@@ -49,7 +49,8 @@ typedef enum {
     CSD_ERR_CUDA = 2,
     CSD_ERR_OOM = 3,
     CSD_ERR_UNSUPPORTED = 4,
-    CSD_ERR_WORKSPACE = 5
+    CSD_ERR_WORKSPACE = 5,
+    CSD_ERR_IO = 6
 } csd_status_t;
 
 typedef enum { CSD_F32 = 0, CSD_BF16 = 1 } csd_dtype_t;
@@ -330,6 +331,40 @@ csd_status_t csd_ocm_export(const csd_ocm_t *ocm, int32_t *d, int32_t *t, uint32
  * export is csd_ocm_reset followed by csd_ocm_import.  Device arrays; asynchronous. */
 csd_status_t csd_ocm_import(csd_ocm_t *ocm, const int32_t *d, const int32_t *t, const uint32_t *cnt,
                             uint64_t n, void *stream);
+
+/* Ageing, an opt-in alternative to "frozen once full" (the paper's Sec. 4.2 lets the memory
+ * evolve online and names no forgetting rule; this one is the library's): every count is
+ * halved, rounding down, and the pairs that reach zero are forgotten, which frees their room
+ * for new pairs.  The result depends only on the stored set.  The serving loop calls it at
+ * the cadence it wants (say every N steps), stream-ordered like any call; n_dropped and the
+ * step statistics are untouched.  Two launches; asynchronous; nothing is allocated. */
+csd_status_t csd_ocm_age(csd_ocm_t *ocm, void *stream);
+
+/* dst += src: every pair of src, in ascending (draft, target) order, is added to dst with its
+ * count as the weight, under the admission rule of csd_ocm_update (common pairs add, saturating;
+ * new pairs enter while dst has room, else that entry is dropped and counted once).  Combining
+ * the tables of several calibration runs (Sec. 4.2, Phase 1) is a sequence of merges.  Both
+ * memories live on the same device; src is unchanged.  Allocates temporaries; synchronises. */
+csd_status_t csd_ocm_merge(csd_ocm_t *dst, const csd_ocm_t *src, void *stream);
+
+/* The memory as a file: what calibration hands to deployment (Sec. 4.2: the table is built
+ * offline, then loaded and kept evolving online).  Little-endian layout:
+ *     offset  0  char     magic[8]   "CSDOCM\0\0"
+ *             8  uint32   version    1
+ *            12  uint32   lambda
+ *            16  uint64   n_slots    capacity of the table that was saved
+ *            24  uint64   n          number of stored pairs
+ *            32  uint64   n_dropped  occurrences dropped so far (informational)
+ *            40  uint8    reserved[24]  zero
+ *            64  n records { int32 draft; int32 target; uint32 count; }, strictly ascending
+ *                in (draft, target)
+ * csd_ocm_save writes it (synchronises `stream`; host path).  csd_ocm_load creates a new
+ * memory on `device` with the file's lambda and n_slots slots (0 = as saved) and adds the
+ * records in file order, so a smaller table keeps the first n_slots/2 pairs in (draft, target)
+ * order and counts the rest as dropped.  Errors: IO (cannot open / short / bad magic, version
+ * or order), plus those of csd_ocm_create. */
+csd_status_t csd_ocm_save(const csd_ocm_t *ocm, const char *path, void *stream);
+csd_status_t csd_ocm_load(csd_ocm_t **out, const char *path, uint64_t n_slots, int device);
 
 /* Copy the statistics block to the HOST struct.  Synchronises `stream`. */
 csd_status_t csd_ocm_stats(const csd_ocm_t *ocm, csd_stats_t *host_out, void *stream);

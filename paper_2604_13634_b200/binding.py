@@ -28,6 +28,7 @@ EXPORTS = [
     "csd_host_staging_bytes", "csd_step_host", "csd_verify_static", "csd_ocm_export", "csd_ocm_import", "csd_ocm_stats",
     "csd_scg_threshold", "csd_launch_shape", "csd_set_tuning", "csd_set_overlap", "csd_status_string",
     "csd_sampled_workspace_bytes", "csd_verify_sampled", "csd_step_sampled",
+    "csd_ocm_age", "csd_ocm_merge", "csd_ocm_save", "csd_ocm_load",
 ]
 
 
@@ -90,6 +91,10 @@ def lib():
         "csd_ocm_export": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_uint64, POINTER(c_uint64), c_void_p]),
         "csd_ocm_import": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_uint64, c_void_p]),
         "csd_ocm_stats": (c_int, [c_void_p, POINTER(Stats), c_void_p]),
+        "csd_ocm_age": (c_int, [c_void_p, c_void_p]),
+        "csd_ocm_merge": (c_int, [c_void_p, c_void_p, c_void_p]),
+        "csd_ocm_save": (c_int, [c_void_p, c_char_p, c_void_p]),
+        "csd_ocm_load": (c_int, [POINTER(c_void_p), c_char_p, c_uint64, c_int]),
         "csd_scg_threshold": (c_float, [c_float]),
         "csd_launch_shape": (c_int, [c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
         "csd_set_tuning": (c_int, [c_int, c_int, c_int]),
@@ -213,25 +218,30 @@ class Ocm:
         order = torch.argsort(d * (1 << 32) + t)
         return d[order], t[order], c[order]
 
+    def age(self, stream=None):
+        """Halve every count (rounding down) and forget the pairs that reach zero."""
+        _check(lib().csd_ocm_age(self.handle, _stream_ptr(stream)), "csd_ocm_age")
+
+    def merge(self, other: "Ocm", stream=None):
+        """Add every pair of `other`, with its count, to this memory."""
+        _check(lib().csd_ocm_merge(self.handle, other.handle, _stream_ptr(stream)), "csd_ocm_merge")
+
     def save(self, path: str, stream=None):
-        """Write the stored (draft, target, count) triples, lambda and the slot count to an .npz file:
-        the table of Sec. 4.2 as it is handed from the calibration phase to deployment."""
-        import numpy as np
-        d, t, c = self.export(stream)
-        st = self.stats(stream)
-        np.savez(path, draft=d.numpy().astype(np.int32), target=t.numpy().astype(np.int32),
-                 count=c.numpy().astype(np.uint32), lam=np.uint32(st["lambda"]), n_slots=np.uint64(self.n_slots))
+        """Write the memory to a file in the library's own format (csd_ocm_save): the table of Sec. 4.2 as it
+        is handed from the calibration phase to deployment."""
+        _check(lib().csd_ocm_save(self.handle, os.fsencode(path), _stream_ptr(stream)), "csd_ocm_save")
 
     @classmethod
-    def load(cls, path: str, device: int = 0, n_slots: int = 0, stream=None) -> "Ocm":
-        """A new memory holding the triples of a file written by `save` (n_slots = 0: as saved)."""
-        import numpy as np
-        f = np.load(path)
-        ocm = cls(int(n_slots or f["n_slots"]), int(f["lam"]), device)
-        if len(f["draft"]):
-            dev = ocm.device
-            ocm.import_(torch.from_numpy(f["draft"].astype(np.int32)).to(dev), torch.from_numpy(f["target"].astype(np.int32)).to(dev),
-                        torch.from_numpy(f["count"].astype(np.int64)).to(dev).to(torch.int32), stream)
+    def load(cls, path: str, device: int = 0, n_slots: int = 0) -> "Ocm":
+        """A new memory holding the pairs of a file written by `save` (n_slots = 0: as saved)."""
+        if not torch.cuda.is_available():
+            raise CsdError("a CUDA device is required")
+        h = c_void_p()
+        _check(lib().csd_ocm_load(byref(h), os.fsencode(path), n_slots, device), "csd_ocm_load")
+        ocm = cls.__new__(cls)
+        ocm.handle = h
+        ocm.device = torch.device("cuda", device)
+        ocm.n_slots = ocm.stats()["n_slots"]
         return ocm
 
     def stats(self, stream=None) -> dict:

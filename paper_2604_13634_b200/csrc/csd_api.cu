@@ -2,8 +2,10 @@
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <algorithm>
 #include <cstring>
 #include <mutex>
+#include <vector>
 #include <new>
 
 #include "../../include/csd.h"
@@ -20,6 +22,8 @@ struct csd_ocm {
     uint32_t lambda;
     OcmSlot *slots;
     OcmStatsDev *stats;
+    unsigned long long *age_keys;   // side arrays of csd_ocm_age: n_slots / 2 entries each
+    unsigned int *age_counts;
 };
 
 namespace {
@@ -547,10 +551,18 @@ csd_status_t csd_ocm_create(csd_ocm_t **out, uint64_t n_slots, uint32_t lambda, 
     o->lambda = lambda;
     o->slots = nullptr;
     o->stats = nullptr;
+    o->age_keys = nullptr;
+    o->age_counts = nullptr;
     if (cudaMalloc(&o->slots, n_slots * sizeof(OcmSlot)) != cudaSuccess ||
-        cudaMalloc(&o->stats, sizeof(OcmStatsDev)) != cudaSuccess) {
+        cudaMalloc(&o->stats, sizeof(OcmStatsDev)) != cudaSuccess ||
+        cudaMalloc(&o->age_keys, n_slots / 2 * sizeof(unsigned long long)) != cudaSuccess ||
+        cudaMalloc(&o->age_counts, n_slots / 2 * sizeof(unsigned int)) != cudaSuccess) {
         (void)cudaGetLastError();
-        if (o->slots) cudaFree(o->slots);
+        cudaFree(o->slots);
+        cudaFree(o->stats);
+        cudaFree(o->age_keys);
+        cudaFree(o->age_counts);
+        (void)cudaGetLastError();
         delete o;
         return CSD_ERR_OOM;
     }
@@ -559,6 +571,8 @@ csd_status_t csd_ocm_create(csd_ocm_t **out, uint64_t n_slots, uint32_t lambda, 
     if (rc != CSD_OK) {
         cudaFree(o->slots);
         cudaFree(o->stats);
+        cudaFree(o->age_keys);
+        cudaFree(o->age_counts);
         delete o;
         return rc;
     }
@@ -584,8 +598,10 @@ csd_status_t csd_ocm_destroy(csd_ocm_t *ocm)
     chain_break();
     cudaError_t a = cudaFree(ocm->slots);
     cudaError_t b = cudaFree(ocm->stats);
+    cudaError_t c = cudaFree(ocm->age_keys);
+    cudaError_t d = cudaFree(ocm->age_counts);
     delete ocm;
-    return (a == cudaSuccess && b == cudaSuccess) ? CSD_OK : CSD_ERR_CUDA;
+    return (a == cudaSuccess && b == cudaSuccess && c == cudaSuccess && d == cudaSuccess) ? CSD_OK : CSD_ERR_CUDA;
 }
 
 csd_status_t csd_ocm_set_lambda(csd_ocm_t *ocm, uint32_t lambda)
@@ -836,6 +852,186 @@ csd_status_t csd_ocm_export(const csd_ocm_t *ocm, int32_t *d, int32_t *t, uint32
     return CSD_OK;
 }
 
+csd_status_t csd_ocm_age(csd_ocm_t *ocm, void *stream)
+{
+    if (!ocm) return CSD_ERR_INVALID_ARG;
+    chain_break();
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(&ocm->stats->export_count, 0, sizeof(unsigned long long), st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    unsigned long long blocks = (ocm->n_slots + 255) / 256;
+    const unsigned long long cap = static_cast<unsigned long long>(sm_count()) * 8;
+    if (blocks > cap) blocks = cap;
+    ocm_age_collect_kernel<<<static_cast<unsigned int>(blocks), 256, 0, st>>>(view_of(ocm), ocm->age_keys, ocm->age_counts);
+    if (cudaGetLastError() != cudaSuccess) return CSD_ERR_CUDA;
+    unsigned long long blocks2 = (ocm->n_slots / 2 + 255) / 256;
+    if (blocks2 > cap) blocks2 = cap;
+    ocm_age_reinsert_kernel<<<static_cast<unsigned int>(blocks2), 256, 0, st>>>(view_of(ocm), ocm->age_keys, ocm->age_counts);
+    return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_CUDA;
+}
+
+// ---- the memory as sorted triples on the host: file format and merge ------------------------
+namespace {
+
+struct Triple {
+    int32_t d, t;
+    uint32_t c;
+};
+
+// Every stored pair, sorted by (draft, target).  Synchronises `stream`.
+csd_status_t sorted_triples(const csd_ocm *ocm, std::vector<Triple> &out, cudaStream_t st)
+{
+    out.clear();
+    const uint64_t cap = ocm->n_slots / 2;
+    int32_t *dd = nullptr, *dt = nullptr;
+    uint32_t *dc = nullptr;
+    if (cudaMalloc(&dd, cap * 4) != cudaSuccess || cudaMalloc(&dt, cap * 4) != cudaSuccess || cudaMalloc(&dc, cap * 4) != cudaSuccess) {
+        (void)cudaGetLastError();
+        cudaFree(dd); cudaFree(dt); cudaFree(dc);
+        (void)cudaGetLastError();
+        return CSD_ERR_OOM;
+    }
+    uint64_t n = 0;
+    csd_status_t rc = csd_ocm_export(ocm, dd, dt, dc, cap, &n, st);
+    if (rc == CSD_OK) {
+        if (n > cap) n = cap;
+        std::vector<int32_t> hd(n), ht(n);
+        std::vector<uint32_t> hc(n);
+        bool ok = true;
+        if (n) {
+            ok = cudaMemcpyAsync(hd.data(), dd, n * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+                 cudaMemcpyAsync(ht.data(), dt, n * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+                 cudaMemcpyAsync(hc.data(), dc, n * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+                 cudaStreamSynchronize(st) == cudaSuccess;
+        }
+        if (!ok) {
+            (void)cudaGetLastError();
+            rc = CSD_ERR_CUDA;
+        } else {
+            out.resize(n);
+            for (uint64_t j = 0; j < n; ++j) out[j] = Triple{hd[j], ht[j], hc[j]};
+            std::sort(out.begin(), out.end(), [](const Triple &a, const Triple &b) { return a.d != b.d ? a.d < b.d : a.t < b.t; });
+        }
+    }
+    cudaFree(dd); cudaFree(dt); cudaFree(dc);
+    return rc;
+}
+
+// count[(d, t)] += c for the triples in order.  Synchronises `stream`.
+csd_status_t add_triples(csd_ocm *ocm, const std::vector<Triple> &tr, cudaStream_t st)
+{
+    const size_t n = tr.size();
+    if (n == 0) return CSD_OK;
+    std::vector<int32_t> hd(n), ht(n);
+    std::vector<uint32_t> hc(n);
+    for (size_t j = 0; j < n; ++j) { hd[j] = tr[j].d; ht[j] = tr[j].t; hc[j] = tr[j].c; }
+    int32_t *dd = nullptr, *dt = nullptr;
+    uint32_t *dc = nullptr;
+    if (cudaMalloc(&dd, n * 4) != cudaSuccess || cudaMalloc(&dt, n * 4) != cudaSuccess || cudaMalloc(&dc, n * 4) != cudaSuccess) {
+        (void)cudaGetLastError();
+        cudaFree(dd); cudaFree(dt); cudaFree(dc);
+        (void)cudaGetLastError();
+        return CSD_ERR_OOM;
+    }
+    csd_status_t rc = CSD_OK;
+    if (cudaMemcpyAsync(dd, hd.data(), n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dt, ht.data(), n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dc, hc.data(), n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        rc = CSD_ERR_CUDA;
+    }
+    if (rc == CSD_OK) rc = csd_ocm_import(ocm, dd, dt, dc, n, st);
+    if (cudaStreamSynchronize(st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        rc = rc == CSD_OK ? CSD_ERR_CUDA : rc;
+    }
+    cudaFree(dd); cudaFree(dt); cudaFree(dc);
+    return rc;
+}
+
+constexpr char kFileMagic[8] = {'C', 'S', 'D', 'O', 'C', 'M', '\0', '\0'};
+constexpr uint32_t kFileVersion = 1;
+
+struct FileHeader {            // 64 bytes, little-endian, see csd.h
+    char magic[8];
+    uint32_t version, lambda;
+    uint64_t n_slots, n, n_dropped;
+    uint8_t reserved[24];
+};
+static_assert(sizeof(FileHeader) == 64, "file header layout");
+static_assert(sizeof(Triple) == 12, "file record layout");
+
+}  // namespace
+
+csd_status_t csd_ocm_merge(csd_ocm_t *dst, const csd_ocm_t *src, void *stream)
+{
+    if (!dst || !src || dst == src) return CSD_ERR_INVALID_ARG;
+    if (dst->device != src->device) return CSD_ERR_UNSUPPORTED;
+    std::vector<Triple> tr;
+    const csd_status_t rc = sorted_triples(src, tr, static_cast<cudaStream_t>(stream));
+    if (rc != CSD_OK) return rc;
+    return add_triples(dst, tr, static_cast<cudaStream_t>(stream));
+}
+
+csd_status_t csd_ocm_save(const csd_ocm_t *ocm, const char *path, void *stream)
+{
+    if (!ocm || !path) return CSD_ERR_INVALID_ARG;
+    std::vector<Triple> tr;
+    csd_status_t rc = sorted_triples(ocm, tr, static_cast<cudaStream_t>(stream));
+    if (rc != CSD_OK) return rc;
+    csd_stats_t st;
+    rc = csd_ocm_stats(ocm, &st, stream);
+    if (rc != CSD_OK) return rc;
+    FileHeader h;
+    std::memset(&h, 0, sizeof h);
+    std::memcpy(h.magic, kFileMagic, 8);
+    h.version = kFileVersion;
+    h.lambda = ocm->lambda;
+    h.n_slots = ocm->n_slots;
+    h.n = tr.size();
+    h.n_dropped = st.n_dropped;
+    FILE *f = std::fopen(path, "wb");
+    if (!f) return CSD_ERR_IO;
+    bool ok = std::fwrite(&h, sizeof h, 1, f) == 1;
+    if (ok && !tr.empty()) ok = std::fwrite(tr.data(), sizeof(Triple), tr.size(), f) == tr.size();
+    ok = (std::fclose(f) == 0) && ok;
+    return ok ? CSD_OK : CSD_ERR_IO;
+}
+
+csd_status_t csd_ocm_load(csd_ocm_t **out, const char *path, uint64_t n_slots, int device)
+{
+    if (!out || !path) return CSD_ERR_INVALID_ARG;
+    *out = nullptr;
+    FILE *f = std::fopen(path, "rb");
+    if (!f) return CSD_ERR_IO;
+    FileHeader h;
+    std::vector<Triple> tr;
+    bool ok = std::fread(&h, sizeof h, 1, f) == 1 && std::memcmp(h.magic, kFileMagic, 8) == 0 && h.version == kFileVersion &&
+              h.n <= (1ull << 29);
+    if (ok) {
+        tr.resize(h.n);
+        if (h.n) ok = std::fread(tr.data(), sizeof(Triple), h.n, f) == h.n;
+    }
+    std::fclose(f);
+    if (!ok) return CSD_ERR_IO;
+    for (size_t j = 0; j < tr.size(); ++j) {      // a well-formed file: valid pairs, strictly ascending
+        if (tr[j].d < 0 || tr[j].t < 0) return CSD_ERR_IO;
+        if (j && !(tr[j - 1].d < tr[j].d || (tr[j - 1].d == tr[j].d && tr[j - 1].t < tr[j].t))) return CSD_ERR_IO;
+    }
+    csd_ocm_t *o = nullptr;
+    csd_status_t rc = csd_ocm_create(&o, n_slots ? n_slots : h.n_slots, h.lambda, device);
+    if (rc != CSD_OK) return rc;
+    rc = add_triples(o, tr, nullptr);
+    if (rc != CSD_OK) {
+        csd_ocm_destroy(o);
+        return rc;
+    }
+    *out = o;
+    return CSD_OK;
+}
+
 csd_status_t csd_ocm_stats(const csd_ocm_t *ocm, csd_stats_t *host_out, void *stream)
 {
     if (!ocm || !host_out) return CSD_ERR_INVALID_ARG;
@@ -908,6 +1104,7 @@ const char *csd_status_string(csd_status_t status)
         case CSD_ERR_OOM: return "out of memory";
         case CSD_ERR_UNSUPPORTED: return "unsupported shape";
         case CSD_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case CSD_ERR_IO: return "file cannot be opened, read or written, or is not a memory file";
     }
     return "unknown status";
 }

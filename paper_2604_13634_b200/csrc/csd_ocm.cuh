@@ -367,6 +367,69 @@ __global__ void __launch_bounds__(1024) ocm_update_kernel(OcmView tb, const int 
     }
 }
 
+// ---- ageing: every count halves (rounding down), pairs that reach zero are forgotten -----------
+// Two launches.  The first moves the survivors (key, count / 2) to a side array and empties every
+// slot; the second inserts them again, each at its own probe position in the emptied table (open
+// addressing cannot delete in place: an emptied slot in the middle of a probe run would hide the keys
+// behind it).  The table's contents never depend on slot positions, so the rebuilt table is the
+// same table.  `cursor` (the statistics block's export cursor) counts the survivors.
+__global__ void ocm_age_collect_kernel(OcmView tb, unsigned long long *keys, unsigned int *counts)
+{
+    const unsigned long long stride = static_cast<unsigned long long>(gridDim.x) * blockDim.x;
+    for (unsigned long long i = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x; i <= tb.mask;
+         i += stride) {
+        unsigned long long k;
+        unsigned int c;
+        load_slot(tb.slots + i, k, c);
+        if (k == kEmptyKey) continue;
+        const unsigned int half = c >> 1;
+        if (half) {
+            const unsigned long long pos = atomicAdd(&tb.stats->export_count, 1ull);
+            if (CSD_CHECKED(pos < tb.key_limit, tb.stats, 20u)) {     // at most key_limit pairs are ever stored
+                keys[pos] = k;
+                counts[pos] = half;
+            }
+        }
+        uint4 v;
+        v.x = 0xffffffffu; v.y = 0xffffffffu; v.z = 0u; v.w = 0u;
+        __stcg(reinterpret_cast<uint4 *>(tb.slots + i), v);
+    }
+}
+
+__global__ void ocm_age_reinsert_kernel(OcmView tb, const unsigned long long *keys, const unsigned int *counts)
+{
+    __shared__ bool last;
+    unsigned long long n = __ldcg(&tb.stats->export_count);
+    if (n > tb.key_limit) n = tb.key_limit;
+    const unsigned long long stride = static_cast<unsigned long long>(gridDim.x) * blockDim.x;
+    for (unsigned long long j = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += stride) {
+        const unsigned long long key = __ldcg(keys + j);
+        unsigned long long slot = mix64(key) & tb.mask;
+        bool placed = false;
+        for (unsigned long long probe = 0; probe <= tb.mask; ++probe) {      // keys are distinct: claim the first empty slot
+            if (atomicCAS(&tb.slots[slot].key, kEmptyKey, key) == kEmptyKey) {
+                tb.slots[slot].count = __ldcg(counts + j);
+                placed = true;
+                break;
+            }
+            slot = (slot + 1) & tb.mask;
+        }
+        if (!placed) atomicOr(&tb.stats->flags, 0x4u);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        last = atomicAdd(&tb.stats->ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (last && threadIdx.x == 0) {
+        __threadfence();
+        tb.stats->n_keys = n;
+        tb.stats->n_keys_start = n;
+        tb.stats->ticket = 0u;
+    }
+}
+
 __global__ void ocm_export_kernel(OcmView tb, int *d, int *t, unsigned int *cnt, unsigned long long cap)
 {
     const unsigned long long stride = static_cast<unsigned long long>(gridDim.x) * blockDim.x;

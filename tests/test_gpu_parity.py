@@ -346,15 +346,27 @@ def test_update_kernel_regimes_and_import_export():
 
 
 def test_memory_survives_a_file(tmp_path):
-    """Calibration hands its table to deployment through a file (Sec. 4.2, Phase 1): save, load, same triples,
-    same lambda; a smaller table admits the saved pairs in sorted order up to its own limit."""
+    """Calibration hands its table to deployment through a file (Sec. 4.2, Phase 1): csd_ocm_save, csd_ocm_load,
+    same triples, same lambda; the bytes on disk are the documented layout; a smaller table admits the saved pairs
+    in sorted order up to its own limit; a damaged file is refused."""
+    import struct
+    from paper_2604_13634_b200 import CsdError
     g = torch.Generator(device="cuda").manual_seed(11)
     ocm = Ocm(4096, 3)
     d = torch.randint(0, 50, (5000,), generator=g, device="cuda", dtype=torch.int32)
     t = torch.randint(0, 50, (5000,), generator=g, device="cuda", dtype=torch.int32)
     ocm.update(d, t)
-    path = str(tmp_path / "table.npz")
+    mem = ORACLE.OCM(4096, 3)
+    mem.update(zip(d.cpu().tolist(), t.cpu().tolist()))
+    path = str(tmp_path / "table.ocm")
     ocm.save(path)
+    raw = open(path, "rb").read()
+    magic, version, lam, n_slots, n, n_dropped = struct.unpack_from("<8sIIQQQ", raw, 0)
+    assert (magic, version, lam, n_slots, n, n_dropped) == (b"CSDOCM\0\0", 1, 3, 4096, mem.n_keys, mem.n_dropped)
+    assert raw[40:64] == bytes(24) and len(raw) == 64 + 12 * n
+    rec = np.frombuffer(raw, dtype=np.dtype([("d", "<i4"), ("t", "<i4"), ("c", "<u4")]), offset=64)
+    rd, rt, rc = mem.export()
+    assert np.array_equal(rec["d"], rd) and np.array_equal(rec["t"], rt) and np.array_equal(rec["c"], rc)
     back = Ocm.load(path)
     assert all(torch.equal(a, b) for a, b in zip(ocm.export(), back.export()))
     assert back.stats()["lambda"] == 3 and back.n_slots == 4096
@@ -363,8 +375,76 @@ def test_memory_survives_a_file(tmp_path):
     fd, ft, fc = ocm.export()
     assert small.stats()["n_keys"] == 128 and small.stats()["n_dropped"] == len(fd) - 128
     assert torch.equal(sd, fd[:128]) and torch.equal(st_, ft[:128]) and torch.equal(sc, fc[:128])
+    for damaged in (raw[:40], b"X" + raw[1:], raw[:64] + raw[76:88] + raw[64:76] + raw[88:], raw[:-5]):
+        open(path, "wb").write(damaged)
+        with pytest.raises(CsdError):
+            Ocm.load(path)
+    with pytest.raises(CsdError):
+        Ocm.load(str(tmp_path / "missing.ocm"))
     for o in (ocm, back, small):
         o.close()
+
+
+def test_merge_of_overlapping_weighted_tables():
+    """Two tables with common and distinct pairs: dst += src equals the oracle's merge (update with the
+    source's sorted triples as weighted entries), with room for everything and across the capacity limit."""
+    g = torch.Generator(device="cuda").manual_seed(12)
+    for dst_slots, vocab in ((4096, 40), (256, 40), (64, 12)):
+        a, b = Ocm(dst_slots, 2), Ocm(4096, 2)
+        ma, mb = ORACLE.OCM(dst_slots, 2), ORACLE.OCM(4096, 2)
+        for ocm, mem, n, lo in ((a, ma, 700, 0), (b, mb, 3000, vocab // 3)):
+            d = torch.randint(lo, lo + vocab, (n,), generator=g, device="cuda", dtype=torch.int32)
+            t = torch.randint(lo, lo + vocab, (n,), generator=g, device="cuda", dtype=torch.int32)
+            ocm.update(d, t)
+            mem.update(zip(d.cpu().tolist(), t.cpu().tolist()))
+        common = set(ma.table) & set(mb.table)
+        assert common and set(mb.table) - set(ma.table)
+        a.merge(b)
+        ma.merge(mb)
+        st = compare_memory(a, ma)
+        compare_memory(b, mb)                                   # the source is unchanged
+        if dst_slots < 4096:
+            assert st["n_keys"] == dst_slots // 2 and st["n_dropped"] > 0
+        a.merge(b); ma.merge(mb)                                # once more: now every admitted pair is common
+        compare_memory(a, ma)
+        a.close(); b.close()
+
+
+def test_ageing_matches_the_oracle():
+    """csd_ocm_age on its own, and inside a run of the contention workload with a 512-slot table that is aged
+    every 40 steps: the table fills, ageing frees room, new pairs are admitted again, and the memory equals the oracle's after every step."""
+    g = torch.Generator(device="cuda").manual_seed(13)
+    for n_slots, n, vocab in ((1 << 14, 20000, 90), (64, 200, 7), (256, 3000, 30)):
+        ocm, mem = Ocm(n_slots, 1), ORACLE.OCM(n_slots, 1)
+        for rep in range(4):
+            d = torch.randint(0, vocab, (n,), generator=g, device="cuda", dtype=torch.int32)
+            t = torch.randint(0, vocab, (n,), generator=g, device="cuda", dtype=torch.int32)
+            ocm.update(d, t); mem.update(zip(d.cpu().tolist(), t.cpu().tolist()))
+            compare_memory(ocm, mem)
+            ocm.age(); mem.age()
+            compare_memory(ocm, mem)
+        for _ in range(34):                                     # down to nothing
+            ocm.age(); mem.age()
+        assert compare_memory(ocm, mem)["n_keys"] == 0
+        ocm.close()
+    wl = dataclasses.replace(WORKLOADS["ocm_contention"], B=16, V=32768, ocm_slots=512)
+    syn = Synth(wl, 0, "cuda")
+    ocm, mem = Ocm(wl.ocm_slots, wl.lam), ORACLE.OCM(wl.ocm_slots, wl.lam)
+    buf = StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, diag=True)
+    full_seen = forgotten = 0
+    for s in range(160):
+        z, d = syn.step(s)
+        csd_step(z, d, ocm, 0.3, buf)
+        compare(buf, oracle_step(z, d, mem, 0.3))
+        full_seen += mem.n_keys == mem.limit
+        if (s + 1) % 40 == 0:
+            before = mem.n_keys
+            ocm.age(); mem.age()
+            forgotten += before - mem.n_keys
+        compare_memory(ocm, mem)
+    st = ocm.stats()
+    assert full_seen > 0 and forgotten > 100 and st["rescues"] > 0 and st["flags"] == 0
+    ocm.close()
 
 
 def test_host_entry_point_matches_device_entry_point():
