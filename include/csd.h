@@ -19,7 +19,8 @@
  *     memory behind a csd_ocm_t.
  *   - All work is enqueued on the CUDA stream passed as `stream` (a cudaStream_t
  *     cast to void*; NULL is the legacy default stream).  Nothing synchronises
- *     unless documented.  Calls on one csd_ocm_t must be stream-ordered.
+ *     unless documented.  Calls on one csd_ocm_t must be stream-ordered (but see
+ *     csd_ocm_set_shared).
  *   - Every function returns a csd_status_t and never throws or aborts.  Misuse
  *     that the host can see is refused before anything is launched.  Conditions
  *     only the device can see (a NaN logit, a draft id outside [0,V), a full
@@ -126,6 +127,26 @@ csd_status_t csd_ocm_destroy(csd_ocm_t *ocm);
 
 /* Change lambda for subsequent calls (host side; stream-ordered like any call). */
 csd_status_t csd_ocm_set_lambda(csd_ocm_t *ocm, uint32_t lambda);
+
+/* Several streams on one memory (the paper's Limitations leave concurrent updates of T open; this is
+ * the library's reading).  By default all calls on one csd_ocm_t are stream-ordered, which is what makes
+ * every look-up of a step see exactly the step-start counts and admission near the key limit follow the
+ * canonical order.  With sharing switched on, csd_step / csd_step_sampled / csd_ocm_update /
+ * csd_ocm_import calls on DIFFERENT streams (each with its own workspace and output buffers) may run at
+ * the same time on one memory:
+ *   - every recorded pair is counted exactly once whatever the interleaving (counts are the multiset
+ *     union of all streams' recorded pairs, as long as no pair is dropped for lack of room);
+ *   - a look-up sees the count of its pair at some moment between the start and the end of its own
+ *     step: pairs recorded by the SAME step are never seen (they are added after its last look-up),
+ *     pairs that other streams record meanwhile may or may not be;
+ *   - the table never holds more than n_slots/2 pairs; which new pairs are admitted when it is nearly
+ *     full depends on arrival order (each new pair takes one unit of the remaining room atomically, and
+ *     claims in flight -- at most B*K per step, 1024 per bulk update -- count against the room, so within
+ *     that margin of the limit a new pair may be dropped, and counted in n_dropped, although room remains).
+ * Calls that rebuild or read the whole table (csd_ocm_reset / age / merge / export / save) must still
+ * not run beside anything else.  Host function; set it while no work on the memory is in flight
+ * (switching it off synchronises the device). */
+csd_status_t csd_ocm_set_shared(csd_ocm_t *ocm, int enable);
 
 /* ---- one verification step ---------------------------------------------------- */
 

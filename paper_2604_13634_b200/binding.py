@@ -28,7 +28,7 @@ EXPORTS = [
     "csd_host_staging_bytes", "csd_step_host", "csd_verify_static", "csd_ocm_export", "csd_ocm_import", "csd_ocm_stats",
     "csd_scg_threshold", "csd_launch_shape", "csd_set_tuning", "csd_set_overlap", "csd_status_string",
     "csd_sampled_workspace_bytes", "csd_verify_sampled", "csd_step_sampled",
-    "csd_ocm_age", "csd_ocm_merge", "csd_ocm_save", "csd_ocm_load",
+    "csd_ocm_age", "csd_ocm_merge", "csd_ocm_save", "csd_ocm_load", "csd_ocm_set_shared",
 ]
 
 
@@ -92,6 +92,7 @@ def lib():
         "csd_ocm_import": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_uint64, c_void_p]),
         "csd_ocm_stats": (c_int, [c_void_p, POINTER(Stats), c_void_p]),
         "csd_ocm_age": (c_int, [c_void_p, c_void_p]),
+        "csd_ocm_set_shared": (c_int, [c_void_p, c_int]),
         "csd_ocm_merge": (c_int, [c_void_p, c_void_p, c_void_p]),
         "csd_ocm_save": (c_int, [c_void_p, c_char_p, c_void_p]),
         "csd_ocm_load": (c_int, [POINTER(c_void_p), c_char_p, c_uint64, c_int]),
@@ -217,6 +218,10 @@ class Ocm:
         c = c[:k].cpu().to(torch.int64) & 0xFFFFFFFF
         order = torch.argsort(d * (1 << 32) + t)
         return d[order], t[order], c[order]
+
+    def set_shared(self, enable: bool):
+        """Allow steps and updates on different streams to run on this memory at the same time."""
+        _check(lib().csd_ocm_set_shared(self.handle, 1 if enable else 0), "csd_ocm_set_shared")
 
     def age(self, stream=None):
         """Halve every count (rounding down) and forget the pairs that reach zero."""

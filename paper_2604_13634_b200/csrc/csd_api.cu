@@ -22,6 +22,7 @@ struct csd_ocm {
     uint32_t lambda;
     OcmSlot *slots;
     OcmStatsDev *stats;
+    int shared;                     // csd_ocm_set_shared
     unsigned long long *age_keys;   // side arrays of csd_ocm_age: n_slots / 2 entries each
     unsigned int *age_counts;
 };
@@ -194,7 +195,10 @@ Shape pick_shape(int B, int K, int V, csd_dtype_t dt, bool overlap)
     s.total_units = rows * s.units_per_row;
     long long blocks = static_cast<long long>(sm_count()) * ctas_per_sm;
     if (blocks > rows * 64) blocks = rows * 64;
-    if (blocks > (s.total_units + 15) / 16) blocks = (s.total_units + 15) / 16;
+    // at least 8 KiB per block; for a launch that runs alone 32 KiB (one full iteration for each of eight
+    // warps): below that more blocks only mean more partial results to exchange and fold at the end
+    const long long min_units = overlap ? 16 : 64;
+    if (blocks > (s.total_units + min_units - 1) / min_units) blocks = (s.total_units + min_units - 1) / min_units;
     if (blocks < 1) blocks = 1;
     s.grid = static_cast<int>(blocks);
     // span boundaries lie at floor(c*T/G): at most ceil((U-1)*G/T) of them fall inside a row
@@ -245,6 +249,7 @@ OcmView view_of(const csd_ocm *o)
     v.key_limit = o->n_slots / 2;
     v.lambda = o->lambda;
     v.stats = o->stats;
+    v.shared = o->shared;
     return v;
 }
 
@@ -294,7 +299,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.slots_per_row = s.slots_per_row;
     p.chunk_units = s.chunk_units;
     p.total_units = s.total_units;
-    p.narrow = (s.total_units + 1) * (static_cast<long long>(s.grid) + 1) < (1ll << 32) ? 1 : 0;
+    p.narrow = ((s.total_units + 1) * (static_cast<long long>(s.grid) + 1) < (1ll << 32) && s.total_units * 40 < (1ll << 32)) ? 1 : 0;
     if (track_layout) {
         const unsigned long long sig[3] = {
             (static_cast<unsigned long long>(static_cast<unsigned int>(B)) << 32) | static_cast<unsigned int>(K),
@@ -549,6 +554,7 @@ csd_status_t csd_ocm_create(csd_ocm_t **out, uint64_t n_slots, uint32_t lambda, 
     o->device = device;
     o->n_slots = n_slots;
     o->lambda = lambda;
+    o->shared = 0;
     o->slots = nullptr;
     o->stats = nullptr;
     o->age_keys = nullptr;
@@ -608,6 +614,22 @@ csd_status_t csd_ocm_set_lambda(csd_ocm_t *ocm, uint32_t lambda)
 {
     if (!ocm) return CSD_ERR_INVALID_ARG;
     ocm->lambda = lambda;
+    return CSD_OK;
+}
+
+csd_status_t csd_ocm_set_shared(csd_ocm_t *ocm, int enable)
+{
+    if (!ocm) return CSD_ERR_INVALID_ARG;
+    chain_break();
+    if (ocm->shared && !enable) {
+        // back to a single writer: the key count the ordered path starts from is brought up to date
+        if (cudaDeviceSynchronize() != cudaSuccess ||
+            cudaMemcpy(&ocm->stats->n_keys_start, &ocm->stats->n_keys, sizeof(unsigned long long), cudaMemcpyDeviceToDevice) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CSD_ERR_CUDA;
+        }
+    }
+    ocm->shared = enable ? 1 : 0;
     return CSD_OK;
 }
 

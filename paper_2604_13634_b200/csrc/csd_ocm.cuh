@@ -62,6 +62,7 @@ struct OcmView {
     unsigned long long key_limit;  // n_slots / 2
     unsigned int lambda;
     OcmStatsDev *stats;
+    int shared;                    // 1: other streams may be updating the table while this launch runs
 };
 
 __device__ __forceinline__ unsigned long long make_key(int d, int t)
@@ -176,6 +177,59 @@ __device__ __forceinline__ long long ocm_reserve(const OcmView &tb, unsigned lon
     }
     atomicOr(&tb.stats->flags, 0x4u);
     return -1;
+}
+
+// ---- admission when several streams update one table at the same time ------------------------
+// With a single writer the room for a batch's new keys is established before anyone inserts.  With
+// concurrent writers every new key first takes one unit of the key budget from the live key count and
+// gives it back if it turns out not to need it, so the table never holds more than key_limit keys
+// whatever the interleaving; which keys get in near the limit then depends on arrival order.  Units
+// that are held for the moment count against the room: while fewer keys of room remain than claims
+// are in flight (at most B*K per step launch, 1024 per bulk update), a new key may be refused although
+// room remains.  Far from the limit nothing is ever refused.
+__device__ __forceinline__ bool ocm_take_key_budget(const OcmView &tb)
+{
+    const unsigned long long old = atomicAdd(&tb.stats->n_keys, 1ull);
+    if (old < tb.key_limit) return true;
+    atomicAdd(&tb.stats->n_keys, ~0ull);   // minus one
+    return false;
+}
+
+// Slot of `key`, claiming an empty slot (count 0) if it is absent and the budget allows; -1 if the table
+// is at its limit (or, flagged, if the probe wrapped around).  `from` as in ocm_reserve.
+__device__ __forceinline__ long long ocm_reserve_shared(const OcmView &tb, unsigned long long key, long long from = -1)
+{
+    unsigned long long slot = from >= 0 ? static_cast<unsigned long long>(from) : (mix64(key) & tb.mask);
+    bool budget = false;
+    for (unsigned long long probe = 0; probe <= tb.mask; ++probe) {
+        unsigned long long *kp = &tb.slots[slot].key;
+        unsigned long long k = *reinterpret_cast<volatile unsigned long long *>(kp);
+        if (k == kEmptyKey) {
+            if (!budget) {
+                if (!ocm_take_key_budget(tb)) return -1;
+                budget = true;
+            }
+            k = atomicCAS(kp, kEmptyKey, key);
+            if (k == kEmptyKey) return static_cast<long long>(slot);       // claimed: the budget unit is this key's
+        }
+        if (k == key) {
+            if (budget) atomicAdd(&tb.stats->n_keys, ~0ull);               // somebody else brought the key in
+            return static_cast<long long>(slot);
+        }
+        slot = (slot + 1) & tb.mask;
+    }
+    if (budget) atomicAdd(&tb.stats->n_keys, ~0ull);
+    atomicOr(&tb.stats->flags, 0x4u);
+    return -1;
+}
+
+__device__ __forceinline__ void ocm_insert_or_add_shared(const OcmView &tb, unsigned long long key, unsigned int w)
+{
+    const long long slot = ocm_reserve_shared(tb, key);
+    if (slot >= 0)
+        ocm_add(tb, static_cast<unsigned long long>(slot), w);
+    else
+        atomicAdd(&tb.stats->n_dropped, 1ull);
 }
 
 // Increment if present, else count a dropped occurrence (table full: nothing is admitted).
@@ -343,7 +397,17 @@ __global__ void __launch_bounds__(1024) ocm_update_kernel(OcmView tb, const int 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const unsigned long long nk0 = __ldcg(&tb.stats->n_keys_start);
-    if (nk0 + static_cast<unsigned long long>(n) <= tb.key_limit) {
+    if (tb.shared) {
+        // One block only: every thread that meets an absent key holds a unit of the key budget for the
+        // duration of its claim, and a unit held is room that other writers cannot use meanwhile; a single
+        // block bounds what one bulk update can hold at a time.
+        if (blockIdx.x == 0) {
+            for (long long j = threadIdx.x; j < n; j += blockDim.x) {
+                unsigned long long key;
+                if (entry_key(rd, rt, j, key)) ocm_insert_or_add_shared(tb, key, w ? __ldcg(w + j) : 1u);
+            }
+        }
+    } else if (nk0 + static_cast<unsigned long long>(n) <= tb.key_limit) {
         const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
         for (long long j = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += stride) {
             unsigned long long key;
@@ -352,6 +416,7 @@ __global__ void __launch_bounds__(1024) ocm_update_kernel(OcmView tb, const int 
     } else if (blockIdx.x == 0) {
         ocm_update_group<true>(tb, rd, rt, w, n, sc, threadIdx.x, blockDim.x);
     }
+    if (tb.shared) return;     // other launches may be counting in as well; n_keys_start is not used while shared
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();

@@ -109,6 +109,14 @@ __device__ __forceinline__ void st_release(unsigned int *p, unsigned int v)
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void fence_acq_rel() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+// Arrival counter: the add releases everything this thread has observed or written so far (and, through a
+// preceding __syncwarp, what the other lanes of its warp wrote) and acquires what earlier arrivals released.
+__device__ __forceinline__ unsigned int atom_add_acq_rel(unsigned int *p, unsigned int v)
+{
+    unsigned int old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 
 constexpr int kFlagPolls = 1 << 14;   // bounded: a few milliseconds, then the hardware wait takes over
 
@@ -424,6 +432,10 @@ struct BlockState {
     Partial chunk_part[kMaxChunks];
     int n_todo;                         // batch rows this block has to finalise in this window ...
     int todo_b[kMaxSegs];               // ... and which
+    // Draft tokens of the first two batch rows the block touches, fetched when the block starts (their logits
+    // are requested into L2 at the same time): a row this block then finalises finds them here.
+    int pre_b[2];
+    int pre_d[2][CSD_MAX_K];
 };
 
 // ---- S2..S5 for one batch row, by one warp ------------------------------------------
@@ -435,7 +447,7 @@ struct RowScratch {
     int parts[CSD_MAX_K + 1];   // number of blocks touching the row
 };
 
-enum UpdateRegime { kRegimeRoom = 0, kRegimeFull = 1, kRegimeTransition = 2 };
+enum UpdateRegime { kRegimeRoom = 0, kRegimeFull = 1, kRegimeTransition = 2, kRegimeShared = 3 };
 
 // Which of the three update regimes this step is in.  n_keys_start is written when the
 // previous update finished, so every warp of the launch computes the same answer.
@@ -526,24 +538,27 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, const ScratchCopy
 }
 
 template <typename L>
-__device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, int lane, RowScratch &rs)
+__device__ __forceinline__ const typename L::elem *logit_row(const StepParams &p, long long b, int i)
 {
-    using E = typename L::elem;
+    return reinterpret_cast<const typename L::elem *>(p.logits) + b * p.stride_b + static_cast<long long>(i) * p.stride_k;
+}
+
+__device__ __forceinline__ void prefetch_l2(const void *ptr) { asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr)); }
+
+template <typename L>
+__device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, int lane, RowScratch &rs, const BlockState &bs)
+{
     const int K = p.K;
 
-    // S2 (first half): the draft tokens and their logits do not depend on the
-    // reduction, so their loads are issued before the partials are folded.
+    // S2 (first half): the draft tokens and their logits do not depend on the reduction: the tokens were
+    // fetched when the block started (else they are loaded now), the logits' loads are issued before the
+    // partials are folded.
     int d = -1;
-    bool valid = false;
     float zd = __int_as_float(0x7fc00000);
-    if (lane < K) {
-        d = __ldg(p.draft + (size_t)b * K + lane);
-        valid = static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V);
-        if (valid) {
-            const E *rowp = reinterpret_cast<const E *>(p.logits) + (size_t)b * p.stride_b + (size_t)lane * p.stride_k;
-            zd = L::load_elem(rowp, d);
-        }
-    }
+    const int pre = bs.pre_b[0] == b ? 0 : (bs.pre_b[1] == b ? 1 : -1);
+    if (lane < K) d = pre >= 0 ? bs.pre_d[pre][lane] : __ldg(p.draft + (size_t)b * K + lane);
+    const bool valid = lane < K && static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V);
+    if (valid) zd = L::load_elem(logit_row<L>(p, b, lane), d);
     const ScratchCopy sc = scratch_of(p, seq);
     fold_rows(p, sc, b, lane, rs);
 
@@ -553,7 +568,7 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
     wait_completed(p, seq);
     // S3.  The update regime (one load, used only after the look-up) is requested first so
     // that it travels together with the probe.
-    const int regime = p.do_update ? update_regime(p) : kRegimeFull;
+    const int regime = p.do_update ? (p.ocm.shared ? kRegimeShared : update_regime(p)) : kRegimeFull;
     bool match = false, ok = false;
     int t = -1;
     unsigned int cnt = 0;
@@ -606,6 +621,7 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
             int hint = kHintNone;
             if (record) {
                 if (slot < 0 && regime == kRegimeRoom) slot = ocm_reserve(p.ocm, make_key(d, t), empty_slot);
+                if (slot < 0 && regime == kRegimeShared) slot = ocm_reserve_shared(p.ocm, make_key(d, t), empty_slot);
                 hint = slot < 0 ? kHintAbsent : static_cast<int>(slot);
                 const unsigned int room = 0xffffffffu - static_cast<unsigned int>(p.B * p.K);
                 if (slot >= 0 && cnt > room) hint |= kHintCareful;
@@ -693,8 +709,7 @@ __device__ void publish_parts(const StepParams &p, BlockState &bs, int first_row
             st_partial_cg(sc.partials + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
         my_b = row / K1;
     }
-    __threadfence();
-    __syncwarp();
+    __syncwarp();         // every lane's partial before any lane's ticket (the ticket's add releases them)
     const int below_b = __shfl_down_sync(kFull, my_b, 1);
     bool completes = false;
     if (lane < nseg) {
@@ -703,31 +718,32 @@ __device__ void publish_parts(const StepParams &p, BlockState &bs, int first_row
         if (closes) {
             const long long u0 = static_cast<long long>(my_b) * K1 * U;
             const unsigned int expected = owner_of(p, u0 + static_cast<long long>(K1) * U - 1) - owner_of(p, u0) + 1;
-            completes = atomicAdd(sc.b_ticket + my_b, 1u) == expected - 1;
+            // the last arrival has acquired the other blocks' partials of the row; this block's warps read
+            // them after the block barrier that follows
+            completes = atom_add_acq_rel(sc.b_ticket + my_b, 1u) == expected - 1;
         }
     }
     const unsigned int todo = __ballot_sync(kFull, completes);
     if (completes && CSD_INDEX_OK(my_b >= 0 && my_b < p.B, p.ocm.stats, 2u)) bs.todo_b[__popc(todo & ((1u << lane) - 1u))] = my_b;
     if (lane == 0) bs.n_todo = __popc(todo);
-    __threadfence();      // the other blocks' partials of those rows, before this block's warps read them
 }
 
 // S2..S5 of batch row b by one warp, and, if that was the launch's last row, S6.
 template <typename L>
-__device__ void finalize_and_update(const StepParams &p, unsigned int seq, int b, int lane, RowScratch &rs, CanonScratch &canon)
+__device__ void finalize_and_update(const StepParams &p, unsigned int seq, int b, int lane, RowScratch &rs, CanonScratch &canon,
+                                    const BlockState &bs)
 {
     const ScratchCopy sc = scratch_of(p, seq);
-    const int regime = finalize_batch_row<L>(p, seq, b, lane, rs);   // the same for every row of a launch
+    const int regime = finalize_batch_row<L>(p, seq, b, lane, rs, bs);   // the same for every row of a launch
     bool last = false;
     if (lane == 0) sc.b_ticket[b] = 0u;               // ready for this copy's next launch
-    fence_acq_rel();                                  // each lane's outputs and hints of this row ...
-    __syncwarp();                                     // ... all of them before the row's ticket
-    if (lane == 0) last = atomicAdd(sc.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;
+    __syncwarp();                                     // each lane's outputs and hints of this row before the row's ticket,
+    if (lane == 0) last = atom_add_acq_rel(sc.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;   // whose add releases them
     last = __shfl_sync(kFull, last, 0);
     if (!last) return;
 
-    // ---- every batch row is final: S6 ----
-    fence_acq_rel();
+    // ---- every batch row is final (lane 0 has acquired what their warps released): S6 ----
+    __syncwarp();
     OcmStatsDev *st = p.ocm.stats;
     // new keys are claimed by the look-ups (above) except near the key limit, where the
     // update itself inserts: only then does the key count have to be read afterwards
@@ -778,77 +794,49 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
     const int cpr = (U + CH - 1) / CH;                       // chunks of a whole row
     long long g = span_begin(p, blockIdx.x);
     const long long g_end = span_begin(p, blockIdx.x + 1);
+    // quotients of unit and row indices: 32-bit division where the host found that everything fits
+    auto quot = [&](long long a, int b) -> long long {
+        return p.narrow ? static_cast<long long>(static_cast<unsigned int>(a) / static_cast<unsigned int>(b)) : a / b;
+    };
 
     bool first_window = true;
     while (g < g_end) {
         // ---- a window: up to kMaxSegs consecutive row parts of this block's span ----
-        const long long row0 = g / U;
+        const long long row0 = quot(g, U);
         const int o0 = static_cast<int>(g - row0 * U);
         long long w_end = (row0 + kMaxSegs) * U;
         if (w_end > g_end) w_end = g_end;
-        const int nseg = static_cast<int>((w_end - row0 * U + U - 1) / U);
+        const int nseg = static_cast<int>(quot(w_end - row0 * U + U - 1, U));
         const long long first_len = w_end - row0 * U;        // units from row0's start to the window end
         const int b0 = first_len < U ? static_cast<int>(first_len) : U;
         const int n0 = (b0 - o0 + CH - 1) / CH;               // chunks of the first row part
         const int last_units = static_cast<int>(w_end - (row0 + nseg - 1) * U);
         const int n_last = (last_units + CH - 1) / CH;
         const int nchunks = nseg == 1 ? n0 : n0 + (nseg - 2) * cpr + n_last;
-
+        const int next_b = w_end < g_end ? static_cast<int>(quot(quot(w_end, U), K1)) : -1;
         // the first window's fold count has one extra party: the sequence number's arrival
         const unsigned int fold_target = static_cast<unsigned int>(nseg) + (first_window ? 1u : 0u);
-        if (threadIdx.x == 0) {
-            bs.next_chunk = 0u;
-            bs.segs_folded = 0u;
-            bs.n_todo = 0;
-        }
-        if (threadIdx.x < kMaxSegs) bs.seg_done[threadIdx.x] = 0u;   // kMaxSegs <= 32: warp 0 only
-        if (!first_window || nwarps == 1) {
-            __syncthreads();
-        } else if (seq_warp) {
-            named_barrier_sync(2, 64);                  // tables are set up (warp 0 arrived)
-        } else {
-            if (warp == 0) named_barrier_arrive(2, 64);
-            named_barrier_sync(1, 32 * (nwarps - 1));   // the streaming warps start without the last warp
-        }
-        if (first_window && seq_warp) {
-            if (lane == 0)
-                bs.seq = (seq_old >> 32) == 0ull ? static_cast<unsigned int>(seq_old) / gridDim.x
-                                                 : static_cast<unsigned int>(seq_old / gridDim.x);
-            __syncwarp();
-            pdl_launch_dependents();
-            bool block_complete = false;
-            if (lane == 0) {
-                __threadfence_block();
-                block_complete = atomicAdd(&bs.segs_folded, 1u) == fold_target - 1u;
-            }
-            if (__shfl_sync(kFull, block_complete, 0)) {   // everything else was already folded
-                __threadfence_block();
-                const int next_b = w_end < g_end ? static_cast<int>((w_end / U) / K1) : -1;
-                publish_parts(p, bs, static_cast<int>(row0), nseg, next_b, lane);
-            }
-        }
-        first_window = false;
 
-        while (true) {
-            unsigned int q = 0;
-            if (lane == 0) q = atomicAdd(&bs.next_chunk, 1u);
-            q = __shfl_sync(kFull, q, 0);
-            if (q >= static_cast<unsigned int>(nchunks)) break;
-
-            // ---- S1: which row part and which chunk of it ----
-            int seg, k, seg_first, seg_n, ua, ub;
+        // ---- S1 for chunk q of the window: which row part, which run of it, and its reduction ----
+        struct ChunkAt {
+            int seg, seg_first, seg_n;
+            bool ok;
+        };
+        auto reduce_chunk = [&](unsigned int q, Partial &r) -> ChunkAt {
+            ChunkAt at;
+            int k, ua, ub;
             if (static_cast<int>(q) < n0) {
-                seg = 0; k = q; seg_first = 0; seg_n = n0; ua = o0; ub = b0;
+                at.seg = 0; k = q; at.seg_first = 0; at.seg_n = n0; ua = o0; ub = b0;
             } else {
-                const int r = static_cast<int>(q) - n0;
-                seg = 1 + r / cpr;
-                k = r - (seg - 1) * cpr;
-                seg_first = n0 + (seg - 1) * cpr;
+                const int rr = static_cast<int>(q) - n0;
+                at.seg = 1 + rr / cpr;
+                k = rr - (at.seg - 1) * cpr;
+                at.seg_first = n0 + (at.seg - 1) * cpr;
                 ua = 0;
-                if (seg == nseg - 1) { seg_n = n_last; ub = last_units; } else { seg_n = cpr; ub = U; }
+                if (at.seg == nseg - 1) { at.seg_n = n_last; ub = last_units; } else { at.seg_n = cpr; ub = U; }
             }
-            const long long row = row0 + seg;
-            const long long b = row / K1;
+            const long long row = row0 + at.seg;
+            const long long b = quot(row, K1);
             const int i = static_cast<int>(row - b * K1);
             const E *rp = reinterpret_cast<const E *>(p.logits) + b * p.stride_b + i * p.stride_k;
             const int u0 = ua + k * CH;
@@ -856,44 +844,128 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             const int e0 = u0 * p.unit_elems;
             const long long e1l = static_cast<long long>(u1) * p.unit_elems;
             const int e1 = e1l < p.V ? static_cast<int>(e1l) : p.V;
-            if (!CSD_INDEX_OK(row < static_cast<long long>(p.B) * K1 && seg >= 0 && seg < nseg && nseg <= kMaxSegs &&
-                                  q < static_cast<unsigned int>(kMaxChunks) && e0 >= 0 && e0 < e1 && seg_first + seg_n <= kMaxChunks,
-                              p.ocm.stats, 5u))
-                continue;
-            const Partial r = warp_tile<L>(rp, e0, e1, lane);
-
-            // ---- deliver it; the warp bringing a row part's last chunk folds that part ----
+            at.ok = CSD_INDEX_OK(row < static_cast<long long>(p.B) * K1 && at.seg >= 0 && at.seg < nseg && nseg <= kMaxSegs &&
+                                     q < static_cast<unsigned int>(kMaxChunks) && e0 >= 0 && e0 < e1 &&
+                                     at.seg_first + at.seg_n <= kMaxChunks,
+                                 p.ocm.stats, 5u);
+            if (at.ok) r = warp_tile<L>(rp, e0, e1, lane);
+            return at;
+        };
+        // ---- deliver a chunk's result; the warp bringing a row part's last chunk folds that part, the warp
+        // completing the block's last fold publishes ----
+        auto deliver = [&](unsigned int q, const ChunkAt &at, const Partial &r) {
             bool seg_complete = false;
             if (lane == 0) {
                 bs.chunk_part[q] = r;
                 __threadfence_block();
-                seg_complete = atomicAdd(&bs.seg_done[seg], 1u) == static_cast<unsigned int>(seg_n) - 1u;
+                seg_complete = atomicAdd(&bs.seg_done[at.seg], 1u) == static_cast<unsigned int>(at.seg_n) - 1u;
             }
-            if (!__shfl_sync(kFull, seg_complete, 0)) continue;
+            if (!__shfl_sync(kFull, seg_complete, 0)) return;
             __threadfence_block();
             Partial v = partial_identity();
-            for (int j = lane; j < seg_n; j += 32) {
-                const Partial x = bs.chunk_part[seg_first + j];
+            for (int j = lane; j < at.seg_n; j += 32) {
+                const Partial x = bs.chunk_part[at.seg_first + j];
                 v = (j == lane) ? x : combine(v, x);
             }
             v = butterfly_fold(v, 32);
             bool block_complete = false;
             if (lane == 0) {
-                bs.seg_result[seg] = v;
+                bs.seg_result[at.seg] = v;
                 __threadfence_block();
                 block_complete = atomicAdd(&bs.segs_folded, 1u) == fold_target - 1u;
             }
-            if (!__shfl_sync(kFull, block_complete, 0)) continue;
+            if (!__shfl_sync(kFull, block_complete, 0)) return;
             __threadfence_block();
-            const int next_b = w_end < g_end ? static_cast<int>((w_end / U) / K1) : -1;
             publish_parts(p, bs, static_cast<int>(row0), nseg, next_b, lane);
+        };
+
+        // The shared tables of the window.  In the block's first window nothing waits for them yet: every warp
+        // first takes chunk number `warp` without asking and reduces it, so that its loads are in flight a few
+        // hundred cycles after the block started; the tables are needed only to deliver the result.
+        if (threadIdx.x == 0) {
+            bs.next_chunk = first_window ? static_cast<unsigned int>(nwarps) : 0u;
+            bs.segs_folded = 0u;
+            bs.n_todo = 0;
+            if (!first_window) {
+                bs.pre_b[0] = -1;
+                bs.pre_b[1] = -1;
+            }
         }
+        if (threadIdx.x < kMaxSegs) bs.seg_done[threadIdx.x] = 0u;   // kMaxSegs <= 32: warp 0 only
+        if (!first_window) __syncthreads();
+        if (first_window && seq_warp) {
+            // The launch's sequence number has arrived: from here on the next launch on the stream may begin.
+            // This comes before the warp's own first chunk, because every block of a launch must get here
+            // before the next launch can start at all.
+            // While the sequence number travels, the same warp fetches the draft tokens of the first two batch
+            // rows the block touches (a block that later finalises one of them finds them in shared memory).
+            const int fb = static_cast<int>(quot(row0, K1));
+            const bool two = quot(row0 + nseg - 1, K1) > fb;
+            int d0 = -1, d1 = -1;
+            if (lane < p.K) {
+                d0 = __ldg(p.draft + (size_t)fb * p.K + lane);
+                if (two) d1 = __ldg(p.draft + (size_t)(fb + 1) * p.K + lane);
+            }
+            if (lane == 0)
+                bs.seq = (seq_old >> 32) == 0ull ? static_cast<unsigned int>(seq_old) / gridDim.x
+                                                 : static_cast<unsigned int>(seq_old / gridDim.x);
+            __syncwarp();
+            pdl_launch_dependents();
+            if (lane < p.K) {
+                bs.pre_d[0][lane] = d0;
+                bs.pre_d[1][lane] = d1;
+                if (static_cast<unsigned int>(d0) < static_cast<unsigned int>(p.V)) prefetch_l2(logit_row<L>(p, fb, lane) + d0);
+                if (static_cast<unsigned int>(d1) < static_cast<unsigned int>(p.V)) prefetch_l2(logit_row<L>(p, fb + 1, lane) + d1);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                bs.pre_b[0] = fb;
+                bs.pre_b[1] = two ? fb + 1 : -1;
+            }
+        }
+
+        for (bool static_pick = first_window;; static_pick = false) {
+            unsigned int q = static_cast<unsigned int>(warp);
+            if (!static_pick) {
+                if (lane == 0) q = atomicAdd(&bs.next_chunk, 1u);
+                q = __shfl_sync(kFull, q, 0);
+                if (q >= static_cast<unsigned int>(nchunks)) break;
+            }
+            Partial r;
+            ChunkAt at;
+            at.ok = false;
+            if (q < static_cast<unsigned int>(nchunks)) at = reduce_chunk(q, r);
+            if (static_pick) {
+                // ---- once per block: the tables are set up; the sequence number counts as one more fold ----
+                if (nwarps == 1) {
+                    __syncthreads();
+                } else if (seq_warp) {
+                    named_barrier_sync(2, 64);                  // tables are set up (warp 0 arrived)
+                } else {
+                    if (warp == 0) named_barrier_arrive(2, 64);
+                    named_barrier_sync(1, 32 * (nwarps - 1));   // the other warps go on without the last warp
+                }
+                if (seq_warp) {
+                    bool block_complete = false;
+                    if (lane == 0) {
+                        __threadfence_block();
+                        block_complete = atomicAdd(&bs.segs_folded, 1u) == fold_target - 1u;
+                    }
+                    if (__shfl_sync(kFull, block_complete, 0)) {   // everything else was already folded
+                        __threadfence_block();
+                        publish_parts(p, bs, static_cast<int>(row0), nseg, next_b, lane);
+                    }
+                }
+            }
+            if (at.ok) deliver(q, at, r);
+        }
+        first_window = false;
         // ---- the batch rows this block completed are shared out over its warps: S2..S6 ----
         __syncthreads();
         const int fin_warps = nwarps < kFinalizeWarps ? nwarps : kFinalizeWarps;
         if (warp < fin_warps && CSD_INDEX_OK(bs.n_todo >= 0 && bs.n_todo <= kMaxSegs, p.ocm.stats, 6u))
             for (int j = warp; j < bs.n_todo; j += fin_warps)
-                finalize_and_update<L>(p, bs.seq, bs.todo_b[j], lane, row_scratch[warp], canon);
+                finalize_and_update<L>(p, bs.seq, bs.todo_b[j], lane, row_scratch[warp], canon, bs);
         g = w_end;
         if (g < g_end) __syncthreads();       // the next window reuses the shared-memory tables
     }

@@ -36,25 +36,25 @@ def _run(name, tau, steps, checkpoint, overlap, prewarm_steps=0):
 @pytest.mark.parametrize("overlap", [False, True], ids=["alone", "overlap"])
 @pytest.mark.parametrize("tau", [0.2, 0.4])
 def test_large_batch(tau, overlap):
-    out = _run("large_batch", tau, 60, 20, overlap)              # 200 000-pair pre-warm inside; 61 440 positions
+    out = _run("large_batch", tau, 150, 50, overlap)             # 200 000-pair pre-warm inside; 153 600 positions
     assert out["n_keys"] > 5000
 
 
 @pytest.mark.parametrize("overlap", [False, True], ids=["alone", "overlap"])
 def test_batched_serving(overlap):
-    _run("batched_serving", 0.3, 700, 100, overlap)              # 112 000 positions
+    _run("batched_serving", 0.3, 2000, 250, overlap)             # 320 000 positions
 
 
 @pytest.mark.parametrize("overlap", [False, True], ids=["alone", "overlap"])
 def test_ocm_contention(overlap):
-    out = _run("ocm_contention", 0.3, 600, 100, overlap)         # 230 400 positions, memory compared every 100 steps
-    assert out["checkpoints"] == 6
+    out = _run("ocm_contention", 0.3, 1500, 100, overlap)        # 576 000 positions, memory compared every 100 steps
+    assert out["checkpoints"] == 15
 
 
 @pytest.mark.parametrize("overlap", [False, True], ids=["alone", "overlap"])
 @pytest.mark.parametrize("tau", [0.1, 0.3, 0.5])
 def test_single_stream(tau, overlap):
-    _run("single_stream", tau, 1500, 500, overlap, prewarm_steps=500)
+    _run("single_stream", tau, 3000, 500, overlap, prewarm_steps=500)
 
 
 def _oracle_sampled_by_rows(z, y, d, r, seed, T, mem, tau, rows_at_a_time=16):
