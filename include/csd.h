@@ -324,6 +324,41 @@ csd_status_t csd_step_sampled(const void *logits, const void *draft_logits, csd_
                               const csd_sampled_diag_t *diag,
                               void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- the step taken straight from the LM head: logits never stored -------------------------------
+ *
+ * Algorithm 1 gets the distributions of all gamma + 1 positions from ONE parallel target pass, and the paper's
+ * starting point is that this pass is bound by memory traffic (Introduction).  Its last operation is the LM
+ * head, z[b, i, v] = sum_h hidden[b, i, h] * weight[v, h]; these entry points take the inputs of that operation
+ * instead of its result.  A tensor-core GEMM produces the logits tile by tile and reduces each tile at once to
+ * the row statistics of csd_verify (max, lowest arg-max, sum of exponentials) and the draft tokens' logits, so
+ * the [B, K+1, V] logit tensor is neither written nor read; everything after that is csd_verify / csd_step.
+ *
+ * hidden : [B, K+1, H] bf16, dense, 16-byte aligned.   weight : [V, H] bf16, dense, 16-byte aligned.
+ * Shapes: H a multiple of 64; B*(K+1) <= 256 (larger batches: split the batch); any V.
+ * The logits are the fp32 tensor-core accumulations of the exact bf16 products, NOT rounded to bf16: they
+ * differ from an exactly summed product by at most about 2^-16 * ||hidden row|| * max ||weight row|| (see
+ * the tests), so an arg-max or a gate decision that hangs on a smaller difference may come out either way;
+ * everything else is the result csd_verify would give on the exact logits.  diag as for csd_verify.
+ * workspace: csd_lmhead_workspace_bytes bytes, 16-byte aligned, no initialisation needed.
+ * Three launches (GEMM + statistics, decisions, memory update); asynchronous.  A wait inside the GEMM
+ * kernel that does not end within about two seconds raises CSD_FLAG_INTERNAL (debug_site 30).
+ * Errors as csd_verify; UNSUPPORTED for shapes outside the limits above; CUDA if the driver offers no
+ * tensor-map encoder. */
+size_t csd_lmhead_workspace_bytes(int B, int K, int H, int V);
+csd_status_t csd_verify_lmhead(const void *hidden, const void *weight, int B, int K, int H, int V,
+                               const int32_t *draft, const csd_ocm_t *ocm, float tau,
+                               int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                               int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
+                               void *workspace, size_t workspace_bytes, void *stream);
+csd_status_t csd_step_lmhead(const void *hidden, const void *weight, int B, int K, int H, int V,
+                             const int32_t *draft, csd_ocm_t *ocm, float tau,
+                             int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                             int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
+                             void *workspace, size_t workspace_bytes, void *stream);
+/* How the vocabulary is cut for this shape: blocks of the GEMM grid, columns per tile, number of tiles and
+ * tiles per block.  Host function; for reports and tests. */
+csd_status_t csd_lmhead_shape(int B, int K, int H, int V, int *grid, int *tile_cols, int *tiles, int *tiles_per_block);
+
 /* csd_step for callers whose tensors live in HOST memory (pinned memory gives
  * the full copy rate).  Copies logits and draft to `staging`, runs the step, and
  * copies accept_len, next_token and rescued_mask back; returns after the stream

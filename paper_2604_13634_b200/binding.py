@@ -29,6 +29,7 @@ EXPORTS = [
     "csd_scg_threshold", "csd_launch_shape", "csd_set_tuning", "csd_set_overlap", "csd_status_string",
     "csd_sampled_workspace_bytes", "csd_verify_sampled", "csd_step_sampled",
     "csd_ocm_age", "csd_ocm_merge", "csd_ocm_save", "csd_ocm_load", "csd_ocm_set_shared",
+    "csd_lmhead_workspace_bytes", "csd_verify_lmhead", "csd_step_lmhead", "csd_lmhead_shape",
 ]
 
 
@@ -71,6 +72,8 @@ def lib():
     sampled_args = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_int64, c_int64, c_int64, c_int64, c_void_p, c_void_p,
                     c_uint64, c_float, c_void_p, c_float, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
                     POINTER(SampledDiag), c_void_p, c_size_t, c_void_p]
+    lmhead_args = [c_void_p, c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_float, c_void_p, c_void_p, c_void_p,
+                   c_void_p, c_void_p, POINTER(Diag), c_void_p, c_size_t, c_void_p]
     sigs = {
         "csd_sampled_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int]),
         "csd_verify_sampled": (c_int, sampled_args),
@@ -91,6 +94,10 @@ def lib():
         "csd_ocm_export": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_uint64, POINTER(c_uint64), c_void_p]),
         "csd_ocm_import": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_uint64, c_void_p]),
         "csd_ocm_stats": (c_int, [c_void_p, POINTER(Stats), c_void_p]),
+        "csd_lmhead_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int]),
+        "csd_verify_lmhead": (c_int, lmhead_args),
+        "csd_step_lmhead": (c_int, lmhead_args),
+        "csd_lmhead_shape": (c_int, [c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
         "csd_ocm_age": (c_int, [c_void_p, c_void_p]),
         "csd_ocm_set_shared": (c_int, [c_void_p, c_int]),
         "csd_ocm_merge": (c_int, [c_void_p, c_void_p, c_void_p]),
@@ -408,3 +415,45 @@ def csd_step_sampled(logits, draft_logits, draft, r_accept, seed: int, temperatu
 def sampled_launches_per_step() -> int:
     """Kernel launches one csd_step_sampled call makes (for launch counts in reports)."""
     return 7
+
+
+class LmheadBuffers(StepBuffers):
+    """Outputs, optional diagnostics and workspace of the step that starts from the LM head's inputs."""
+
+    def __init__(self, B: int, K: int, H: int, V: int, device="cuda", diag: bool = False):
+        self.H = H
+        bytes_ = int(lib().csd_lmhead_workspace_bytes(B, K, H, V))
+        if bytes_ == 0:
+            raise CsdError(f"unsupported shape B={B} K={K} H={H} V={V} (H % 64 == 0 and B*(K+1) <= 256 are required)")
+        super().__init__(B, K, V, torch.bfloat16, device=device, diag=diag)
+        self.ws_bytes = bytes_
+        self.workspace = torch.empty(bytes_, dtype=torch.uint8, device=torch.device(device))
+
+
+def csd_lmhead_shape(B, K, H, V):
+    g, n, t, per = c_int(), c_int(), c_int(), c_int()
+    _check(lib().csd_lmhead_shape(B, K, H, V, byref(g), byref(n), byref(t), byref(per)), "csd_lmhead_shape")
+    return dict(grid=g.value, tile_cols=n.value, tiles=t.value, tiles_per_block=per.value)
+
+
+def _lmhead_call(fn_name, hidden, weight, draft, ocm: Ocm, tau, buf: LmheadBuffers, stream):
+    assert hidden.is_cuda and weight.is_cuda and draft.is_cuda and draft.dtype == torch.int32 and draft.is_contiguous()
+    assert hidden.dtype == torch.bfloat16 and weight.dtype == torch.bfloat16 and hidden.is_contiguous() and weight.is_contiguous()
+    B, K1, H = hidden.shape
+    V, H2 = weight.shape
+    assert (B, K1 - 1, H, V) == (buf.B, buf.K, buf.H, buf.V) and H2 == H and tuple(draft.shape) == (B, K1 - 1)
+    rc = getattr(lib(), fn_name)(hidden.data_ptr(), weight.data_ptr(), B, K1 - 1, H, V, draft.data_ptr(), ocm.handle, c_float(tau),
+                                 _ptr(buf.accept_len), _ptr(buf.next_token), _ptr(buf.rescued_mask), _ptr(buf.rej_draft),
+                                 _ptr(buf.rej_target), byref(buf._diag_struct) if buf._diag_struct is not None else None,
+                                 _ptr(buf.workspace), buf.ws_bytes, _stream_ptr(stream))
+    _check(rc, fn_name)
+
+
+def csd_verify_lmhead(hidden, weight, draft, ocm: Ocm, tau: float, buf: LmheadBuffers, stream=None):
+    """csd_verify on the logits hidden @ weight^T, which are never stored; the memory is only read."""
+    _lmhead_call("csd_verify_lmhead", hidden, weight, draft, ocm, tau, buf, stream)
+
+
+def csd_step_lmhead(hidden, weight, draft, ocm: Ocm, tau: float, buf: LmheadBuffers, stream=None):
+    """csd_step on the logits hidden @ weight^T, which are never stored."""
+    _lmhead_call("csd_step_lmhead", hidden, weight, draft, ocm, tau, buf, stream)

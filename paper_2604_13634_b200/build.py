@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcsd.so")
 LIB_DEBUG = os.path.join(HERE, "libcsd_debug.so")     # the same sources with -DCSD_DEBUG: every index checked
 SOURCES = ["csd_api.cu"]
-HEADERS = ["csd_common.cuh", "csd_ocm.cuh", "csd_step.cuh", "csd_sampled.cuh", os.path.join("..", "..", "include", "csd.h")]
+HEADERS = ["csd_common.cuh", "csd_ocm.cuh", "csd_step.cuh", "csd_sampled.cuh", "csd_lmhead.cuh", os.path.join("..", "..", "include", "csd.h")]
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-shared", "-Xcompiler", "-fPIC", "--use_fast_math=false"]

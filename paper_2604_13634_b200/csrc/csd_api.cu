@@ -13,6 +13,7 @@
 #include "csd_ocm.cuh"
 #include "csd_step.cuh"
 #include "csd_sampled.cuh"
+#include "csd_lmhead.cuh"
 
 using namespace csd;
 
@@ -30,6 +31,7 @@ struct csd_ocm {
 namespace {
 
 constexpr int kDefaultSms = 148;   // B200; used only when no device can be queried
+constexpr int kMaxLmheadDevices = 64;
 
 int g_chunk_bytes_override = 0;
 int g_ctas_per_sm_override = 0;
@@ -770,6 +772,189 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
     return run_step(logits, dtype, B, K, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
                     rej_draft, rej_target, diag, scratch, need, stream, false, /*may_chain=*/false,
                     /*may_overlap=*/false, /*track_layout=*/false);   // cleared just above, whatever it held
+}
+
+// ---- the step taken straight from the LM head --------------------------------------------------
+namespace {
+
+struct LmheadPlan {
+    int grid, n_tile, tiles_total, tiles_per_cta;
+    size_t partials_off, zd_off, total;
+};
+
+bool lmhead_shape_ok(int B, int K, int H, int V)
+{
+    if (!(B > 0 && K > 0 && K <= CSD_MAX_K && V > 0 && H > 0)) return false;
+    if (H % lmhead::kBlockK != 0) return false;
+    return static_cast<long long>(B) * (K + 1) <= lmhead::kRowsMax;
+}
+
+// The vocabulary is cut into tiles of n_tile columns (a multiple of 16, at most 256) such that every CTA of a
+// one-per-SM grid owns the same number of consecutive tiles.
+LmheadPlan lmhead_plan(int B, int K, int V)
+{
+    LmheadPlan pl;
+    const long long sms = sm_count();
+    long long per = (V + sms * lmhead::kNMax - 1) / (sms * lmhead::kNMax);          // tiles per CTA
+    if (per < 1) per = 1;
+    long long width = (V + sms * per - 1) / (sms * per);
+    width = (width + 15) / 16 * 16;
+    if (width > lmhead::kNMax) width = lmhead::kNMax;
+    if (width < 16) width = 16;
+    pl.n_tile = static_cast<int>(width);
+    pl.tiles_total = static_cast<int>((V + width - 1) / width);
+    pl.tiles_per_cta = static_cast<int>(per);
+    long long grid = (pl.tiles_total + per - 1) / per;
+    pl.grid = static_cast<int>(grid < 1 ? 1 : grid);
+    const size_t rows = static_cast<size_t>(B) * (K + 1);
+    pl.partials_off = 0;
+    pl.zd_off = align_up(rows * pl.grid * sizeof(Partial), 256);
+    pl.total = align_up(pl.zd_off + static_cast<size_t>(B) * K * sizeof(float), 256);
+    return pl;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static std::mutex m;
+    static EncodeTiledFn fn = nullptr;
+    std::lock_guard<std::mutex> lock(m);
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// A [rows, cols] row-major bf16 matrix as a tensor map whose box is box_rows x 64 columns, 128-byte swizzle;
+// elements outside the matrix read as zero.
+bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(lmhead::kBlockK), box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, int H, int V, const int32_t *draft, csd_ocm *ocm,
+                        float tau, int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask, int32_t *rej_draft,
+                        int32_t *rej_target, const csd_diag_t *diag, void *workspace, size_t workspace_bytes, void *stream,
+                        bool do_update)
+{
+    if (!hidden || !weight || !draft || !ocm || !accept_len || !next_token || !rescued_mask || !rej_draft || !rej_target || !workspace)
+        return CSD_ERR_INVALID_ARG;
+    if (B <= 0 || K <= 0 || H <= 0 || V <= 0) return CSD_ERR_INVALID_ARG;
+    if (!(tau >= 0.0f) || std::isinf(tau)) return CSD_ERR_INVALID_ARG;
+    if (!lmhead_shape_ok(B, K, H, V)) return CSD_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(weight) & 15u)) return CSD_ERR_INVALID_ARG;
+    const LmheadPlan pl = lmhead_plan(B, K, V);
+    if (workspace_bytes < pl.total || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
+    chain_break();
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int R = B * (K + 1);
+
+    static std::mutex attr_mutex;
+    static bool attr_set[kMaxLmheadDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxLmheadDevices) {
+        (void)cudaGetLastError();
+        return CSD_ERR_CUDA;
+    }
+    {
+        std::lock_guard<std::mutex> lock(attr_mutex);
+        if (!attr_set[dev]) {
+            if (cudaFuncSetAttribute(lmhead::lmhead_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lmhead::kSmemBytes) !=
+                cudaSuccess) {
+                (void)cudaGetLastError();
+                return CSD_ERR_CUDA;
+            }
+            attr_set[dev] = true;
+        }
+    }
+    CUtensorMap map_h, map_w;
+    if (!make_map(&map_h, hidden, static_cast<uint64_t>(R), static_cast<uint64_t>(H), lmhead::kMTile) ||
+        !make_map(&map_w, weight, static_cast<uint64_t>(V), static_cast<uint64_t>(H), static_cast<uint32_t>(pl.n_tile)))
+        return CSD_ERR_CUDA;
+
+    char *ws = static_cast<char *>(workspace);
+    lmhead::Params p;
+    std::memset(&p, 0, sizeof p);
+    p.R = R; p.H = H; p.V = V; p.B = B; p.K = K;
+    p.n_tile = pl.n_tile;
+    p.tiles_total = pl.tiles_total;
+    p.tiles_per_cta = pl.tiles_per_cta;
+    p.draft = draft;
+    p.partials = reinterpret_cast<Partial *>(ws + pl.partials_off);
+    p.zd = reinterpret_cast<float *>(ws + pl.zd_off);
+    p.stats = ocm->stats;
+    lmhead::lmhead_stats_kernel<<<pl.grid, lmhead::kThreads, lmhead::kSmemBytes, st>>>(map_h, map_w, p);
+    if (cudaGetLastError() != cudaSuccess) return CSD_ERR_CUDA;
+
+    lmhead::FinalizeParams f;
+    std::memset(&f, 0, sizeof f);
+    f.B = B; f.K = K; f.V = V; f.n_parts = pl.grid;
+    f.partials = p.partials;
+    f.zd = p.zd;
+    f.draft = draft;
+    f.ocm = view_of(ocm);
+    f.log_tau = csd_scg_threshold(tau);
+    f.accept_len = accept_len; f.next_token = next_token; f.rescued = rescued_mask;
+    f.rej_d = rej_draft; f.rej_t = rej_target;
+    if (diag) f.diag = *diag;
+    lmhead::lmhead_finalize_kernel<<<(B + 3) / 4, 128, 0, st>>>(f);
+    if (cudaGetLastError() != cudaSuccess) return CSD_ERR_CUDA;
+    if (do_update) return run_update(ocm, rej_draft, rej_target, nullptr, static_cast<int64_t>(B) * K, stream);
+    return CSD_OK;
+}
+
+}  // namespace
+
+size_t csd_lmhead_workspace_bytes(int B, int K, int H, int V)
+{
+    if (!lmhead_shape_ok(B, K, H, V)) return 0;
+    return lmhead_plan(B, K, V).total;
+}
+
+csd_status_t csd_verify_lmhead(const void *hidden, const void *weight, int B, int K, int H, int V, const int32_t *draft,
+                               const csd_ocm_t *ocm, float tau, int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                               int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag, void *workspace,
+                               size_t workspace_bytes, void *stream)
+{
+    return run_lmhead(hidden, weight, B, K, H, V, draft, const_cast<csd_ocm_t *>(ocm), tau, accept_len, next_token, rescued_mask,
+                      rej_draft, rej_target, diag, workspace, workspace_bytes, stream, false);
+}
+
+csd_status_t csd_step_lmhead(const void *hidden, const void *weight, int B, int K, int H, int V, const int32_t *draft, csd_ocm_t *ocm,
+                             float tau, int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask, int32_t *rej_draft,
+                             int32_t *rej_target, const csd_diag_t *diag, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return run_lmhead(hidden, weight, B, K, H, V, draft, ocm, tau, accept_len, next_token, rescued_mask, rej_draft, rej_target,
+                      diag, workspace, workspace_bytes, stream, true);
+}
+
+csd_status_t csd_lmhead_shape(int B, int K, int H, int V, int *grid, int *tile_cols, int *tiles, int *tiles_per_block)
+{
+    if (!lmhead_shape_ok(B, K, H, V)) return CSD_ERR_UNSUPPORTED;
+    const LmheadPlan pl = lmhead_plan(B, K, V);
+    if (grid) *grid = pl.grid;
+    if (tile_cols) *tile_cols = pl.n_tile;
+    if (tiles) *tiles = pl.tiles_total;
+    if (tiles_per_block) *tiles_per_block = pl.tiles_per_cta;
+    return CSD_OK;
 }
 
 size_t csd_sampled_workspace_bytes(int B, int K, int V, csd_dtype_t dtype)

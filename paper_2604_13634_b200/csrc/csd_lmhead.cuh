@@ -1,0 +1,514 @@
+// The verification step taken straight from the LM head: the logits z[r, v] = sum_h hidden[r, h] * W[v, h] of
+// Algorithm 1's single target pass are produced by a tcgen05 GEMM whose epilogue reduces them to the per-row
+// statistics of S1 (maximum, lowest arg-max, sum of exponentials) and picks out the draft tokens' logits, so
+// the [rows, V] logit tensor never reaches HBM.
+//
+//   lmhead_stats_kernel     persistent, one CTA per SM, 192 threads:
+//       warp 0      one thread issues the TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of the k-blocks:
+//                   64 columns of all hidden rows (two boxes of 128 rows; rows beyond R read as zero) and of
+//                   the vocabulary tile's W rows, into a ring of shared-memory stages
+//       warp 1      one thread issues the MMAs (tcgen05.mma, kind::f16, M = 128, N = tile width, K = 16, fp32
+//                   accumulators in tensor memory: columns [0, N) for rows 0..127, [256, 256 + N) for rows
+//                   128..255) and commits each stage back to the loader, each finished tile to the epilogue
+//       warps 2..5  epilogue: thread i of the warp covering TMEM lanes 32q..32q+31 owns logit rows 32q + i and
+//                   128 + 32q + i; it reads its rows' accumulators 32 columns at a time (tcgen05.ld) and folds
+//                   them into a running (max, arg-max, reference exponent, sum) -- no exchange between threads,
+//                   a row lives in one thread -- and keeps z[row, draft[row]] when that column comes by
+//     A CTA owns a contiguous run of vocabulary tiles and ends with one partial per logit row.
+//   lmhead_finalize_kernel  one warp per batch row: folds the CTAs' partials in a fixed order, then S2..S5
+//                           exactly as the streaming step does; the memory update follows as its own launch.
+//
+// Every wait on an mbarrier is bounded (about two seconds of clock cycles): when one runs out, the CTA raises
+// CSD_FLAG_INTERNAL (debug_site 30), all its roles leave their loops, it waits for copies that may still be in
+// flight, frees its tensor memory and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "../../include/csd.h"
+#include "csd_common.cuh"
+#include "csd_ocm.cuh"
+
+namespace csd {
+namespace lmhead {
+
+constexpr int kBlockK = 64;                 // bf16 elements of a k-block: one 128-byte swizzle row
+constexpr int kStages = 3;
+constexpr int kMTile = 128;
+constexpr int kRowsMax = 2 * kMTile;        // logit rows a step may have
+constexpr int kNMax = 256;                  // widest vocabulary tile
+constexpr int kThreads = 192;
+constexpr int kStageABytes = kRowsMax * kBlockK * 2;
+constexpr int kStageBBytes = kNMax * kBlockK * 2;
+constexpr int kStageBytes = kStageABytes + kStageBBytes;
+constexpr int kBarrierBytes = 256;
+constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;     // + room to align the stages to 1 KiB
+constexpr int kTmemCols = 512;
+constexpr long long kWaitCycles = 4000000000ll;
+
+struct Params {
+    int R, H, V, B, K;
+    int n_tile;             // columns of a vocabulary tile: multiple of 16, at most kNMax
+    int tiles_total;        // ceil(V / n_tile)
+    int tiles_per_cta;
+    const int *draft;       // [B, K]
+    Partial *partials;      // [R, gridDim.x]
+    float *zd;              // [B, K]  z[b, i, draft[b, i]] (written for valid draft ids only)
+    OcmStatsDev *stats;
+};
+
+__device__ __forceinline__ unsigned int smem_u32(const void *p) { return static_cast<unsigned int>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(unsigned int bar, unsigned int count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned int bar, unsigned int bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned int bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned int bar, unsigned int parity)
+{
+    unsigned int ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok)
+                 : "r"(bar), "r"(parity)
+                 : "memory");
+    return ok != 0u;
+}
+// Bounded wait.  False if the wait ran out or another role of the CTA has given up.
+__device__ __forceinline__ bool mbar_wait(unsigned int bar, unsigned int parity, volatile int *give_up)
+{
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*give_up) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *give_up = 1;
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(unsigned int dst, const CUtensorMap *map, unsigned int bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+                 "l"(map), "r"(bar), "r"(x), "r"(y)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(unsigned int smem_dst, unsigned int cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(unsigned int taddr, unsigned int cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(unsigned int bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 operands, fp32 accumulators.
+__device__ __forceinline__ void tc_mma_bf16(unsigned int d_tmem, unsigned long long a_desc, unsigned long long b_desc, unsigned int idesc,
+                                            unsigned int accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+                 "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+                 : "memory");
+}
+// 32 consecutive accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(unsigned int taddr, float (&x)[32])
+{
+    unsigned int r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(r[j]);
+}
+
+// Shared-memory operand descriptor of a K-major bf16 tile stored as rows of 128 bytes with the 128-byte swizzle
+// (what the TMA loads above produce): groups of 8 rows lie 1024 bytes apart, the tile starts on a 1 KiB boundary.
+__device__ __forceinline__ unsigned long long operand_desc(unsigned int smem_addr)
+{
+    unsigned long long d = 0;
+    d |= static_cast<unsigned long long>((smem_addr & 0x3FFFFu) >> 4);     // start address
+    d |= 1ull << 16;                                                       // leading-dimension offset: unused for this layout
+    d |= static_cast<unsigned long long>(1024 >> 4) << 32;                 // stride between 8-row groups
+    d |= 1ull << 46;                                                       // descriptor version of this architecture
+    d |= 2ull << 61;                                                       // 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ unsigned int instr_desc(int n)
+{
+    // fp32 accumulators, bf16 A and B, both K-major, N = n, M = 128
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<unsigned int>(n >> 3) << 17) | (static_cast<unsigned int>(kMTile >> 4) << 24);
+}
+
+// Running reduction of one logit row inside one thread.
+struct RowRun {
+    float m, c;
+    int idx;
+    unsigned long long acc0, acc1;
+};
+
+__device__ __forceinline__ void row_init(RowRun &r)
+{
+    r.m = -INFINITY;
+    r.c = kNoRef;
+    r.idx = 0x7fffffff;
+    r.acc0 = pack2(0.f, 0.f);
+    r.acc1 = r.acc0;
+}
+
+// 32 logits of columns v0 .. v0 + 31 (ascending over a thread's life, so a strict improvement keeps the lowest index).
+__device__ __forceinline__ void row_take(RowRun &r, const float (&x)[32], int v0)
+{
+    float cm = x[0];
+#pragma unroll
+    for (int j = 1; j < 32; ++j) cm = fmaxf(cm, x[j]);
+    if (cm > r.m) {
+        int at = 31;
+#pragma unroll
+        for (int j = 30; j >= 0; --j) at = (x[j] == cm) ? j : at;
+        r.m = cm;
+        r.idx = v0 + at;
+        const float cn = rintf(cm * kLog2e);
+        if (cn > r.c) {
+            const float f = pow2_nonpos(r.c - cn);
+            const unsigned long long f2 = pack2(f, f);
+            r.acc0 = mul2(r.acc0, f2);
+            r.acc1 = mul2(r.acc1, f2);
+            r.c = cn;
+        }
+    }
+    const unsigned long long l2e2 = pack2(kLog2e, kLog2e), negc2 = pack2(-r.c, -r.c);
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+        accum_pair(x[j], x[j + 1], l2e2, negc2, r.acc0);
+        accum_pair(x[j + 2], x[j + 3], l2e2, negc2, r.acc1);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_weight, const Params p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ unsigned int tmem_base_slot;
+    __shared__ int give_up_flag;
+    volatile int *give_up = &give_up_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const unsigned int raw = smem_u32(smem_raw);
+    const unsigned int stages = (raw + 1023u) & ~1023u;
+    const unsigned int bars = stages + kStages * kStageBytes;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
+    const unsigned int tmem_full = bars + 8u * (2 * kStages);
+    const unsigned int tmem_empty = bars + 8u * (2 * kStages + 1);
+
+    const int n_mt = p.R > kMTile ? 2 : 1;
+    const int kblocks = p.H / kBlockK;
+    const int tile0 = blockIdx.x * p.tiles_per_cta;
+    int tile1 = tile0 + p.tiles_per_cta;
+    if (tile1 > p.tiles_total) tile1 = p.tiles_total;
+    const int my_tiles = tile1 > tile0 ? tile1 - tile0 : 0;
+
+    if (threadIdx.x == 0) {
+        give_up_flag = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        mbar_init(tmem_full, 1);
+        mbar_init(tmem_empty, 4 * 32);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned int tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // ---- loader ----
+        if (lane == 0) {
+            const unsigned int tx = static_cast<unsigned int>(n_mt * kMTile * kBlockK * 2 + p.n_tile * kBlockK * 2);
+            int it = 0;
+            for (int t = tile0; t < tile1 && !*give_up; ++t) {
+                const int v0 = t * p.n_tile;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    if (!mbar_wait(empty_bar(s), ((it / kStages) & 1) ^ 1, give_up)) break;
+                    const unsigned int a = stages + s * kStageBytes, b = a + kStageABytes;
+                    mbar_expect_tx(full_bar(s), tx);
+                    tma_load_2d(a, &map_hidden, full_bar(s), kb * kBlockK, 0);
+                    if (n_mt == 2) tma_load_2d(a + kMTile * kBlockK * 2, &map_hidden, full_bar(s), kb * kBlockK, kMTile);
+                    tma_load_2d(b, &map_weight, full_bar(s), kb * kBlockK, v0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer ----
+        if (lane == 0) {
+            const unsigned int idesc = instr_desc(p.n_tile);
+            int it = 0;
+            for (int t = 0; t < my_tiles && !*give_up; ++t) {
+                if (!mbar_wait(tmem_empty, (t & 1) ^ 1, give_up)) break;      // the epilogue has drained the previous tile
+                tc_fence_after();
+                bool ok = true;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % kStages;
+                    if (!mbar_wait(full_bar(s), (it / kStages) & 1, give_up)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const unsigned int a = stages + s * kStageBytes, b = a + kStageABytes;
+                    const unsigned long long a0_desc = operand_desc(a), a1_desc = operand_desc(a + kMTile * kBlockK * 2);
+                    const unsigned long long b_desc = operand_desc(b);
+#pragma unroll
+                    for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
+                        const unsigned int acc = (kb | k4) != 0 ? 1u : 0u;
+                        // 16 columns further along K: 32 bytes, 2 in the descriptor's units of 16 bytes
+                        tc_mma_bf16(tmem_base, a0_desc + 2ull * k4, b_desc + 2ull * k4, idesc, acc);
+                        if (n_mt == 2) tc_mma_bf16(tmem_base + kNMax, a1_desc + 2ull * k4, b_desc + 2ull * k4, idesc, acc);
+                    }
+                    tc_commit(empty_bar(s));          // the stage may be refilled once these MMAs have read it
+                }
+                if (!ok) break;
+                tc_commit(tmem_full);                 // the tile's accumulators are complete
+            }
+        }
+    } else {
+        // ---- epilogue: warp w covers TMEM lanes 32 (w % 4) .. + 31 ----
+        const int q = warp & 3;
+        const int row_a = 32 * q + lane, row_b = kMTile + row_a;
+        const bool has_a = row_a < p.R, has_b = row_b < p.R;             // has_b implies has_a
+        const bool warp_b = kMTile + 32 * q < p.R;                       // the warp has any row in the second tile
+        RowRun ra, rb;
+        row_init(ra);
+        row_init(rb);
+        auto draft_of = [&](int row) {
+            const int b = row / (p.K + 1), i = row - b * (p.K + 1);
+            return (row < p.R && i < p.K) ? __ldg(p.draft + b * p.K + i) : -1;
+        };
+        const int da = draft_of(row_a), db = draft_of(row_b);
+        float zda = 0.f, zdb = 0.f;
+        bool got_a = false, got_b = false;
+        for (int t = 0; t < my_tiles; ++t) {
+            if (!mbar_wait(tmem_full, t & 1, give_up)) break;
+            tc_fence_after();
+            const int v0 = (tile0 + t) * p.n_tile;
+            const int v_end = min(p.V, v0 + p.n_tile);          // columns beyond the tile or the vocabulary are masked
+            for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
+                const int vc = v0 + c0;
+                if (vc >= v_end) break;
+                float x[32];
+                tmem_ld32(tmem_base + (static_cast<unsigned int>(32 * q) << 16) + c0, x);
+                if (vc + 32 > v_end) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) x[j] = (vc + j < v_end) ? x[j] : -INFINITY;
+                }
+                if (has_a) {
+                    row_take(ra, x, vc);
+                    if (static_cast<unsigned int>(da - vc) < 32u && da < v_end) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) zda = (da - vc == j) ? x[j] : zda;
+                        got_a = true;
+                    }
+                }
+                if (warp_b) {
+                    tmem_ld32(tmem_base + (static_cast<unsigned int>(32 * q) << 16) + kNMax + c0, x);
+                    if (vc + 32 > v_end) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) x[j] = (vc + j < v_end) ? x[j] : -INFINITY;
+                    }
+                    if (has_b) {
+                        row_take(rb, x, vc);
+                        if (static_cast<unsigned int>(db - vc) < 32u && db < v_end) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) zdb = (db - vc == j) ? x[j] : zdb;
+                            got_b = true;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(tmem_empty);
+        }
+        auto finish = [&](const RowRun &r, int row, bool got, float zd, int d) {
+            if (row >= p.R) return;
+            float s0, s1, s2, s3;
+            unpack2(r.acc0, s0, s1);
+            unpack2(r.acc1, s2, s3);
+            Partial out;
+            out.m = r.m;
+            out.idx = r.idx;
+            out.c = r.c;
+            out.s = (s0 + s1) + (s2 + s3);
+            st_partial_cg(p.partials + static_cast<size_t>(row) * gridDim.x + blockIdx.x, out);
+            if (got) {
+                const int b = row / (p.K + 1), i = row - b * (p.K + 1);
+                __stcg(p.zd + b * p.K + i, zd);
+            }
+            (void)d;
+        };
+        finish(ra, row_a, got_a, zda, da);
+        finish(rb, row_b, got_b, zdb, db);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*give_up) {
+        // a wait ran out: say so, and let copies that may still be in flight land before the block's memory is released
+        if (threadIdx.x == 0) index_check_failed(p.stats, 30u);
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) {
+        }
+        __syncthreads();
+    }
+    if (warp == 2) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---- S1 (last level) and S2..S5 per batch row, from the partials of the LM-head kernel ----------------
+struct FinalizeParams {
+    int B, K, V, n_parts;
+    const Partial *partials;     // [B*(K+1), n_parts]
+    const float *zd;             // [B, K]
+    const int *draft;
+    OcmView ocm;
+    float log_tau;
+    int *accept_len;
+    int *next_token;
+    unsigned char *rescued;
+    int *rej_d;
+    int *rej_t;
+    csd_diag_t diag;
+};
+
+__global__ void __launch_bounds__(128) lmhead_finalize_kernel(const FinalizeParams p)
+{
+    __shared__ float sm_m[4][CSD_MAX_K + 1], sm_s[4][CSD_MAX_K + 1];
+    __shared__ int sm_t[4][CSD_MAX_K + 1];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int b = blockIdx.x * 4 + w;
+    if (b >= p.B) return;
+    const int K = p.K, K1 = K + 1;
+    // the draft tokens and their logits do not depend on the fold: requested first
+    int d = -1;
+    bool valid = false;
+    float zd = __int_as_float(0x7fc00000);
+    if (lane < K) {
+        d = __ldg(p.draft + (size_t)b * K + lane);
+        valid = static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V);
+        if (valid) zd = __ldcg(p.zd + (size_t)b * K + lane);
+    }
+    for (int i = 0; i < K1; ++i) {
+        const Partial *src = p.partials + (static_cast<size_t>(b) * K1 + i) * p.n_parts;
+        Partial v = partial_identity();
+        for (int k = lane; k < p.n_parts; k += 32) {          // lane k folds parts k, k + 32, ... in order
+            const Partial x = ld_partial_cg(src + k);
+            v = (k == lane) ? x : combine(v, x);
+        }
+        // fixed-shape butterfly: maximum and its lowest index, then the sums rescaled (exactly) to its reference
+        float m = v.m;
+        int idx = v.idx;
+        for (int o = 1; o < 32; o <<= 1) {
+            const float om = __shfl_xor_sync(kFull, m, o);
+            const int oi = __shfl_xor_sync(kFull, idx, o);
+            const bool take = (om > m) || (om == m && oi < idx);
+            m = take ? om : m;
+            idx = take ? oi : idx;
+        }
+        const float c = (m == -INFINITY) ? kNoRef : rintf(m * kLog2e);
+        float s = v.s * pow2_nonpos(v.c - c);
+        for (int o = 1; o < 32; o <<= 1) s += __shfl_xor_sync(kFull, s, o);
+        if (lane == 0) {
+            sm_m[w][i] = m;
+            sm_s[w][i] = s * exp2f(fmaf(-m, kLog2e, c));      // sum exp(x - m)
+            sm_t[w][i] = idx;
+        }
+    }
+    __syncwarp();
+    for (int row = lane; row <= K; row += 32) {
+        const size_t at = (size_t)b * K1 + row;
+        const float s_m = sm_s[w][row];
+        if (!(s_m == s_m) || s_m == INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
+        if (p.diag.m) p.diag.m[at] = sm_m[w][row];
+        if (p.diag.s) p.diag.s[at] = s_m;
+        if (p.diag.lse) p.diag.lse[at] = sm_m[w][row] + logf(s_m);
+        if (p.diag.t) p.diag.t[at] = sm_t[w][row];
+    }
+    bool match = false, ok = false;
+    int t = -1;
+    unsigned int cnt = 0;
+    if (lane < K) {
+        t = sm_t[w][lane];
+        match = (d == t);
+        if (valid) cnt = ocm_lookup(p.ocm, make_key(d, t));                        // S3
+        const float m = sm_m[w][lane], s_m = sm_s[w][lane];
+        const bool is_freq = cnt >= p.ocm.lambda;
+        const bool is_safe = (static_cast<double>(zd) - static_cast<double>(m)) >= static_cast<double>(p.log_tau);   // S4, Eq. 3
+        ok = match || (valid && is_freq && is_safe);
+        const size_t pos = (size_t)b * K + lane;
+        if (p.diag.zd) p.diag.zd[pos] = zd;
+        if (p.diag.cnt) p.diag.cnt[pos] = cnt;
+        if (p.diag.score) p.diag.score[pos] = expf(zd - m);
+        if (p.diag.p_d) p.diag.p_d[pos] = expf(zd - m) / s_m;
+        if (p.diag.p_t) p.diag.p_t[pos] = 1.0f / s_m;
+    }
+    const unsigned int kmask = (K == 32) ? kFull : ((1u << K) - 1u);
+    const unsigned int fail = ~(__ballot_sync(kFull, ok) & kmask) & kmask;
+    const int n_acc = fail ? (__ffs(fail) - 1) : K;                                    // S5
+    const bool reached = lane <= n_acc && lane < K;
+    const bool record = reached && !match && valid;
+    if (lane < K) {
+        const size_t pos = (size_t)b * K + lane;
+        p.rescued[pos] = (lane < n_acc && !match) ? 1 : 0;
+        p.rej_d[pos] = record ? d : -1;
+        p.rej_t[pos] = record ? t : -1;
+    }
+    const unsigned int m_match = __ballot_sync(kFull, reached && match);
+    const unsigned int m_resc = __ballot_sync(kFull, lane < n_acc && !match && lane < K);
+    const unsigned int m_rec = __ballot_sync(kFull, record);
+    const unsigned int m_bad = __ballot_sync(kFull, lane < K && !valid);
+    if (lane == 0) {
+        p.accept_len[b] = n_acc;
+        p.next_token[b] = sm_t[w][n_acc];
+        OcmStatsDev *st = p.ocm.stats;
+        atomicAdd(&st->positions, static_cast<unsigned long long>(K));
+        if (m_match) atomicAdd(&st->matches, static_cast<unsigned long long>(__popc(m_match)));
+        if (m_resc) atomicAdd(&st->rescues, static_cast<unsigned long long>(__popc(m_resc)));
+        if (m_rec) atomicAdd(&st->rejections, static_cast<unsigned long long>(__popc(m_rec)));
+        if (m_bad) atomicOr(&st->flags, CSD_FLAG_BAD_DRAFT);
+        if (b == 0) atomicAdd(&st->steps, 1ull);
+    }
+}
+
+}  // namespace lmhead
+}  // namespace csd

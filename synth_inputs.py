@@ -192,6 +192,56 @@ class Synth:
         return z, y.to(wl.torch_dtype).contiguous(), draft, r.contiguous()
 
 
+    # ---- inputs of the LM head: the step that never stores its logits --------------------------------
+    def lmhead_weight(self, H: int) -> torch.Tensor:
+        """W[V, H] bf16, N(0, 1/H) entries: with hidden rows of N(0, sigma^2) entries the logits hidden . W[v]
+        are N(0, sigma^2) noise, as in `step`.  Fixed by (seed, workload)."""
+        g = self._gen(5, 0)
+        w = torch.randn(self.wl.V, H, generator=g, device=self.device, dtype=torch.float32)
+        return w.mul_(H ** -0.5).to(torch.bfloat16).contiguous()
+
+    def step_lmhead(self, step: int, W: torch.Tensor):
+        """(hidden[B, K+1, H] bf16, draft[B, K] int32) for one step whose logits are hidden @ W^T.
+
+        The same recipe as `step`, expressed through the hidden state: a row is noise plus `peak` times the
+        (normalised) weight row of its raised token, which lifts that token's logit by `peak`; at a synonym
+        position a component along the draft token's weight row puts its logit U(0, 3) below the raised
+        token's (up to the small overlap of two random weight rows).  "Match" drafts are the arg-max of the
+        finished row, taken from a float32 product of the rounded inputs."""
+        wl, dev = self.wl, self.device
+        B, K, V = wl.B, wl.K, wl.V
+        H = W.shape[1]
+        g = self._gen(6, step)
+        h = torch.randn(B, K + 1, H, generator=g, device=dev, dtype=torch.float32).mul_(wl.sigma)
+        kind_u = torch.rand(B, K, generator=g, device=dev)
+        pair_u = torch.rand(B, K, generator=g, device=dev)
+        gap_u = torch.rand(B, K, generator=g, device=dev)
+        peak_u = torch.rand(B, generator=g, device=dev)
+        top = torch.randint(0, V, (B, K + 1), generator=g, device=dev)
+        uni = torch.randint(0, V, (B, K), generator=g, device=dev)
+        is_match = kind_u < wl.mix[0]
+        is_syn = (~is_match) & (kind_u < wl.mix[0] + wl.mix[1])
+        pair = self._draw_pairs(pair_u.reshape(-1)).reshape(B, K)
+        syn_t, syn_d = self.map_target[pair], self.map_draft[pair]
+        top[:, :K] = torch.where(is_syn, syn_t, top[:, :K])
+        peak = (wl.peak[0] + (wl.peak[1] - wl.peak[0]) * peak_u).view(B, 1, 1)
+        wt = W[top].to(torch.float32)                                        # [B, K+1, H]
+        h = h + peak * wt / wt.pow(2).sum(-1, keepdim=True)
+        wd = W[syn_d].to(torch.float32)                                      # [B, K, H]
+        z_top = (h[:, :K] * wt[:, :K]).sum(-1)
+        z_d = (h[:, :K] * wd).sum(-1)
+        lift = torch.where(is_syn, z_top - 3.0 * gap_u - z_d, torch.zeros_like(z_d))
+        h[:, :K] = h[:, :K] + lift.unsqueeze(-1) * wd / wd.pow(2).sum(-1, keepdim=True)
+        h = h.to(torch.bfloat16).contiguous()
+        arg = torch.empty(B, K, dtype=torch.int64, device=dev)
+        for b in range(B):                                                   # a [K, V] product at a time
+            arg[b] = (h[b, :K].to(torch.float32) @ W.to(torch.float32).T if V * H <= (1 << 24) else
+                      torch.cat([h[b, :K].to(torch.float32) @ W[v0:v0 + 32768].to(torch.float32).T
+                                 for v0 in range(0, V, 32768)], dim=1)).argmax(dim=1)
+        draft = torch.where(is_match, arg, torch.where(is_syn, syn_d, uni)).to(torch.int32)
+        return h, draft.contiguous()
+
+
 def logits_to_numpy(z: torch.Tensor):
     """Exact host copy for the oracle: float32 array (bf16 widens exactly)."""
     return z.detach().to("cpu").to(torch.float32).numpy()
