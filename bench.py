@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0            # earlier measurement on this machine, used wh
 DEFAULT_WORKLOAD = "large_batch"
 # DRAM bytes per launch of the step kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); a workload is absent where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"large_batch": 596683008, "batched_serving": 58530816}
+NCU_TRAFFIC_BYTES = {"ocm_contention": 140787712}
 
 
 def measured_peak():
@@ -464,6 +464,13 @@ def run_ours(args, wl, tau):
                 line["sampled"] = measure_sampled(args, wl, tau, device, graph_steps=16, min_steps=48, count_draws=True)
             except Exception as e:             # the greedy line stands on its own
                 line["sampled"] = {"error": repr(e)}
+            try:
+                from synth_inputs import WORKLOADS
+                torch.cuda.empty_cache()
+                line["lmhead"] = measure_lmhead(WORKLOADS["batched_serving"], 0.3, device)
+                pkg.csd_set_overlap(overlap)
+            except Exception as e:
+                line["lmhead"] = {"error": repr(e)}
         print(json.dumps(line), flush=True)
     else:
         bench.ocm.close()
@@ -607,6 +614,97 @@ def run_sampled(args, wl, tau):
     print(json.dumps(line), flush=True)
 
 
+def measure_lmhead(wl, tau, device, H=4096, steps=12, repeats=7):
+    """csd_step_lmhead (the step taken straight from the LM head: tcgen05 GEMM with the row statistics in its
+    epilogue, decisions, memory update) on hidden[B, K+1, H] and weight[V, H], beside the unfused pair it
+    replaces (a library bf16 GEMM that stores the logits, then csd_step on them)."""
+    import torch
+
+    import paper_2604_13634_b200 as pkg
+    from synth_inputs import Synth
+
+    syn = Synth(wl, 0, device)
+    W = syn.lmhead_weight(H)
+    ins = [syn.step_lmhead(s, W) for s in range(3)]
+    ocm = pkg.Ocm(wl.ocm_slots, wl.lam, device.index)
+    buf = pkg.LmheadBuffers(wl.B, wl.K, H, wl.V, device=device)
+    R = wl.B * (wl.K + 1)
+
+    def timed(fn):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize(device)
+        ts = []
+        for _ in range(repeats):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(steps):
+                fn(i)
+            b.record()
+            b.synchronize()
+            ts.append(a.elapsed_time(b) * 1e-3 / steps)
+        return statistics.median(ts)
+
+    fused = timed(lambda i: pkg.csd_step_lmhead(ins[i % 3][0], W, ins[i % 3][1], ocm, tau, buf))
+    sb = pkg.StepBuffers(wl.B, wl.K, wl.V, torch.bfloat16, device=device)
+    pkg.csd_set_overlap(False)
+
+    def unfused(i):
+        h, d = ins[i % 3]
+        z = torch.matmul(h.view(R, H), W.T).view(wl.B, wl.K + 1, wl.V)
+        pkg.csd_step(z, d, ocm, tau, sb)
+    plain = timed(unfused)
+    st = ocm.stats()
+    ocm.close()
+    hbm, kind = measured_peak()
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            tensor_peak = float(json.load(f)["bf16_tflops"])
+    except Exception:
+        tensor_peak = 1590.0
+    flops = 2.0 * R * H * wl.V
+    hbm_bytes = (wl.V + R) * H * 2.0                     # the weight matrix and the hidden states once
+    t_bound = max(flops / (tensor_peak * 1e12), hbm_bytes / (hbm * 1e9))
+    return {"us_per_step": 1e6 * fused, "positions_per_s": wl.B * wl.K / fused, "steps": steps, "repeats": repeats,
+            "H": H, "rows": R, "V": wl.V, "shape": pkg.csd_lmhead_shape(wl.B, wl.K, H, wl.V),
+            "tensor_TFLOPs": flops / fused / 1e12, "tensor_frac": flops / fused / 1e12 / tensor_peak,
+            "hbm_GBs": hbm_bytes / fused / 1e9, "hbm_frac": hbm_bytes / fused / 1e9 / hbm,
+            "bound": "hbm" if hbm_bytes / (hbm * 1e9) >= flops / (tensor_peak * 1e12) else "tensor",
+            "roofline_us": 1e6 * t_bound, "frac_of_roofline": t_bound / fused, "peak_source": f"of {kind}",
+            "unfused_us_per_step": 1e6 * plain,
+            "unfused": "torch.matmul (bf16 logits stored, 58 MB written and read back) followed by csd_step",
+            "launches_per_step": 3, "launch": "eager",
+            "ocm": {k: st[k] for k in ("n_keys", "rescues", "rejections", "flags")}}
+
+
+def run_lmhead(args, wl, tau):
+    """--mode lmhead: a bench line of its own for the step taken straight from the LM head."""
+    import torch
+
+    import paper_2604_13634_b200 as pkg
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    pkg.lib()
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    sampler = ClockSampler(device.index, period_s=0.005)
+    sampler.start()
+    m = measure_lmhead(wl, tau, device, H=args.hidden, steps=max(3, min(args.steps, 48)))
+    clocks = sampler.stop()
+    line = {"metric": METRIC, "value": m["positions_per_s"], "unit": UNIT, "n_gpus": 1, "steps": m["steps"],
+            "warmup": 3, "ms_per_step": m["us_per_step"] * 1e-3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "repeats": m["repeats"],
+            "config": workload_config(wl, tau, {"mode": "step taken straight from the LM head (logits never stored)",
+                                                "H": m["H"], "kernel_shape": m["shape"], "launch": m["launch"],
+                                                "l2_policy": "the 1.2 GB weight matrix is larger than L2"}),
+            "roofline": {"bound": m["bound"], "achieved": m["hbm_GBs"] if m["bound"] == "hbm" else m["tensor_TFLOPs"],
+                         "peak": measured_peak()[0] if m["bound"] == "hbm" else None, "unit": "GB/s" if m["bound"] == "hbm" else "TFLOP/s",
+                         "frac": m["frac_of_roofline"], "traffic": None, "peak_source": m["peak_source"],
+                         "kernel": "lmhead_stats_kernel", "tensor_TFLOPs": m["tensor_TFLOPs"], "tensor_frac": m["tensor_frac"]},
+            "gpu_launches": 3 * m["steps"], "clocks": clocks, "lmhead": m}
+    print(json.dumps(line), flush=True)
+
+
 def run_extras(device, skip, peak, names, overlap):
     """Short device-resident runs of the other workloads (extra keys, not bench lines): the pipelined loop
     (about a quarter of a second, median of 7 regions) and the latency of a step that runs alone."""
@@ -661,8 +759,10 @@ def main():
     ap.add_argument("--lean", action="store_true", help="only the headline measurement: no other workloads, no stand-alone "
                                                          "latency, no stochastic sub-record")
     ap.add_argument("--repeats", type=int, default=0, help="how often the timed region is taken (0 = automatic, at least 7)")
-    ap.add_argument("--mode", default="greedy", choices=["greedy", "sampled"],
-                    help="sampled: the stochastic verification step (its own JSON line; 1 GPU)")
+    ap.add_argument("--mode", default="greedy", choices=["greedy", "sampled", "lmhead"],
+                    help="sampled: the stochastic verification step; lmhead: the step taken straight from the LM head "
+                         "(each its own JSON line; 1 GPU)")
+    ap.add_argument("--hidden", type=int, default=4096, help="H of --mode lmhead")
     ap.add_argument("--temperature", type=float, default=0.3, help="T of --mode sampled")
     args = ap.parse_args()
 
@@ -673,6 +773,8 @@ def main():
         run_reference(args, wl, tau)
     elif args.mode == "sampled":
         run_sampled(args, wl, tau)
+    elif args.mode == "lmhead":
+        run_lmhead(args, WORKLOADS["batched_serving"] if args.workload == DEFAULT_WORKLOAD else wl, tau if args.workload != DEFAULT_WORKLOAD else 0.3)
     else:
         run_ours(args, wl, tau)
 

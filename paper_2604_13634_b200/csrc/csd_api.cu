@@ -779,6 +779,7 @@ namespace {
 
 struct LmheadPlan {
     int grid, n_tile, tiles_total, tiles_per_cta;
+    int rows2, a_bytes, stage_bytes, n_stages, smem_bytes;
     size_t partials_off, zd_off, total;
 };
 
@@ -807,6 +808,14 @@ LmheadPlan lmhead_plan(int B, int K, int V)
     long long grid = (pl.tiles_total + per - 1) / per;
     pl.grid = static_cast<int>(grid < 1 ? 1 : grid);
     const size_t rows = static_cast<size_t>(B) * (K + 1);
+    // shared-memory ring: as many stages as fit beside the barriers, the alignment room and the slack
+    pl.rows2 = rows > lmhead::kMTile ? static_cast<int>((rows - lmhead::kMTile + 7) / 8 * 8) : 0;
+    pl.a_bytes = static_cast<int>(align_up(static_cast<size_t>(lmhead::kMTile + pl.rows2) * lmhead::kRowBytes, 1024));
+    pl.stage_bytes = pl.a_bytes + static_cast<int>(align_up(static_cast<size_t>(pl.n_tile) * lmhead::kRowBytes, 1024));
+    const int fixed = 1024 + lmhead::kBarrierBytes + lmhead::kSlackBytes;
+    int stages = (lmhead::kSmemLimit - fixed) / pl.stage_bytes;
+    pl.n_stages = stages > lmhead::kMaxStages ? lmhead::kMaxStages : stages;
+    pl.smem_bytes = fixed + pl.n_stages * pl.stage_bytes;
     pl.partials_off = 0;
     pl.zd_off = align_up(rows * pl.grid * sizeof(Partial), 256);
     pl.total = align_up(pl.zd_off + static_cast<size_t>(B) * K * sizeof(float), 256);
@@ -877,7 +886,7 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     {
         std::lock_guard<std::mutex> lock(attr_mutex);
         if (!attr_set[dev]) {
-            if (cudaFuncSetAttribute(lmhead::lmhead_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lmhead::kSmemBytes) !=
+            if (cudaFuncSetAttribute(lmhead::lmhead_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lmhead::kSmemLimit) !=
                 cudaSuccess) {
                 (void)cudaGetLastError();
                 return CSD_ERR_CUDA;
@@ -885,8 +894,9 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
             attr_set[dev] = true;
         }
     }
-    CUtensorMap map_h, map_w;
+    CUtensorMap map_h, map_h2, map_w;
     if (!make_map(&map_h, hidden, static_cast<uint64_t>(R), static_cast<uint64_t>(H), lmhead::kMTile) ||
+        !make_map(&map_h2, hidden, static_cast<uint64_t>(R), static_cast<uint64_t>(H), static_cast<uint32_t>(pl.rows2 ? pl.rows2 : 8)) ||
         !make_map(&map_w, weight, static_cast<uint64_t>(V), static_cast<uint64_t>(H), static_cast<uint32_t>(pl.n_tile)))
         return CSD_ERR_CUDA;
 
@@ -897,11 +907,15 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     p.n_tile = pl.n_tile;
     p.tiles_total = pl.tiles_total;
     p.tiles_per_cta = pl.tiles_per_cta;
+    p.rows2 = pl.rows2;
+    p.a_bytes = pl.a_bytes;
+    p.stage_bytes = pl.stage_bytes;
+    p.n_stages = pl.n_stages;
     p.draft = draft;
     p.partials = reinterpret_cast<Partial *>(ws + pl.partials_off);
     p.zd = reinterpret_cast<float *>(ws + pl.zd_off);
     p.stats = ocm->stats;
-    lmhead::lmhead_stats_kernel<<<pl.grid, lmhead::kThreads, lmhead::kSmemBytes, st>>>(map_h, map_w, p);
+    lmhead::lmhead_stats_kernel<<<pl.grid, lmhead::kThreads, pl.smem_bytes, st>>>(map_h, map_h2, map_w, p);
     if (cudaGetLastError() != cudaSuccess) return CSD_ERR_CUDA;
 
     lmhead::FinalizeParams f;

@@ -5,8 +5,8 @@
 //
 //   lmhead_stats_kernel     persistent, one CTA per SM, 192 threads:
 //       warp 0      one thread issues the TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of the k-blocks:
-//                   64 columns of all hidden rows (two boxes of 128 rows; rows beyond R read as zero) and of
-//                   the vocabulary tile's W rows, into a ring of shared-memory stages
+//                   64 columns of all hidden rows (a box of 128 rows and one of the rows beyond) and of the
+//                   vocabulary tile's W rows, into a ring of as many shared-memory stages as fit (3 to 8)
 //       warp 1      one thread issues the MMAs (tcgen05.mma, kind::f16, M = 128, N = tile width, K = 16, fp32
 //                   accumulators in tensor memory: columns [0, N) for rows 0..127, [256, 256 + N) for rows
 //                   128..255) and commits each stage back to the loader, each finished tile to the epilogue
@@ -33,16 +33,18 @@ namespace csd {
 namespace lmhead {
 
 constexpr int kBlockK = 64;                 // bf16 elements of a k-block: one 128-byte swizzle row
-constexpr int kStages = 3;
+constexpr int kMaxStages = 8;
 constexpr int kMTile = 128;
 constexpr int kRowsMax = 2 * kMTile;        // logit rows a step may have
 constexpr int kNMax = 256;                  // widest vocabulary tile
 constexpr int kThreads = 192;
-constexpr int kStageABytes = kRowsMax * kBlockK * 2;
-constexpr int kStageBBytes = kNMax * kBlockK * 2;
-constexpr int kStageBytes = kStageABytes + kStageBBytes;
-constexpr int kBarrierBytes = 256;
-constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;     // + room to align the stages to 1 KiB
+constexpr int kRowBytes = kBlockK * 2;      // one row of a k-block
+constexpr int kBarrierBytes = 1024;
+// The second row tile's operand is read as 128 rows although only the rows that exist are loaded: the read
+// runs on into whatever follows (the stage's W tile, the next stage, or this slack), which only feeds
+// accumulator rows that nobody reads.
+constexpr int kSlackBytes = kMTile * kRowBytes;
+constexpr int kSmemLimit = 226 * 1024;      // of the 227 KiB a block may have (some is static)
 constexpr int kTmemCols = 512;
 constexpr long long kWaitCycles = 4000000000ll;
 
@@ -51,6 +53,10 @@ struct Params {
     int n_tile;             // columns of a vocabulary tile: multiple of 16, at most kNMax
     int tiles_total;        // ceil(V / n_tile)
     int tiles_per_cta;
+    int rows2;              // rows loaded for the second row tile (0 if R <= 128), a multiple of 8
+    int a_bytes;            // bytes of the hidden k-block in a stage (both row tiles), a multiple of 1 KiB
+    int stage_bytes;        // a_bytes + the W tile's k-block, a multiple of 1 KiB
+    int n_stages;
     const int *draft;       // [B, K]
     Partial *partials;      // [R, gridDim.x]
     float *zd;              // [B, K]  z[b, i, draft[b, i]] (written for valid draft ids only)
@@ -208,7 +214,8 @@ __device__ __forceinline__ void row_take(RowRun &r, const float (&x)[32], int v0
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_weight, const Params p)
+lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_hidden2,
+                    const __grid_constant__ CUtensorMap map_weight, const Params p)
 {
     extern __shared__ unsigned char smem_raw[];
     __shared__ unsigned int tmem_base_slot;
@@ -218,12 +225,14 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const unsigned int raw = smem_u32(smem_raw);
-    const unsigned int stages = (raw + 1023u) & ~1023u;
-    const unsigned int bars = stages + kStages * kStageBytes;
+    const unsigned int bars = (raw + 1023u) & ~1023u;
+    const unsigned int stages = bars + kBarrierBytes;
+    const int kStages = p.n_stages;
+    const int kStageBytes = p.stage_bytes, kStageABytes = p.a_bytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
-    const unsigned int tmem_full = bars + 8u * (2 * kStages);
-    const unsigned int tmem_empty = bars + 8u * (2 * kStages + 1);
+    auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    const unsigned int tmem_full = bars + 8u * (2 * kMaxStages);
+    const unsigned int tmem_empty = bars + 8u * (2 * kMaxStages + 1);
 
     const int n_mt = p.R > kMTile ? 2 : 1;
     const int kblocks = p.H / kBlockK;
@@ -254,7 +263,7 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
     if (warp == 0) {
         // ---- loader ----
         if (lane == 0) {
-            const unsigned int tx = static_cast<unsigned int>(n_mt * kMTile * kBlockK * 2 + p.n_tile * kBlockK * 2);
+            const unsigned int tx = static_cast<unsigned int>((kMTile + p.rows2 + p.n_tile) * kRowBytes);
             int it = 0;
             for (int t = tile0; t < tile1 && !*give_up; ++t) {
                 const int v0 = t * p.n_tile;
@@ -264,7 +273,7 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
                     const unsigned int a = stages + s * kStageBytes, b = a + kStageABytes;
                     mbar_expect_tx(full_bar(s), tx);
                     tma_load_2d(a, &map_hidden, full_bar(s), kb * kBlockK, 0);
-                    if (n_mt == 2) tma_load_2d(a + kMTile * kBlockK * 2, &map_hidden, full_bar(s), kb * kBlockK, kMTile);
+                    if (n_mt == 2) tma_load_2d(a + kMTile * kRowBytes, &map_hidden2, full_bar(s), kb * kBlockK, kMTile);
                     tma_load_2d(b, &map_weight, full_bar(s), kb * kBlockK, v0);
                 }
             }
@@ -286,7 +295,7 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
                     }
                     tc_fence_after();
                     const unsigned int a = stages + s * kStageBytes, b = a + kStageABytes;
-                    const unsigned long long a0_desc = operand_desc(a), a1_desc = operand_desc(a + kMTile * kBlockK * 2);
+                    const unsigned long long a0_desc = operand_desc(a), a1_desc = operand_desc(a + kMTile * kRowBytes);
                     const unsigned long long b_desc = operand_desc(b);
 #pragma unroll
                     for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
