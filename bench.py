@@ -465,6 +465,12 @@ def run_ours(args, wl, tau):
             except Exception as e:             # the greedy line stands on its own
                 line["sampled"] = {"error": repr(e)}
             try:
+                torch.cuda.empty_cache()
+                line["early_exit"] = measure_early_exit(wl, tau, device)
+                pkg.csd_set_overlap(overlap)
+            except Exception as e:
+                line["early_exit"] = {"error": repr(e)}
+            try:
                 from synth_inputs import WORKLOADS
                 torch.cuda.empty_cache()
                 line["lmhead"] = measure_lmhead(WORKLOADS["batched_serving"], 0.3, device)
@@ -612,6 +618,74 @@ def run_sampled(args, wl, tau):
         line["cpu_baseline"] = {"value": rows_b * wl.K * n / secs, "unit": UNIT, "cores": 1, "kind": "oracle",
                                 "sample": f"{n} oracle steps over {rows_b} of the workload's {wl.B} batch rows in {secs:.1f} s"}
     print(json.dumps(line), flush=True)
+
+
+def measure_early_exit(wl, tau, device, steps=48):
+    """csd_step_early_exit (the step in two phases: batch rows that stop within the first phase are not read any
+    further) as a stream-ordered graph over the ring, beside csd_step run the same way; the bytes it reads follow
+    from how many batch rows survive the first phase."""
+    import torch
+
+    import paper_2604_13634_b200 as pkg
+    from synth_inputs import Synth
+
+    l2 = torch.cuda.get_device_properties(device).L2_cache_size
+    ring_len = max(2, math.ceil(2 * l2 / wl.logit_bytes) + 1)
+    syn = Synth(wl, 0, device)
+    ring = [syn.step(s) for s in range(ring_len)]
+    pkg.csd_set_overlap(False)
+
+    def prepared():
+        ocm = pkg.Ocm(wl.ocm_slots, wl.lam, device.index)
+        if wl.prewarm[0] == "pairs":
+            ocm.update(*syn.prewarm_pairs(wl.prewarm[1]))
+        return ocm
+
+    def graph_time(call):
+        side = torch.cuda.Stream(device)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(ring_len):
+                call(i)
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(steps):
+                call(i)
+        g.replay()
+        torch.cuda.synchronize(device)
+        ts = []
+        for _ in range(7):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            g.replay()
+            b.record()
+            b.synchronize()
+            ts.append(a.elapsed_time(b) * 1e-3 / steps)
+        return statistics.median(ts)
+
+    ocm = prepared()
+    buf = pkg.EarlyExitBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, first=0, device=device)
+    first = min(max(1, (wl.K + 1) // 3), wl.K - 1)
+    t_two = graph_time(lambda i: pkg.csd_step_early_exit(*ring[i % ring_len], ocm, tau, buf))
+    alive = []
+    for i in range(ring_len):                      # with the memory as the timed run left it
+        pkg.csd_step_early_exit(*ring[i], ocm, tau, buf)
+        alive.append(int((buf.accept_len >= first).sum().item()))
+    ocm.close()
+    ocm = prepared()
+    sb = pkg.StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, device=device)
+    t_one = graph_time(lambda i: pkg.csd_step(*ring[i % ring_len], ocm, tau, sb))
+    ocm.close()
+    mean_alive = sum(alive) / len(alive)
+    row_bytes = wl.V * wl.elt_bytes
+    read = (wl.B * (first + 1) + mean_alive * (wl.K + 1 - first)) * row_bytes
+    peak, kind = measured_peak()
+    return {"us_per_step": 1e6 * t_two, "csd_step_alone_us_per_step": 1e6 * t_one, "first_phase_positions": first,
+            "batch_rows_alive_after_first_phase": mean_alive, "of_batch_rows": wl.B,
+            "logit_bytes_read": read, "logit_bytes_of_csd_step": wl.logit_bytes, "bytes_fraction": read / wl.logit_bytes,
+            "achieved_GBs": read / t_two / 1e9, "frac_of_measured_peak": read / t_two / 1e9 / peak, "peak_source": f"of {kind}",
+            "launch": f"CUDA graph of {steps} steps (3 launches each), stream-ordered, replayed", "repeats": 7}
 
 
 def measure_lmhead(wl, tau, device, H=4096, steps=12, repeats=7):

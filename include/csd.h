@@ -221,6 +221,26 @@ csd_status_t csd_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
                       const csd_diag_t *diag,
                       void *workspace, size_t workspace_bytes, void *stream);
 
+/* csd_step in two phases, for steps in which many rows stop early.  Algorithm 1 returns at a row's first
+ * un-rescued rejection and never looks at the positions after it; csd_step nevertheless streams all K+1 logit
+ * rows of every batch row, because it decides everything in one pass.  This variant first verifies positions
+ * 0 .. f-1 of every batch row (reading logit rows 0 .. f), then positions f .. K-1 and the bonus row only of the
+ * batch rows that accepted all of the first f (reading their logit rows f .. K), and finally updates the memory
+ * with all recorded pairs in (b, i) order -- after the last look-up, as csd_step does.  Results are those of
+ * csd_step; the optional diagnostics are written only for the logit rows that were read.  Bytes read:
+ * B (f+1) V + (rows still alive) (K+1-f) V elements instead of B (K+1) V.
+ * first_phase_positions: f, 1 .. K-1 (0 = automatic, about K/3).  K >= 2.  The launches of this call are
+ * plain stream-ordered launches whatever csd_set_overlap says.
+ * workspace: csd_early_exit_workspace_bytes bytes for the same first_phase_positions, 16-byte aligned.
+ * Three launches; asynchronous.  Errors as csd_step; UNSUPPORTED for K < 2. */
+size_t csd_early_exit_workspace_bytes(int B, int K, int V, csd_dtype_t dtype, int first_phase_positions);
+csd_status_t csd_step_early_exit(const void *logits, csd_dtype_t dtype, int B, int K, int V,
+                                 int64_t stride_b, int64_t stride_k,
+                                 const int32_t *draft, csd_ocm_t *ocm, float tau, int first_phase_positions,
+                                 int32_t *accept_len, int32_t *next_token, uint8_t *rescued_mask,
+                                 int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
+                                 void *workspace, size_t workspace_bytes, void *stream);
+
 /* csd_verify without a workspace argument and without any allocation.  (The paper has
  * no counterpart: this is a deployment convenience of the library.)
  *

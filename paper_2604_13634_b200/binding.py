@@ -30,6 +30,7 @@ EXPORTS = [
     "csd_sampled_workspace_bytes", "csd_verify_sampled", "csd_step_sampled",
     "csd_ocm_age", "csd_ocm_merge", "csd_ocm_save", "csd_ocm_load", "csd_ocm_set_shared",
     "csd_lmhead_workspace_bytes", "csd_verify_lmhead", "csd_step_lmhead", "csd_lmhead_shape",
+    "csd_early_exit_workspace_bytes", "csd_step_early_exit",
 ]
 
 
@@ -98,6 +99,8 @@ def lib():
         "csd_verify_lmhead": (c_int, lmhead_args),
         "csd_step_lmhead": (c_int, lmhead_args),
         "csd_lmhead_shape": (c_int, [c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
+        "csd_early_exit_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int, c_int]),
+        "csd_step_early_exit": (c_int, step_args[:10] + [c_int] + step_args[10:]),
         "csd_ocm_age": (c_int, [c_void_p, c_void_p]),
         "csd_ocm_set_shared": (c_int, [c_void_p, c_int]),
         "csd_ocm_merge": (c_int, [c_void_p, c_void_p, c_void_p]),
@@ -457,3 +460,28 @@ def csd_verify_lmhead(hidden, weight, draft, ocm: Ocm, tau: float, buf: LmheadBu
 def csd_step_lmhead(hidden, weight, draft, ocm: Ocm, tau: float, buf: LmheadBuffers, stream=None):
     """csd_step on the logits hidden @ weight^T, which are never stored."""
     _lmhead_call("csd_step_lmhead", hidden, weight, draft, ocm, tau, buf, stream)
+
+
+class EarlyExitBuffers(StepBuffers):
+    """Outputs, optional diagnostics and workspace of csd_step_early_exit for one shape and first-phase length."""
+
+    def __init__(self, B: int, K: int, V: int, dtype: torch.dtype, first: int = 0, device="cuda", diag: bool = False):
+        super().__init__(B, K, V, dtype, device=device, diag=diag)
+        self.first = first
+        self.ws_bytes = int(lib().csd_early_exit_workspace_bytes(B, K, V, self.dtype_code, first))
+        if self.ws_bytes == 0:
+            raise CsdError(f"unsupported shape for the two-phase step: B={B} K={K} V={V}")
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=torch.device(device))
+
+
+def csd_step_early_exit(logits, draft, ocm: Ocm, tau: float, buf: EarlyExitBuffers, stream=None):
+    """csd_step in two phases: batch rows that stop within the first phase are not read any further."""
+    assert logits.is_cuda and draft.is_cuda and draft.dtype == torch.int32 and draft.is_contiguous()
+    B, K1, V = logits.shape
+    assert (B, K1 - 1, V) == (buf.B, buf.K, buf.V) and logits.stride(2) == 1 and _dtype_code(logits) == buf.dtype_code
+    rc = lib().csd_step_early_exit(
+        logits.data_ptr(), buf.dtype_code, B, K1 - 1, V, logits.stride(0), logits.stride(1), draft.data_ptr(), ocm.handle,
+        c_float(tau), buf.first, _ptr(buf.accept_len), _ptr(buf.next_token), _ptr(buf.rescued_mask), _ptr(buf.rej_draft),
+        _ptr(buf.rej_target), byref(buf._diag_struct) if buf._diag_struct is not None else None, _ptr(buf.workspace),
+        buf.ws_bytes, _stream_ptr(stream))
+    _check(rc, "csd_step_early_exit")

@@ -255,11 +255,22 @@ OcmView view_of(const csd_ocm *o)
     return v;
 }
 
+// A launch that covers positions pos0 .. pos0 + K - 1 of a step with K_total positions, on all batch rows or on
+// the rows listed in device memory (the two phases of csd_step_early_exit).
+struct PhaseSpec {
+    int K_total, pos0;
+    const int *row_map, *n_rows;
+    int *alive_out, *n_alive_out;
+    int count_positions, count_step;
+};
+
+constexpr int kListSlotsPerRow = 66;   // a launch over a row list may put up to 64 blocks (+ 2 boundary blocks) on a logit row
+
 csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b, int64_t stride_k,
                       const int32_t *draft, const csd_ocm *ocm, float tau, int32_t *accept_len, int32_t *next_token,
                       uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target, const csd_diag_t *diag,
                       void *workspace, size_t workspace_bytes, void *stream, bool do_update, bool may_chain = true,
-                      bool may_overlap = true, bool track_layout = true)
+                      bool may_overlap = true, bool track_layout = true, const PhaseSpec *phase = nullptr)
 {
     if (!logits || !draft || !ocm || !accept_len || !next_token || !rescued_mask || !rej_draft || !rej_target || !workspace)
         return CSD_ERR_INVALID_ARG;
@@ -268,9 +279,10 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     if (K > CSD_MAX_K) return CSD_ERR_UNSUPPORTED;
     if (!shape_ok(B, K, V, dtype)) return CSD_ERR_UNSUPPORTED;
     if (!(tau >= 0.0f) || std::isinf(tau)) return CSD_ERR_INVALID_ARG;   // also refuses NaN
-    if (stride_k < V || stride_b < stride_k * (K + 1)) return CSD_ERR_INVALID_ARG;
+    if (stride_k < V || stride_b < stride_k * ((phase ? phase->K_total : K) + 1)) return CSD_ERR_INVALID_ARG;
 
-    const Shape s = pick_shape(B, K, V, dtype, g_overlap_steps != 0);
+    Shape s = pick_shape(B, K, V, dtype, g_overlap_steps != 0 && may_overlap);
+    if (phase && phase->n_rows) s.slots_per_row = s.units_per_row < kListSlotsPerRow ? s.units_per_row : kListSlotsPerRow;
     const WorkspaceLayout w = ws_layout(B, K, s);
     if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
 
@@ -302,6 +314,17 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     p.chunk_units = s.chunk_units;
     p.total_units = s.total_units;
     p.narrow = ((s.total_units + 1) * (static_cast<long long>(s.grid) + 1) < (1ll << 32) && s.total_units * 40 < (1ll << 32)) ? 1 : 0;
+    if (phase) {
+        p.K_total = phase->K_total;
+        p.pos0 = phase->pos0;
+        p.row_map = phase->row_map;
+        p.n_rows = phase->n_rows;
+        p.alive_out = phase->alive_out;
+        p.n_alive_out = phase->n_alive_out;
+        p.count_positions = phase->count_positions;
+        p.count_step = phase->count_step;
+        p.min_units = (g_overlap_steps != 0 && may_overlap) ? 16 : 64;
+    }
     if (track_layout) {
         const unsigned long long sig[3] = {
             (static_cast<unsigned long long>(static_cast<unsigned int>(B)) << 32) | static_cast<unsigned int>(K),
@@ -633,6 +656,66 @@ csd_status_t csd_ocm_set_shared(csd_ocm_t *ocm, int enable)
     }
     ocm->shared = enable ? 1 : 0;
     return CSD_OK;
+}
+
+// ---- the step in two phases: batch rows that have stopped are not read any further ------------
+namespace {
+struct EarlyExitLayout {
+    int first;                       // positions of the first phase
+    size_t ws1, ws1_bytes, ws2, ws2_bytes, rows, n_alive, total;
+};
+
+bool early_exit_layout(int B, int K, int V, csd_dtype_t dtype, int first, EarlyExitLayout &l)
+{
+    if (!shape_ok(B, K, V, dtype) || K < 2) return false;
+    if (first <= 0) first = (K + 1) / 3 > 1 ? (K + 1) / 3 : 1;
+    if (first >= K) first = K - 1;
+    l.first = first;
+    Shape s1 = pick_shape(B, first, V, dtype, false);
+    Shape s2 = pick_shape(B, K - first, V, dtype, false);
+    s2.slots_per_row = s2.units_per_row < kListSlotsPerRow ? s2.units_per_row : kListSlotsPerRow;
+    l.ws1 = 0;
+    l.ws1_bytes = ws_layout(B, first, s1).total;
+    l.ws2 = align_up(l.ws1_bytes, 256);
+    l.ws2_bytes = ws_layout(B, K - first, s2).total;
+    l.rows = align_up(l.ws2 + l.ws2_bytes, 256);
+    l.n_alive = align_up(l.rows + static_cast<size_t>(B) * sizeof(int), 16);
+    l.total = align_up(l.n_alive + 16, 256);
+    return true;
+}
+}  // namespace
+
+size_t csd_early_exit_workspace_bytes(int B, int K, int V, csd_dtype_t dtype, int first_phase_positions)
+{
+    EarlyExitLayout l;
+    return early_exit_layout(B, K, V, dtype, first_phase_positions, l) ? l.total : 0;
+}
+
+csd_status_t csd_step_early_exit(const void *logits, csd_dtype_t dtype, int B, int K, int V, int64_t stride_b, int64_t stride_k,
+                                 const int32_t *draft, csd_ocm_t *ocm, float tau, int first_phase_positions, int32_t *accept_len,
+                                 int32_t *next_token, uint8_t *rescued_mask, int32_t *rej_draft, int32_t *rej_target,
+                                 const csd_diag_t *diag, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (B <= 0 || K <= 0 || V <= 0 || (dtype != CSD_F32 && dtype != CSD_BF16)) return CSD_ERR_INVALID_ARG;
+    if (K > CSD_MAX_K) return CSD_ERR_UNSUPPORTED;
+    if (K < 2) return CSD_ERR_UNSUPPORTED;
+    if (!workspace) return CSD_ERR_INVALID_ARG;
+    EarlyExitLayout l;
+    if (!early_exit_layout(B, K, V, dtype, first_phase_positions, l)) return CSD_ERR_UNSUPPORTED;
+    if (workspace_bytes < l.total || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
+    chain_break();
+    char *ws = static_cast<char *>(workspace);
+    int *rows = reinterpret_cast<int *>(ws + l.rows);
+    int *n_alive = reinterpret_cast<int *>(ws + l.n_alive);
+    PhaseSpec first = {K, 0, nullptr, nullptr, rows, n_alive, K, 1};
+    csd_status_t rc = run_step(logits, dtype, B, l.first, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
+                               rej_draft, rej_target, diag, ws + l.ws1, l.ws1_bytes, stream, false, false, false, true, &first);
+    if (rc != CSD_OK) return rc;
+    PhaseSpec second = {K, l.first, rows, n_alive, nullptr, nullptr, 0, 0};
+    rc = run_step(logits, dtype, B, K - l.first, V, stride_b, stride_k, draft, ocm, tau, accept_len, next_token, rescued_mask,
+                  rej_draft, rej_target, diag, ws + l.ws2, l.ws2_bytes, stream, false, false, false, true, &second);
+    if (rc != CSD_OK) return rc;
+    return run_update(ocm, rej_draft, rej_target, nullptr, static_cast<int64_t>(B) * K, stream);
 }
 
 size_t csd_workspace_bytes(int B, int K, int V, csd_dtype_t dtype)

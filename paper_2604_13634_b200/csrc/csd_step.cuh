@@ -93,7 +93,51 @@ struct StepParams {
     int narrow;              // 1 if the span arithmetic fits 32 bits
     int chain_by_flag;       // 1 if the host vouches that the previous step launch on the stream used this
                              // very workspace, memory and outputs: its completion word is then enough
+    // ---- a launch that covers only some positions of some batch rows (the two phases of the early-exit step) ----
+    // K_total = 0: an ordinary step (the fields below are unused).  Otherwise this launch verifies positions
+    // pos0 .. pos0 + K - 1 of a step with K_total positions: logit rows pos0 .. pos0 + K, draft / output / diagnostic
+    // arrays laid out for K_total; its batch rows are row_map[0 .. *n_rows) if row_map is set, else 0 .. B - 1.
+    int K_total, pos0;
+    const int *row_map;      // virtual batch row -> batch row of the step
+    const int *n_rows;       // device word: how many virtual batch rows there are (at most B)
+    int min_units;           // least 512-byte units per block when the grid is re-derived on the device
+    int *alive_out;          // if set: the batch rows that accepted all K positions of this launch, ascending ...
+    int *n_alive_out;        // ... and how many they are (written by the launch's last warp)
+    int count_positions;     // what a finalised batch row adds to the statistics' position count
+    int count_step;          // whether the launch counts as a step in the statistics
 };
+
+// What a launch works on: ordinary launches take it from the parameters, a launch over a row list from the device.
+struct Extent {
+    int B;                   // batch rows
+    int G;                   // blocks that own a span
+    long long T;             // units in all
+};
+
+// Where batch row b of the launch lives in the step's arrays.
+struct RowPlace {
+    long long br;            // batch row of the step
+    size_t pos;              // index of its first position in [B, K_total] arrays
+    size_t row;              // index of its first logit row in [B, K_total + 1] arrays
+    int i0;                  // first logit row within the batch row
+};
+
+__device__ __forceinline__ RowPlace place_of(const StepParams &p, long long b)
+{
+    RowPlace r;
+    if (p.K_total == 0) {
+        r.br = b;
+        r.pos = static_cast<size_t>(b) * p.K;
+        r.row = static_cast<size_t>(b) * (p.K + 1);
+        r.i0 = 0;
+    } else {
+        r.br = p.row_map ? __ldg(p.row_map + b) : b;
+        r.pos = static_cast<size_t>(r.br) * p.K_total + p.pos0;
+        r.row = static_cast<size_t>(r.br) * (p.K_total + 1) + p.pos0;
+        r.i0 = p.pos0;
+    }
+    return r;
+}
 
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -403,20 +447,20 @@ __device__ __forceinline__ Partial warp_tile(const typename L::elem *row, int e0
 
 // ---- the even split of the unit space over blocks -----------------------------------------
 
-__device__ __forceinline__ long long span_begin(const StepParams &p, int c)
+__device__ __forceinline__ long long span_begin(const StepParams &p, const Extent &e, int c)
 {
     if (p.narrow)   // (T + 1) * (G + 1) < 2^32: 32-bit division is several times cheaper
-        return static_cast<unsigned int>(c) * static_cast<unsigned int>(p.total_units) / static_cast<unsigned int>(p.n_spans);
-    return static_cast<long long>(c) * p.total_units / p.n_spans;
+        return static_cast<unsigned int>(c) * static_cast<unsigned int>(e.T) / static_cast<unsigned int>(e.G);
+    return static_cast<long long>(c) * e.T / e.G;
 }
 
 // The block whose span holds global unit g: the largest c with span_begin(c) <= g.
-__device__ __forceinline__ int owner_of(const StepParams &p, long long g)
+__device__ __forceinline__ int owner_of(const StepParams &p, const Extent &e, long long g)
 {
     if (p.narrow)
-        return static_cast<int>(((static_cast<unsigned int>(g) + 1u) * static_cast<unsigned int>(p.n_spans) - 1u) /
-                                static_cast<unsigned int>(p.total_units));
-    return static_cast<int>(((g + 1) * p.n_spans - 1) / p.total_units);
+        return static_cast<int>(((static_cast<unsigned int>(g) + 1u) * static_cast<unsigned int>(e.G) - 1u) /
+                                static_cast<unsigned int>(e.T));
+    return static_cast<int>(((g + 1) * e.G - 1) / e.T);
 }
 
 constexpr int kFinalizeWarps = 8;  // warps of a block that share its batch rows to finalise
@@ -488,7 +532,7 @@ __device__ __forceinline__ Partial butterfly_fold(Partial v, int width, const fl
 // Fold the per-block partials of the K+1 logit rows of batch row b (S1, last level).  The
 // lanes are arranged as (32 / width) rows x width slots, width = the power of two >= the
 // slots per row (at most 32; more slots are pre-folded in lane order).
-__device__ __forceinline__ void fold_rows(const StepParams &p, const ScratchCopy &sc, int b, int lane, RowScratch &rs)
+__device__ __forceinline__ void fold_rows(const StepParams &p, const Extent &e, const ScratchCopy &sc, int b, int lane, RowScratch &rs)
 {
     const int K1 = p.K + 1, S = p.slots_per_row;
     int width = 1;
@@ -501,7 +545,7 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, const ScratchCopy
 
     for (int r = lane; r < K1; r += 32) {
         const long long u0 = static_cast<long long>(row0 + r) * p.units_per_row;
-        rs.parts[r] = owner_of(p, u0 + p.units_per_row - 1) - owner_of(p, u0) + 1;
+        rs.parts[r] = owner_of(p, e, u0 + p.units_per_row - 1) - owner_of(p, e, u0) + 1;
     }
     __syncwarp();
 
@@ -537,18 +581,22 @@ __device__ __forceinline__ void fold_rows(const StepParams &p, const ScratchCopy
     __syncwarp();
 }
 
+// Logit row i (within the launch) of batch row b (of the launch).
 template <typename L>
 __device__ __forceinline__ const typename L::elem *logit_row(const StepParams &p, long long b, int i)
 {
-    return reinterpret_cast<const typename L::elem *>(p.logits) + b * p.stride_b + static_cast<long long>(i) * p.stride_k;
+    const RowPlace at = place_of(p, b);
+    return reinterpret_cast<const typename L::elem *>(p.logits) + at.br * p.stride_b + static_cast<long long>(at.i0 + i) * p.stride_k;
 }
 
 __device__ __forceinline__ void prefetch_l2(const void *ptr) { asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr)); }
 
 template <typename L>
-__device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, int lane, RowScratch &rs, const BlockState &bs)
+__device__ int finalize_batch_row(const StepParams &p, const Extent &e, unsigned int seq, int b, int lane, RowScratch &rs,
+                                  const BlockState &bs)
 {
     const int K = p.K;
+    const RowPlace at_b = place_of(p, b);
 
     // S2 (first half): the draft tokens and their logits do not depend on the reduction: the tokens were
     // fetched when the block started (else they are loaded now), the logits' loads are issued before the
@@ -556,11 +604,11 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
     int d = -1;
     float zd = __int_as_float(0x7fc00000);
     const int pre = bs.pre_b[0] == b ? 0 : (bs.pre_b[1] == b ? 1 : -1);
-    if (lane < K) d = pre >= 0 ? bs.pre_d[pre][lane] : __ldg(p.draft + (size_t)b * K + lane);
+    if (lane < K) d = pre >= 0 ? bs.pre_d[pre][lane] : __ldg(p.draft + at_b.pos + lane);
     const bool valid = lane < K && static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V);
     if (valid) zd = L::load_elem(logit_row<L>(p, b, lane), d);
     const ScratchCopy sc = scratch_of(p, seq);
-    fold_rows(p, sc, b, lane, rs);
+    fold_rows(p, e, sc, b, lane, rs);
 
     // Everything above read only this launch's inputs and its own copy of the scratch.
     // From here on the previous launch must be complete: the memory, its statistics and
@@ -579,7 +627,7 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
         if (valid) cnt = ocm_lookup(p.ocm, make_key(d, t), &slot, &empty_slot);
     }
     for (int row = lane; row <= K; row += 32) {
-        const size_t at = (size_t)b * (K + 1) + row;
+        const size_t at = at_b.row + row;
         const float s_m = rs.s[row];
         if (!(s_m == s_m) || s_m == INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
         if (p.diag.m) p.diag.m[at] = rs.m[row];
@@ -595,7 +643,7 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
         const bool is_freq = cnt >= p.ocm.lambda;
         const bool is_safe = (static_cast<double>(zd) - static_cast<double>(m)) >= static_cast<double>(p.log_tau);  // S4, Eq. 3
         ok = match || (valid && is_freq && is_safe);
-        const size_t pos = (size_t)b * K + lane;
+        const size_t pos = at_b.pos + lane;
         if (p.diag.zd) p.diag.zd[pos] = zd;
         if (p.diag.cnt) p.diag.cnt[pos] = cnt;
         if (p.diag.score || p.diag.p_d) {
@@ -612,7 +660,7 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
     const bool reached = lane <= n_acc && lane < K;
     const bool record = reached && !match && valid;
     if (lane < K) {
-        const size_t pos = (size_t)b * K + lane;
+        const size_t pos = at_b.pos + lane;
         p.rescued[pos] = (lane < n_acc && !match) ? 1 : 0;
         p.rej_d[pos] = record ? d : -1;
         p.rej_t[pos] = record ? t : -1;
@@ -626,18 +674,25 @@ __device__ int finalize_batch_row(const StepParams &p, unsigned int seq, int b, 
                 const unsigned int room = 0xffffffffu - static_cast<unsigned int>(p.B * p.K);
                 if (slot >= 0 && cnt > room) hint |= kHintCareful;
             }
-            __stcg(sc.slot_hint + pos, hint);
+            __stcg(sc.slot_hint + (size_t)b * K + lane, hint);
         }
+    } else if (p.K_total != 0 && p.pos0 == 0 && lane < p.K_total) {
+        // first phase of a step in two phases: the positions it does not cover start out as "not reached"
+        const size_t pos = at_b.pos + lane;
+        p.rescued[pos] = 0;
+        p.rej_d[pos] = -1;
+        p.rej_t[pos] = -1;
     }
     const unsigned int m_match = __ballot_sync(kFull, reached && match);
     const unsigned int m_resc = __ballot_sync(kFull, lane < n_acc && !match && lane < K);
     const unsigned int m_rec = __ballot_sync(kFull, record);
     const unsigned int m_bad = __ballot_sync(kFull, lane < K && !valid);
     if (lane == 0) {
-        p.accept_len[b] = n_acc;
-        p.next_token[b] = rs.t[n_acc];
+        p.accept_len[at_b.br] = at_b.i0 + n_acc;
+        p.next_token[at_b.br] = rs.t[n_acc];
         OcmStatsDev *st = p.ocm.stats;
-        atomicAdd(&st->positions, static_cast<unsigned long long>(K));
+        const int counted = p.K_total != 0 ? p.count_positions : K;
+        if (counted) atomicAdd(&st->positions, static_cast<unsigned long long>(counted));
         if (m_match) atomicAdd(&st->matches, static_cast<unsigned long long>(__popc(m_match)));
         if (m_resc) atomicAdd(&st->rescues, static_cast<unsigned long long>(__popc(m_resc)));
         if (m_rec) atomicAdd(&st->rejections, static_cast<unsigned long long>(__popc(m_rec)));
@@ -689,7 +744,7 @@ __device__ void apply_step_update(const StepParams &p, const ScratchCopy &sc, in
 // delivered are left in bs.todo_b for the block's warps to finalise.
 //   nseg row parts, rows first_row .. first_row + nseg - 1, results in bs.seg_result;
 //   next_b: batch row of the next row this block will still publish, or -1.
-__device__ void publish_parts(const StepParams &p, BlockState &bs, int first_row, int nseg, int next_b, int lane)
+__device__ void publish_parts(const StepParams &p, const Extent &e, BlockState &bs, int first_row, int nseg, int next_b, int lane)
 {
     const int K1 = p.K + 1;
     const int U = p.units_per_row;
@@ -703,9 +758,9 @@ __device__ void publish_parts(const StepParams &p, BlockState &bs, int first_row
     int my_b = -1;
     if (lane < nseg) {
         const int row = first_row + lane;
-        const int slot = static_cast<int>(blockIdx.x) - owner_of(p, static_cast<long long>(row) * U);
+        const int slot = static_cast<int>(blockIdx.x) - owner_of(p, e, static_cast<long long>(row) * U);
         // the host sized slots_per_row from the same split: a slot beyond it would be a bug, and is reported
-        if (CSD_CHECKED(slot >= 0 && slot < p.slots_per_row && row < p.B * K1, p.ocm.stats, 1u))
+        if (CSD_CHECKED(slot >= 0 && slot < p.slots_per_row && row < e.B * K1, p.ocm.stats, 1u))
             st_partial_cg(sc.partials + (size_t)row * p.slots_per_row + slot, bs.seg_result[lane]);
         my_b = row / K1;
     }
@@ -717,28 +772,28 @@ __device__ void publish_parts(const StepParams &p, BlockState &bs, int first_row
         const bool closes = (lane == nseg - 1) ? (my_b != next_b) : (below_b != my_b);
         if (closes) {
             const long long u0 = static_cast<long long>(my_b) * K1 * U;
-            const unsigned int expected = owner_of(p, u0 + static_cast<long long>(K1) * U - 1) - owner_of(p, u0) + 1;
+            const unsigned int expected = owner_of(p, e, u0 + static_cast<long long>(K1) * U - 1) - owner_of(p, e, u0) + 1;
             // the last arrival has acquired the other blocks' partials of the row; this block's warps read
             // them after the block barrier that follows
             completes = atom_add_acq_rel(sc.b_ticket + my_b, 1u) == expected - 1;
         }
     }
     const unsigned int todo = __ballot_sync(kFull, completes);
-    if (completes && CSD_INDEX_OK(my_b >= 0 && my_b < p.B, p.ocm.stats, 2u)) bs.todo_b[__popc(todo & ((1u << lane) - 1u))] = my_b;
+    if (completes && CSD_INDEX_OK(my_b >= 0 && my_b < e.B, p.ocm.stats, 2u)) bs.todo_b[__popc(todo & ((1u << lane) - 1u))] = my_b;
     if (lane == 0) bs.n_todo = __popc(todo);
 }
 
 // S2..S5 of batch row b by one warp, and, if that was the launch's last row, S6.
 template <typename L>
-__device__ void finalize_and_update(const StepParams &p, unsigned int seq, int b, int lane, RowScratch &rs, CanonScratch &canon,
-                                    const BlockState &bs)
+__device__ void finalize_and_update(const StepParams &p, const Extent &e, unsigned int seq, int b, int lane, RowScratch &rs,
+                                    CanonScratch &canon, const BlockState &bs)
 {
     const ScratchCopy sc = scratch_of(p, seq);
-    const int regime = finalize_batch_row<L>(p, seq, b, lane, rs, bs);   // the same for every row of a launch
+    const int regime = finalize_batch_row<L>(p, e, seq, b, lane, rs, bs);   // the same for every row of a launch
     bool last = false;
     if (lane == 0) sc.b_ticket[b] = 0u;               // ready for this copy's next launch
     __syncwarp();                                     // each lane's outputs and hints of this row before the row's ticket,
-    if (lane == 0) last = atom_add_acq_rel(sc.g_ticket, 1u) == static_cast<unsigned int>(p.B) - 1u;   // whose add releases them
+    if (lane == 0) last = atom_add_acq_rel(sc.g_ticket, 1u) == static_cast<unsigned int>(e.B) - 1u;   // whose add releases them
     last = __shfl_sync(kFull, last, 0);
     if (!last) return;
 
@@ -751,13 +806,30 @@ __device__ void finalize_and_update(const StepParams &p, unsigned int seq, int b
     unsigned long long nk = 0;
     if (lane == 0 && keys_settled) nk = atomicAdd(&st->n_keys, 0ull);   // in flight next to the hint loads
     if (p.do_update) apply_step_update(p, sc, lane, canon, regime);
+    if (p.K_total != 0 && p.alive_out) {
+        // the batch rows that accepted every position of this launch go on to the next phase: their list, ascending
+        int n_alive = 0;
+        for (int b0 = 0; b0 < e.B; b0 += 32) {
+            const int bb = b0 + lane;
+            bool alive = false;
+            long long br = 0;
+            if (bb < e.B) {
+                br = p.row_map ? __ldcg(p.row_map + bb) : bb;
+                alive = __ldcg(p.accept_len + br) == p.pos0 + p.K;
+            }
+            const unsigned int mask = __ballot_sync(kFull, alive);
+            if (alive) p.alive_out[n_alive + __popc(mask & ((1u << lane) - 1u))] = static_cast<int>(br);
+            n_alive += __popc(mask);
+        }
+        if (lane == 0) *p.n_alive_out = n_alive;
+    }
     if (lane == 0) {
         if (!keys_settled) {
             fence_acq_rel();
             nk = atomicAdd(&st->n_keys, 0ull);
         }
         st->n_keys_start = nk;
-        atomicAdd(&st->steps, 1ull);
+        if (p.K_total == 0 || p.count_step) atomicAdd(&st->steps, 1ull);
         *sc.g_ticket = 0u;
         st_release(p.completed, seq + 1u);            // everything above, and all it observed, first
     }
@@ -792,8 +864,26 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
     const int U = p.units_per_row;
     const int CH = p.chunk_units;
     const int cpr = (U + CH - 1) / CH;                       // chunks of a whole row
-    long long g = span_begin(p, blockIdx.x);
-    const long long g_end = span_begin(p, blockIdx.x + 1);
+    Extent e;
+    e.B = p.B;
+    e.G = p.n_spans;
+    e.T = p.total_units;
+    if (p.K_total != 0 && p.n_rows) {
+        // a launch over a list of batch rows that an earlier launch wrote: the extent comes from the device, and the
+        // blocks that share the work are re-derived from it by the host's rules (at most 64 per logit row, at least
+        // min_units units each)
+        e.B = __ldcg(p.n_rows);
+        const long long rows = static_cast<long long>(e.B) * K1;
+        e.T = rows * U;
+        long long blocks = gridDim.x;
+        if (blocks > rows * 64) blocks = rows * 64;
+        const long long most = (e.T + p.min_units - 1) / p.min_units;
+        if (blocks > most) blocks = most;
+        e.G = static_cast<int>(blocks);
+    }
+    const bool idle = static_cast<int>(blockIdx.x) >= e.G;    // only possible for a launch over a row list
+    long long g = idle ? 0 : span_begin(p, e, blockIdx.x);
+    const long long g_end = idle ? 0 : span_begin(p, e, blockIdx.x + 1);
     // quotients of unit and row indices: 32-bit division where the host found that everything fits
     auto quot = [&](long long a, int b) -> long long {
         return p.narrow ? static_cast<long long>(static_cast<unsigned int>(a) / static_cast<unsigned int>(b)) : a / b;
@@ -838,13 +928,13 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             const long long row = row0 + at.seg;
             const long long b = quot(row, K1);
             const int i = static_cast<int>(row - b * K1);
-            const E *rp = reinterpret_cast<const E *>(p.logits) + b * p.stride_b + i * p.stride_k;
+            const E *rp = logit_row<L>(p, b, i);
             const int u0 = ua + k * CH;
             const int u1 = min(ub, u0 + CH);
             const int e0 = u0 * p.unit_elems;
             const long long e1l = static_cast<long long>(u1) * p.unit_elems;
             const int e1 = e1l < p.V ? static_cast<int>(e1l) : p.V;
-            at.ok = CSD_INDEX_OK(row < static_cast<long long>(p.B) * K1 && at.seg >= 0 && at.seg < nseg && nseg <= kMaxSegs &&
+            at.ok = CSD_INDEX_OK(row < static_cast<long long>(e.B) * K1 && at.seg >= 0 && at.seg < nseg && nseg <= kMaxSegs &&
                                      q < static_cast<unsigned int>(kMaxChunks) && e0 >= 0 && e0 < e1 &&
                                      at.seg_first + at.seg_n <= kMaxChunks,
                                  p.ocm.stats, 5u);
@@ -876,7 +966,7 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             }
             if (!__shfl_sync(kFull, block_complete, 0)) return;
             __threadfence_block();
-            publish_parts(p, bs, static_cast<int>(row0), nseg, next_b, lane);
+            publish_parts(p, e, bs, static_cast<int>(row0), nseg, next_b, lane);
         };
 
         // The shared tables of the window.  In the block's first window nothing waits for them yet: every warp
@@ -903,8 +993,8 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
             const bool two = quot(row0 + nseg - 1, K1) > fb;
             int d0 = -1, d1 = -1;
             if (lane < p.K) {
-                d0 = __ldg(p.draft + (size_t)fb * p.K + lane);
-                if (two) d1 = __ldg(p.draft + (size_t)(fb + 1) * p.K + lane);
+                d0 = __ldg(p.draft + place_of(p, fb).pos + lane);
+                if (two) d1 = __ldg(p.draft + place_of(p, fb + 1).pos + lane);
             }
             if (lane == 0)
                 bs.seq = (seq_old >> 32) == 0ull ? static_cast<unsigned int>(seq_old) / gridDim.x
@@ -953,7 +1043,7 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
                     }
                     if (__shfl_sync(kFull, block_complete, 0)) {   // everything else was already folded
                         __threadfence_block();
-                        publish_parts(p, bs, static_cast<int>(row0), nseg, next_b, lane);
+                        publish_parts(p, e, bs, static_cast<int>(row0), nseg, next_b, lane);
                     }
                 }
             }
@@ -965,7 +1055,7 @@ __global__ void __launch_bounds__(1024) csd_step_kernel(const __grid_constant__ 
         const int fin_warps = nwarps < kFinalizeWarps ? nwarps : kFinalizeWarps;
         if (warp < fin_warps && CSD_INDEX_OK(bs.n_todo >= 0 && bs.n_todo <= kMaxSegs, p.ocm.stats, 6u))
             for (int j = warp; j < bs.n_todo; j += fin_warps)
-                finalize_and_update<L>(p, bs.seq, bs.todo_b[j], lane, row_scratch[warp], canon, bs);
+                finalize_and_update<L>(p, e, bs.seq, bs.todo_b[j], lane, row_scratch[warp], canon, bs);
         g = w_end;
         if (g < g_end) __syncthreads();       // the next window reuses the shared-memory tables
     }
