@@ -354,7 +354,8 @@ csd_status_t csd_step_sampled(const void *logits, const void *draft_logits, csd_
  * the [B, K+1, V] logit tensor is neither written nor read; everything after that is csd_verify / csd_step.
  *
  * hidden : [B, K+1, H] bf16, dense, 16-byte aligned.   weight : [V, H] bf16, dense, 16-byte aligned.
- * Shapes: H a multiple of 64; B*(K+1) <= 256 (larger batches: split the batch); any V.
+ * Shapes: H a multiple of 64; any B, K <= 32, V.  Logit rows are processed in groups of 256, and the weight
+ * matrix is streamed once per group: up to 256 rows the step is bound by that stream, beyond by the contraction.
  * The logits are the fp32 tensor-core accumulations of the exact bf16 products, NOT rounded to bf16: they
  * differ from an exactly summed product by at most about 2^-16 * ||hidden row|| * max ||weight row|| (see
  * the tests), so an arg-max or a gate decision that hangs on a smaller difference may come out either way;
@@ -362,7 +363,7 @@ csd_status_t csd_step_sampled(const void *logits, const void *draft_logits, csd_
  * workspace: csd_lmhead_workspace_bytes bytes, 16-byte aligned, no initialisation needed.
  * Three launches (GEMM + statistics, decisions, memory update); asynchronous.  A wait inside the GEMM
  * kernel that does not end within about two seconds raises CSD_FLAG_INTERNAL (debug_site 30).
- * Errors as csd_verify; UNSUPPORTED for shapes outside the limits above; CUDA if the driver offers no
+ * Errors as csd_verify; UNSUPPORTED for H not a multiple of 64; CUDA if the driver offers no
  * tensor-map encoder. */
 size_t csd_lmhead_workspace_bytes(int B, int K, int H, int V);
 csd_status_t csd_verify_lmhead(const void *hidden, const void *weight, int B, int K, int H, int V,
@@ -378,6 +379,10 @@ csd_status_t csd_step_lmhead(const void *hidden, const void *weight, int B, int 
 /* How the vocabulary is cut for this shape: blocks of the GEMM grid, columns per tile, number of tiles and
  * tiles per block.  Host function; for reports and tests. */
 csd_status_t csd_lmhead_shape(int B, int K, int H, int V, int *grid, int *tile_cols, int *tiles, int *tiles_per_block);
+/* Expert knob, process-wide: how many 64-column k-blocks travel through the shared-memory ring together
+ * (1 to 4; 0 = automatic).  More per stage means longer contiguous reads of each weight row and fewer, larger
+ * stages.  Results do not depend on it beyond the rounding order of the accumulation.  Host function. */
+csd_status_t csd_lmhead_set_tuning(int kblocks_per_stage);
 
 /* csd_step for callers whose tensors live in HOST memory (pinned memory gives
  * the full copy rate).  Copies logits and draft to `staging`, runs the step, and

@@ -30,7 +30,7 @@ EXPORTS = [
     "csd_sampled_workspace_bytes", "csd_verify_sampled", "csd_step_sampled",
     "csd_ocm_age", "csd_ocm_merge", "csd_ocm_save", "csd_ocm_load", "csd_ocm_set_shared",
     "csd_lmhead_workspace_bytes", "csd_verify_lmhead", "csd_step_lmhead", "csd_lmhead_shape",
-    "csd_early_exit_workspace_bytes", "csd_step_early_exit",
+    "csd_early_exit_workspace_bytes", "csd_step_early_exit", "csd_lmhead_set_tuning",
 ]
 
 
@@ -101,6 +101,7 @@ def lib():
         "csd_lmhead_shape": (c_int, [c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
         "csd_early_exit_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int, c_int]),
         "csd_step_early_exit": (c_int, step_args[:10] + [c_int] + step_args[10:]),
+        "csd_lmhead_set_tuning": (c_int, [c_int]),
         "csd_ocm_age": (c_int, [c_void_p, c_void_p]),
         "csd_ocm_set_shared": (c_int, [c_void_p, c_int]),
         "csd_ocm_merge": (c_int, [c_void_p, c_void_p, c_void_p]),
@@ -427,7 +428,7 @@ class LmheadBuffers(StepBuffers):
         self.H = H
         bytes_ = int(lib().csd_lmhead_workspace_bytes(B, K, H, V))
         if bytes_ == 0:
-            raise CsdError(f"unsupported shape B={B} K={K} H={H} V={V} (H % 64 == 0 and B*(K+1) <= 256 are required)")
+            raise CsdError(f"unsupported shape B={B} K={K} H={H} V={V} (H % 64 == 0 is required)")
         super().__init__(B, K, V, torch.bfloat16, device=device, diag=diag)
         self.ws_bytes = bytes_
         self.workspace = torch.empty(bytes_, dtype=torch.uint8, device=torch.device(device))
@@ -485,3 +486,7 @@ def csd_step_early_exit(logits, draft, ocm: Ocm, tau: float, buf: EarlyExitBuffe
         _ptr(buf.rej_target), byref(buf._diag_struct) if buf._diag_struct is not None else None, _ptr(buf.workspace),
         buf.ws_bytes, _stream_ptr(stream))
     _check(rc, "csd_step_early_exit")
+
+
+def csd_lmhead_set_tuning(kblocks_per_stage: int = 0):
+    _check(lib().csd_lmhead_set_tuning(kblocks_per_stage), "csd_lmhead_set_tuning")

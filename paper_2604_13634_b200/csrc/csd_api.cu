@@ -862,7 +862,7 @@ namespace {
 
 struct LmheadPlan {
     int grid, n_tile, tiles_total, tiles_per_cta;
-    int rows2, a_bytes, stage_bytes, n_stages, smem_bytes;
+    int rows2, a_bytes, sub_bytes, kps, n_stages, smem_bytes;
     size_t partials_off, zd_off, total;
 };
 
@@ -870,12 +870,14 @@ bool lmhead_shape_ok(int B, int K, int H, int V)
 {
     if (!(B > 0 && K > 0 && K <= CSD_MAX_K && V > 0 && H > 0)) return false;
     if (H % lmhead::kBlockK != 0) return false;
-    return static_cast<long long>(B) * (K + 1) <= lmhead::kRowsMax;
+    return static_cast<long long>(B) * (K + 1) <= (1ll << 20) && static_cast<long long>(V) < (1ll << 30);
 }
+
+int g_lmhead_kblocks_per_stage = 0;   // 0 = automatic
 
 // The vocabulary is cut into tiles of n_tile columns (a multiple of 16, at most 256) such that every CTA of a
 // one-per-SM grid owns the same number of consecutive tiles.
-LmheadPlan lmhead_plan(int B, int K, int V)
+LmheadPlan lmhead_plan(int B, int K, int H, int V)
 {
     LmheadPlan pl;
     const long long sms = sm_count();
@@ -892,13 +894,18 @@ LmheadPlan lmhead_plan(int B, int K, int V)
     pl.grid = static_cast<int>(grid < 1 ? 1 : grid);
     const size_t rows = static_cast<size_t>(B) * (K + 1);
     // shared-memory ring: as many stages as fit beside the barriers, the alignment room and the slack
-    pl.rows2 = rows > lmhead::kMTile ? static_cast<int>((rows - lmhead::kMTile + 7) / 8 * 8) : 0;
-    pl.a_bytes = static_cast<int>(align_up(static_cast<size_t>(lmhead::kMTile + pl.rows2) * lmhead::kRowBytes, 1024));
-    pl.stage_bytes = pl.a_bytes + static_cast<int>(align_up(static_cast<size_t>(pl.n_tile) * lmhead::kRowBytes, 1024));
+    const size_t groups = (rows + lmhead::kRowsMax - 1) / lmhead::kRowsMax;
+    const size_t rows_last = rows - (groups - 1) * lmhead::kRowsMax;
+    pl.rows2 = rows_last > lmhead::kMTile ? static_cast<int>((rows_last - lmhead::kMTile + 7) / 8 * 8) : 0;
+    const int rows2_most = groups > 1 ? lmhead::kMTile : pl.rows2;
+    pl.a_bytes = static_cast<int>(align_up(static_cast<size_t>(lmhead::kMTile + rows2_most) * lmhead::kRowBytes, 1024));
+    pl.sub_bytes = pl.a_bytes + static_cast<int>(align_up(static_cast<size_t>(pl.n_tile) * lmhead::kRowBytes, 1024));
     const int fixed = 1024 + lmhead::kBarrierBytes + lmhead::kSlackBytes;
-    int stages = (lmhead::kSmemLimit - fixed) / pl.stage_bytes;
+    pl.kps = g_lmhead_kblocks_per_stage > 0 ? g_lmhead_kblocks_per_stage : 1;
+    while (pl.kps > 1 && (H % (lmhead::kBlockK * pl.kps) != 0 || (lmhead::kSmemLimit - fixed) / (pl.kps * pl.sub_bytes) < 2)) --pl.kps;
+    int stages = (lmhead::kSmemLimit - fixed) / (pl.kps * pl.sub_bytes);
     pl.n_stages = stages > lmhead::kMaxStages ? lmhead::kMaxStages : stages;
-    pl.smem_bytes = fixed + pl.n_stages * pl.stage_bytes;
+    pl.smem_bytes = fixed + pl.n_stages * pl.kps * pl.sub_bytes;
     pl.partials_off = 0;
     pl.zd_off = align_up(rows * pl.grid * sizeof(Partial), 256);
     pl.total = align_up(pl.zd_off + static_cast<size_t>(B) * K * sizeof(float), 256);
@@ -953,7 +960,7 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     if (!(tau >= 0.0f) || std::isinf(tau)) return CSD_ERR_INVALID_ARG;
     if (!lmhead_shape_ok(B, K, H, V)) return CSD_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(weight) & 15u)) return CSD_ERR_INVALID_ARG;
-    const LmheadPlan pl = lmhead_plan(B, K, V);
+    const LmheadPlan pl = lmhead_plan(B, K, H, V);
     if (workspace_bytes < pl.total || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
     chain_break();
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -992,7 +999,8 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     p.tiles_per_cta = pl.tiles_per_cta;
     p.rows2 = pl.rows2;
     p.a_bytes = pl.a_bytes;
-    p.stage_bytes = pl.stage_bytes;
+    p.sub_bytes = pl.sub_bytes;
+    p.kblocks_per_stage = pl.kps;
     p.n_stages = pl.n_stages;
     p.draft = draft;
     p.partials = reinterpret_cast<Partial *>(ws + pl.partials_off);
@@ -1012,9 +1020,23 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     f.accept_len = accept_len; f.next_token = next_token; f.rescued = rescued_mask;
     f.rej_d = rej_draft; f.rej_t = rej_target;
     if (diag) f.diag = *diag;
-    lmhead::lmhead_finalize_kernel<<<(B + 3) / 4, 128, 0, st>>>(f);
-    if (cudaGetLastError() != cudaSuccess) return CSD_ERR_CUDA;
-    if (do_update) return run_update(ocm, rej_draft, rej_target, nullptr, static_cast<int64_t>(B) * K, stream);
+    {
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(static_cast<unsigned int>((B + 3) / 4));
+        cfg.blockDim = dim3(128);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, lmhead::lmhead_finalize_kernel, f) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CSD_ERR_CUDA;
+        }
+    }
+    if (do_update) return run_update(ocm, rej_draft, rej_target, nullptr, static_cast<int64_t>(B) * K, stream, true);
     return CSD_OK;
 }
 
@@ -1023,7 +1045,7 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
 size_t csd_lmhead_workspace_bytes(int B, int K, int H, int V)
 {
     if (!lmhead_shape_ok(B, K, H, V)) return 0;
-    return lmhead_plan(B, K, V).total;
+    return lmhead_plan(B, K, H, V).total;
 }
 
 csd_status_t csd_verify_lmhead(const void *hidden, const void *weight, int B, int K, int H, int V, const int32_t *draft,
@@ -1043,10 +1065,17 @@ csd_status_t csd_step_lmhead(const void *hidden, const void *weight, int B, int 
                       diag, workspace, workspace_bytes, stream, true);
 }
 
+csd_status_t csd_lmhead_set_tuning(int kblocks_per_stage)
+{
+    if (kblocks_per_stage < 0 || kblocks_per_stage > 4) return CSD_ERR_INVALID_ARG;
+    g_lmhead_kblocks_per_stage = kblocks_per_stage;
+    return CSD_OK;
+}
+
 csd_status_t csd_lmhead_shape(int B, int K, int H, int V, int *grid, int *tile_cols, int *tiles, int *tiles_per_block)
 {
     if (!lmhead_shape_ok(B, K, H, V)) return CSD_ERR_UNSUPPORTED;
-    const LmheadPlan pl = lmhead_plan(B, K, V);
+    const LmheadPlan pl = lmhead_plan(B, K, H, V);
     if (grid) *grid = pl.grid;
     if (tile_cols) *tile_cols = pl.n_tile;
     if (tiles) *tiles = pl.tiles_total;

@@ -3,17 +3,18 @@
 // statistics of S1 (maximum, lowest arg-max, sum of exponentials) and picks out the draft tokens' logits, so
 // the [rows, V] logit tensor never reaches HBM.
 //
-//   lmhead_stats_kernel     persistent, one CTA per SM, 192 threads:
+//   lmhead_stats_kernel     persistent, one CTA per SM, 320 threads:
 //       warp 0      one thread issues the TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of the k-blocks:
 //                   64 columns of all hidden rows (a box of 128 rows and one of the rows beyond) and of the
 //                   vocabulary tile's W rows, into a ring of as many shared-memory stages as fit (3 to 8)
 //       warp 1      one thread issues the MMAs (tcgen05.mma, kind::f16, M = 128, N = tile width, K = 16, fp32
 //                   accumulators in tensor memory: columns [0, N) for rows 0..127, [256, 256 + N) for rows
 //                   128..255) and commits each stage back to the loader, each finished tile to the epilogue
-//       warps 2..5  epilogue: thread i of the warp covering TMEM lanes 32q..32q+31 owns logit rows 32q + i and
-//                   128 + 32q + i; it reads its rows' accumulators 32 columns at a time (tcgen05.ld) and folds
-//                   them into a running (max, arg-max, reference exponent, sum) -- no exchange between threads,
-//                   a row lives in one thread -- and keeps z[row, draft[row]] when that column comes by
+//       warps 2..9  epilogue: warps 2..5 take the first row tile, warps 6..9 the second; thread i of the warp covering
+//                   TMEM lanes 32q..32q+31 owns logit row 32q + i of its tile; it reads the row's accumulators 64
+//                   columns at a time (two tcgen05.ld in flight) and folds them into a running (max, arg-max,
+//                   reference exponent, sum) -- no exchange between threads, a row lives in one thread -- and
+//                   keeps z[row, draft[row]] when that column comes by
 //     A CTA owns a contiguous run of vocabulary tiles and ends with one partial per logit row.
 //   lmhead_finalize_kernel  one warp per batch row: folds the CTAs' partials in a fixed order, then S2..S5
 //                           exactly as the streaming step does; the memory update follows as its own launch.
@@ -35,9 +36,9 @@ namespace lmhead {
 constexpr int kBlockK = 64;                 // bf16 elements of a k-block: one 128-byte swizzle row
 constexpr int kMaxStages = 8;
 constexpr int kMTile = 128;
-constexpr int kRowsMax = 2 * kMTile;        // logit rows a step may have
+constexpr int kRowsMax = 2 * kMTile;        // logit rows of a row group
 constexpr int kNMax = 256;                  // widest vocabulary tile
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                // warp 0 loads, warp 1 issues MMAs, warps 2..5 / 6..9 reduce the first / second row tile
 constexpr int kRowBytes = kBlockK * 2;      // one row of a k-block
 constexpr int kBarrierBytes = 1024;
 // The second row tile's operand is read as 128 rows although only the rows that exist are loaded: the read
@@ -53,9 +54,10 @@ struct Params {
     int n_tile;             // columns of a vocabulary tile: multiple of 16, at most kNMax
     int tiles_total;        // ceil(V / n_tile)
     int tiles_per_cta;
-    int rows2;              // rows loaded for the second row tile (0 if R <= 128), a multiple of 8
-    int a_bytes;            // bytes of the hidden k-block in a stage (both row tiles), a multiple of 1 KiB
-    int stage_bytes;        // a_bytes + the W tile's k-block, a multiple of 1 KiB
+    int rows2;              // rows loaded for the second row tile of the LAST row group (0 if it has <= 128 rows), a multiple of 8
+    int a_bytes;            // bytes of a hidden k-block in a stage (both row tiles), a multiple of 1 KiB
+    int sub_bytes;          // a_bytes + the W tile's k-block, a multiple of 1 KiB
+    int kblocks_per_stage;  // k-blocks loaded, consumed and released together (H is a multiple of 64 times this)
     int n_stages;
     const int *draft;       // [B, K]
     Partial *partials;      // [R, gridDim.x]
@@ -130,23 +132,36 @@ __device__ __forceinline__ void tc_mma_bf16(unsigned int d_tmem, unsigned long l
                  "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
                  : "memory");
 }
-// 32 consecutive accumulator columns of this thread's TMEM lane.
+// 32 consecutive accumulator columns of this thread's TMEM lane.  The load is asynchronous; load and wait are one
+// statement so that nothing can read the registers in between.
 __device__ __forceinline__ void tmem_ld32(unsigned int taddr, float (&x)[32])
 {
     unsigned int r[32];
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
-          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
-          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
-          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr)
         : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(r[j]);
+}
+// 64 consecutive columns: two loads in flight, one wait.
+__device__ __forceinline__ void tmem_ld64(unsigned int taddr, float (&x)[32], float (&y)[32])
+{
+    unsigned int r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%64];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%65];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr), "r"(taddr + 32u)
+        : "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        x[j] = __uint_as_float(r[j]);
+        y[j] = __uint_as_float(r[32 + j]);
+    }
 }
 
 // Shared-memory operand descriptor of a K-major bf16 tile stored as rows of 128 bytes with the 128-byte swizzle
@@ -227,30 +242,36 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
     const unsigned int raw = smem_u32(smem_raw);
     const unsigned int bars = (raw + 1023u) & ~1023u;
     const unsigned int stages = bars + kBarrierBytes;
-    const int kStages = p.n_stages;
-    const int kStageBytes = p.stage_bytes, kStageABytes = p.a_bytes;
+    const int n_stages = p.n_stages;
+    const int kps = p.kblocks_per_stage;                   // k-blocks that travel and are released together
+    const int sub_bytes = p.sub_bytes, a_bytes = p.a_bytes, stage_bytes = kps * sub_bytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
     const unsigned int tmem_full = bars + 8u * (2 * kMaxStages);
     const unsigned int tmem_empty = bars + 8u * (2 * kMaxStages + 1);
 
-    const int n_mt = p.R > kMTile ? 2 : 1;
-    const int kblocks = p.H / kBlockK;
+    // Logit rows are taken in groups of 256 (two row tiles), one group after the other: a group sees the whole
+    // vocabulary range of this CTA before the next begins, so a row's running statistics live in one thread.
+    const int n_groups = (p.R + kRowsMax - 1) / kRowsMax;
+    const int k_steps = p.H / (kBlockK * kps);             // stage fills per tile
     const int tile0 = blockIdx.x * p.tiles_per_cta;
     int tile1 = tile0 + p.tiles_per_cta;
     if (tile1 > p.tiles_total) tile1 = p.tiles_total;
     const int my_tiles = tile1 > tile0 ? tile1 - tile0 : 0;
+    auto rows_of = [&](int g) { return min(kRowsMax, p.R - g * kRowsMax); };
 
     if (threadIdx.x == 0) {
         give_up_flag = 0;
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
         }
         mbar_init(tmem_full, 1);
-        mbar_init(tmem_empty, 4 * 32);
+        mbar_init(tmem_empty, 8 * 32);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // the decision kernel behind this one may be brought in now; it waits for this grid before it reads anything
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (warp == 2) {
         tmem_alloc(smem_u32(&tmem_base_slot), kTmemCols);
         tmem_relinquish();
@@ -263,18 +284,30 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
     if (warp == 0) {
         // ---- loader ----
         if (lane == 0) {
-            const unsigned int tx = static_cast<unsigned int>((kMTile + p.rows2 + p.n_tile) * kRowBytes);
             int it = 0;
-            for (int t = tile0; t < tile1 && !*give_up; ++t) {
-                const int v0 = t * p.n_tile;
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    if (!mbar_wait(empty_bar(s), ((it / kStages) & 1) ^ 1, give_up)) break;
-                    const unsigned int a = stages + s * kStageBytes, b = a + kStageABytes;
-                    mbar_expect_tx(full_bar(s), tx);
-                    tma_load_2d(a, &map_hidden, full_bar(s), kb * kBlockK, 0);
-                    if (n_mt == 2) tma_load_2d(a + kMTile * kRowBytes, &map_hidden2, full_bar(s), kb * kBlockK, kMTile);
-                    tma_load_2d(b, &map_weight, full_bar(s), kb * kBlockK, v0);
+            for (int g = 0; g < n_groups && !*give_up; ++g) {
+                const int rows = rows_of(g);
+                const bool last_group = g == n_groups - 1;
+                // the second row tile: 128 rows in a full group, the rows that exist (rounded up to 8) in the last one
+                const int rows2 = rows > kMTile ? (last_group ? p.rows2 : kMTile) : 0;
+                const unsigned int tx = static_cast<unsigned int>(kps * (kMTile + rows2 + p.n_tile) * kRowBytes);
+                for (int t = tile0; t < tile1 && !*give_up; ++t) {
+                    const int v0 = t * p.n_tile;
+                    for (int ks = 0; ks < k_steps; ++ks, ++it) {
+                        const int s = it % n_stages;
+                        if (!mbar_wait(empty_bar(s), ((it / n_stages) & 1) ^ 1, give_up)) break;
+                        mbar_expect_tx(full_bar(s), tx);
+                        for (int sub = 0; sub < kps; ++sub) {
+                            const unsigned int a = stages + s * stage_bytes + sub * sub_bytes, b = a + a_bytes;
+                            const int x = (ks * kps + sub) * kBlockK;
+                            tma_load_2d(a, &map_hidden, full_bar(s), x, g * kRowsMax);
+                            if (rows2 == kMTile)
+                                tma_load_2d(a + kMTile * kRowBytes, &map_hidden, full_bar(s), x, g * kRowsMax + kMTile);
+                            else if (rows2 > 0)
+                                tma_load_2d(a + kMTile * kRowBytes, &map_hidden2, full_bar(s), x, g * kRowsMax + kMTile);
+                            tma_load_2d(b, &map_weight, full_bar(s), x, v0);
+                        }
+                    }
                 }
             }
         }
@@ -282,110 +315,117 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
         // ---- MMA issuer ----
         if (lane == 0) {
             const unsigned int idesc = instr_desc(p.n_tile);
-            int it = 0;
-            for (int t = 0; t < my_tiles && !*give_up; ++t) {
-                if (!mbar_wait(tmem_empty, (t & 1) ^ 1, give_up)) break;      // the epilogue has drained the previous tile
-                tc_fence_after();
-                bool ok = true;
-                for (int kb = 0; kb < kblocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    if (!mbar_wait(full_bar(s), (it / kStages) & 1, give_up)) {
+            int it = 0, tt = 0;
+            bool ok = true;
+            for (int g = 0; g < n_groups && ok && !*give_up; ++g) {
+                const int n_mt = rows_of(g) > kMTile ? 2 : 1;
+                for (int t = 0; t < my_tiles && ok && !*give_up; ++t, ++tt) {
+                    if (!mbar_wait(tmem_empty, (tt & 1) ^ 1, give_up)) {      // the epilogue has drained the previous tile
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const unsigned int a = stages + s * kStageBytes, b = a + kStageABytes;
-                    const unsigned long long a0_desc = operand_desc(a), a1_desc = operand_desc(a + kMTile * kRowBytes);
-                    const unsigned long long b_desc = operand_desc(b);
+                    for (int ks = 0; ks < k_steps; ++ks, ++it) {
+                        const int s = it % n_stages;
+                        if (!mbar_wait(full_bar(s), (it / n_stages) & 1, give_up)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        for (int sub = 0; sub < kps; ++sub) {
+                            const unsigned int a = stages + s * stage_bytes + sub * sub_bytes, b = a + a_bytes;
+                            const unsigned long long a0_desc = operand_desc(a), a1_desc = operand_desc(a + kMTile * kRowBytes);
+                            const unsigned long long b_desc = operand_desc(b);
 #pragma unroll
-                    for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
-                        const unsigned int acc = (kb | k4) != 0 ? 1u : 0u;
-                        // 16 columns further along K: 32 bytes, 2 in the descriptor's units of 16 bytes
-                        tc_mma_bf16(tmem_base, a0_desc + 2ull * k4, b_desc + 2ull * k4, idesc, acc);
-                        if (n_mt == 2) tc_mma_bf16(tmem_base + kNMax, a1_desc + 2ull * k4, b_desc + 2ull * k4, idesc, acc);
+                            for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
+                                const unsigned int acc = (ks | sub | k4) != 0 ? 1u : 0u;
+                                // 16 columns further along K: 32 bytes, 2 in the descriptor's units of 16 bytes
+                                tc_mma_bf16(tmem_base, a0_desc + 2ull * k4, b_desc + 2ull * k4, idesc, acc);
+                                if (n_mt == 2) tc_mma_bf16(tmem_base + kNMax, a1_desc + 2ull * k4, b_desc + 2ull * k4, idesc, acc);
+                            }
+                        }
+                        tc_commit(empty_bar(s));          // the stage may be refilled once these MMAs have read it
                     }
-                    tc_commit(empty_bar(s));          // the stage may be refilled once these MMAs have read it
+                    if (ok) tc_commit(tmem_full);         // the tile's accumulators are complete
                 }
-                if (!ok) break;
-                tc_commit(tmem_full);                 // the tile's accumulators are complete
             }
         }
     } else {
-        // ---- epilogue: warp w covers TMEM lanes 32 (w % 4) .. + 31 ----
+        // ---- epilogue: warp w covers TMEM lanes 32 (w % 4) .. + 31; warps 2..5 take the first row tile of a
+        // group, warps 6..9 the second; a thread owns one logit row ----
         const int q = warp & 3;
-        const int row_a = 32 * q + lane, row_b = kMTile + row_a;
-        const bool has_a = row_a < p.R, has_b = row_b < p.R;             // has_b implies has_a
-        const bool warp_b = kMTile + 32 * q < p.R;                       // the warp has any row in the second tile
-        RowRun ra, rb;
-        row_init(ra);
-        row_init(rb);
-        auto draft_of = [&](int row) {
-            const int b = row / (p.K + 1), i = row - b * (p.K + 1);
-            return (row < p.R && i < p.K) ? __ldg(p.draft + b * p.K + i) : -1;
-        };
-        const int da = draft_of(row_a), db = draft_of(row_b);
-        float zda = 0.f, zdb = 0.f;
-        bool got_a = false, got_b = false;
-        for (int t = 0; t < my_tiles; ++t) {
-            if (!mbar_wait(tmem_full, t & 1, give_up)) break;
-            tc_fence_after();
-            const int v0 = (tile0 + t) * p.n_tile;
-            const int v_end = min(p.V, v0 + p.n_tile);          // columns beyond the tile or the vocabulary are masked
-            for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
-                const int vc = v0 + c0;
-                if (vc >= v_end) break;
-                float x[32];
-                tmem_ld32(tmem_base + (static_cast<unsigned int>(32 * q) << 16) + c0, x);
-                if (vc + 32 > v_end) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) x[j] = (vc + j < v_end) ? x[j] : -INFINITY;
-                }
-                if (has_a) {
-                    row_take(ra, x, vc);
-                    if (static_cast<unsigned int>(da - vc) < 32u && da < v_end) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) zda = (da - vc == j) ? x[j] : zda;
-                        got_a = true;
-                    }
-                }
-                if (warp_b) {
-                    tmem_ld32(tmem_base + (static_cast<unsigned int>(32 * q) << 16) + kNMax + c0, x);
-                    if (vc + 32 > v_end) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) x[j] = (vc + j < v_end) ? x[j] : -INFINITY;
-                    }
-                    if (has_b) {
-                        row_take(rb, x, vc);
-                        if (static_cast<unsigned int>(db - vc) < 32u && db < v_end) {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) zdb = (db - vc == j) ? x[j] : zdb;
-                            got_b = true;
-                        }
-                    }
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(tmem_empty);
-        }
-        auto finish = [&](const RowRun &r, int row, bool got, float zd, int d) {
-            if (row >= p.R) return;
-            float s0, s1, s2, s3;
-            unpack2(r.acc0, s0, s1);
-            unpack2(r.acc1, s2, s3);
-            Partial out;
-            out.m = r.m;
-            out.idx = r.idx;
-            out.c = r.c;
-            out.s = (s0 + s1) + (s2 + s3);
-            st_partial_cg(p.partials + static_cast<size_t>(row) * gridDim.x + blockIdx.x, out);
-            if (got) {
+        const int mt = warp >= 6 ? 1 : 0;
+        const unsigned int lane_base = tmem_base + (static_cast<unsigned int>(32 * q) << 16) + (mt ? kNMax : 0);
+        int tt = 0;
+        bool ok = true;
+        for (int g = 0; g < n_groups && ok; ++g) {
+            const int row = g * kRowsMax + mt * kMTile + 32 * q + lane;
+            const bool has = row < p.R;
+            const bool warp_has = g * kRowsMax + mt * kMTile + 32 * q < p.R;      // the warp has any row in this group
+            RowRun rr;
+            row_init(rr);
+            int d = -1;
+            if (has) {
                 const int b = row / (p.K + 1), i = row - b * (p.K + 1);
-                __stcg(p.zd + b * p.K + i, zd);
+                if (i < p.K) d = __ldg(p.draft + b * p.K + i);
             }
-            (void)d;
-        };
-        finish(ra, row_a, got_a, zda, da);
-        finish(rb, row_b, got_b, zdb, db);
+            float zd = 0.f;
+            bool got = false;
+            for (int t = 0; t < my_tiles; ++t, ++tt) {
+                if (!mbar_wait(tmem_full, tt & 1, give_up)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const int v0 = (tile0 + t) * p.n_tile;
+                const int v_end = min(p.V, v0 + p.n_tile);          // columns beyond the tile or the vocabulary are masked
+                if (warp_has) {
+                    for (int c0 = 0; c0 < p.n_tile; c0 += 64) {
+                        const int vc = v0 + c0;
+                        if (vc >= v_end) break;
+                        const bool second = c0 + 32 < p.n_tile && vc + 32 < v_end;
+                        float x[32], y[32];
+                        if (second)
+                            tmem_ld64(lane_base + c0, x, y);
+                        else
+                            tmem_ld32(lane_base + c0, x);
+                        auto take = [&](float (&v)[32], int vb) {
+                            if (vb + 32 > v_end) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) v[j] = (vb + j < v_end) ? v[j] : -INFINITY;
+                            }
+                            if (has) {
+                                row_take(rr, v, vb);
+                                if (static_cast<unsigned int>(d - vb) < 32u && d < v_end) {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) zd = (d - vb == j) ? v[j] : zd;
+                                    got = true;
+                                }
+                            }
+                        };
+                        take(x, vc);
+                        if (second) take(y, vc + 32);
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(tmem_empty);
+            }
+            if (has) {
+                float s0, s1, s2, s3;
+                unpack2(rr.acc0, s0, s1);
+                unpack2(rr.acc1, s2, s3);
+                Partial out;
+                out.m = rr.m;
+                out.idx = rr.idx;
+                out.c = rr.c;
+                out.s = (s0 + s1) + (s2 + s3);
+                st_partial_cg(p.partials + static_cast<size_t>(row) * gridDim.x + blockIdx.x, out);
+                if (got) {
+                    const int b = row / (p.K + 1), i = row - b * (p.K + 1);
+                    __stcg(p.zd + b * p.K + i, zd);
+                }
+            }
+        }
     }
 
     tc_fence_before();
@@ -426,6 +466,9 @@ __global__ void __launch_bounds__(128) lmhead_finalize_kernel(const FinalizePara
     __shared__ int sm_t[4][CSD_MAX_K + 1];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int b = blockIdx.x * 4 + w;
+    // launched programmatically behind the GEMM kernel: let the memory's update kernel in, then wait for the GEMM
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (b >= p.B) return;
     const int K = p.K, K1 = K + 1;
     // the draft tokens and their logits do not depend on the fold: requested first
