@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0            # earlier measurement on this machine, used wh
 DEFAULT_WORKLOAD = "large_batch"
 # DRAM bytes per launch of the step kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); a workload is absent where no capture of the current kernel exists.
-NCU_TRAFFIC_BYTES = {"ocm_contention": 140787712}
+NCU_TRAFFIC_BYTES = {"large_batch": 596126208, "ocm_contention": 140787712, "batched_serving": 58522880}
 
 
 def measured_peak():
