@@ -121,3 +121,23 @@ def test_binding_refuses_without_device():
         pytest.skip("device present")
     with pytest.raises(binding.CsdError):
         binding.Ocm(1024)
+
+
+def test_plans_of_the_other_entry_points(L):
+    """Host-side sizing of the stochastic, two-phase and LM-head steps (no device needed)."""
+    for (B, K, V, dt) in SHAPES[:7]:
+        assert L.csd_sampled_workspace_bytes(B, K, V, dt) > 0
+        if K >= 2:
+            ws = L.csd_early_exit_workspace_bytes(B, K, V, dt, 0)
+            assert ws >= binding.csd_workspace_bytes(B, max(1, (K + 1) // 3), V, dt) // 2 + 4 * B
+            assert L.csd_early_exit_workspace_bytes(B, K, V, dt, K - 1) > 0
+        else:
+            assert L.csd_early_exit_workspace_bytes(B, K, V, dt, 0) == 0
+    g, n, t, per = (ctypes.c_int() for _ in range(4))
+    for (B, K, H, V) in ((32, 5, 4096, 151936), (64, 6, 4096, 152064), (128, 8, 4096, 128256), (1, 1, 64, 17), (2, 3, 128, 1000)):
+        assert L.csd_lmhead_shape(B, K, H, V, ctypes.byref(g), ctypes.byref(n), ctypes.byref(t), ctypes.byref(per)) == 0
+        assert 1 <= g.value <= 148 and n.value % 16 == 0 and 16 <= n.value <= 256
+        assert t.value == -(-V // n.value) and g.value * per.value >= t.value and (g.value - 1) * per.value < t.value
+        assert L.csd_lmhead_workspace_bytes(B, K, H, V) >= B * (K + 1) * g.value * 16 + 4 * B * K
+    assert L.csd_lmhead_workspace_bytes(2, 3, 100, 1000) == 0            # H must be a multiple of 64
+    assert L.csd_lmhead_shape(2, 33, 128, 1000, None, None, None, None) != 0
