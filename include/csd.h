@@ -155,11 +155,14 @@ csd_status_t csd_ocm_set_shared(csd_ocm_t *ocm, int enable);
  * per-block partial reductions, slot hints and arrival counters. */
 size_t csd_workspace_bytes(int B, int K, int V, csd_dtype_t dtype);
 
-/* Zero a workspace.  Required once before its first use (and after any aborted
+/* Zero a workspace.  Do it once before its first use (and after any aborted
  * launch); the kernels leave the counters zeroed again on completion, so the
- * same workspace can be reused step after step without further clearing.  One
- * workspace serves one step at a time, and all steps that use it are issued on
- * one stream. */
+ * same workspace can be reused step after step without further clearing.  (The
+ * library also clears a workspace by itself the first time it sees its address,
+ * and whenever the launch shape it was last used with differs from the current
+ * one; memory that is freed and handed out again at the same address with stale
+ * contents is the case only this call covers.)  One workspace serves one step at
+ * a time, and all steps that use it are issued on one stream. */
 csd_status_t csd_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 
 /* The verification loop of Algorithm 1 (greedy) for all B rows, read-only on the
@@ -484,11 +487,17 @@ csd_status_t csd_set_tuning(int chunk_bytes, int ctas_per_sm, int block_threads)
  * retire.  The automatic launch shape also changes: one block per SM and launch
  * instead of four, so that several steps are resident at a time (the low-order bits of
  * the diagnostic sums s may therefore differ from those with overlap off; all decisions
- * are identical).  Turn it on only if the logits and draft of a step are never written
- * by a kernel that may still be running when the step starts: back-to-back steps over
- * inputs that are already resident qualify; so does a producer kernel launched right
- * before the step as long as it does not itself signal early completion.  Steps that
- * share a memory or output buffers are issued on one stream.  Host function. */
+ * are identical).  Turn it on only if the logits and draft tokens of every step were
+ * complete (their producer finished, and a normal stream dependency, event or host
+ * synchronisation passed) BEFORE the step before it was enqueued: a step reads its inputs
+ * before it waits for its predecessor on the stream, and CUDA makes a predecessor's writes
+ * visible only after that wait.  Back-to-back steps over inputs that are already resident
+ * qualify; a kernel that writes a step's inputs between two steps does not -- a decode loop
+ * with the model's forward pass between steps keeps the default.  Steps that share a memory
+ * or output buffers are issued on one stream (but see csd_ocm_set_shared).  Changing the
+ * setting, or csd_set_tuning, changes the layout of the scratch inside a workspace; the
+ * library notices a workspace that last held another layout and clears it before use, so
+ * no re-initialisation is needed.  Host function. */
 csd_status_t csd_set_overlap(int enable);
 
 const char *csd_status_string(csd_status_t status);
