@@ -465,6 +465,13 @@ def run_ours(args, wl, tau):
             except Exception as e:             # the greedy line stands on its own
                 line["sampled"] = {"error": repr(e)}
             try:
+                from synth_inputs import WORKLOADS
+                torch.cuda.empty_cache()
+                line["multi_stream"] = measure_multi_stream(WORKLOADS["batched_serving"], 0.3, device)
+                pkg.csd_set_overlap(overlap)
+            except Exception as e:
+                line["multi_stream"] = {"error": repr(e)}
+            try:
                 torch.cuda.empty_cache()
                 line["early_exit"] = measure_early_exit(wl, tau, device)
                 pkg.csd_set_overlap(overlap)
@@ -686,6 +693,67 @@ def measure_early_exit(wl, tau, device, steps=48):
             "logit_bytes_read": read, "logit_bytes_of_csd_step": wl.logit_bytes, "bytes_fraction": read / wl.logit_bytes,
             "achieved_GBs": read / t_two / 1e9, "frac_of_measured_peak": read / t_two / 1e9 / peak, "peak_source": f"of {kind}",
             "launch": f"CUDA graph of {steps} steps (3 launches each), stream-ordered, replayed", "repeats": 7}
+
+
+def measure_multi_stream(wl, tau, device, n_streams=4, steps=48):
+    """n_streams serving streams stepping at the same time on ONE shared memory (csd_ocm_set_shared), each with its
+    own workspace and outputs, each replaying its own graph of `steps` steps in the overlap launch shape."""
+    import torch
+
+    import paper_2604_13634_b200 as pkg
+    from synth_inputs import Synth
+
+    l2 = torch.cuda.get_device_properties(device).L2_cache_size
+    ring_len = max(2 * n_streams, math.ceil(2 * l2 / wl.logit_bytes) + 1)
+    syn = Synth(wl, 0, device)
+    ring = [syn.step(s) for s in range(ring_len)]
+    ocm = pkg.Ocm(wl.ocm_slots, wl.lam, device.index)
+    if wl.prewarm[0] == "pairs":
+        ocm.update(*syn.prewarm_pairs(wl.prewarm[1]))
+    ocm.set_shared(True)
+    pkg.csd_set_overlap(True)
+    streams = [torch.cuda.Stream(device) for _ in range(n_streams)]
+    bufs = [pkg.StepBuffers(wl.B, wl.K, wl.V, wl.torch_dtype, device=device) for _ in range(n_streams)]
+    graphs = []
+    torch.cuda.synchronize(device)
+    for s in range(n_streams):
+        off = s * (ring_len // n_streams)
+        with torch.cuda.stream(streams[s]):
+            pkg.csd_step(*ring[off % ring_len], ocm, tau, bufs[s])             # first use of the workspace, outside the capture
+        torch.cuda.synchronize(device)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=streams[s]):
+            for i in range(steps):
+                pkg.csd_step(*ring[(off + i) % ring_len], ocm, tau, bufs[s])
+        graphs.append(g)
+
+    def once():
+        torch.cuda.synchronize(device)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for s in range(n_streams):
+            streams[s].wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(streams[s]):
+                graphs[s].replay()
+        for s in range(n_streams):
+            torch.cuda.current_stream().wait_stream(streams[s])
+        b.record()
+        b.synchronize()
+        return a.elapsed_time(b) * 1e-3
+
+    once()
+    sec = statistics.median(once() for _ in range(7))
+    st = ocm.stats()
+    torch.cuda.synchronize(device)
+    ocm.set_shared(False)
+    ocm.close()
+    peak, kind = measured_peak()
+    total_steps = n_streams * steps
+    return {"streams": n_streams, "steps_per_stream": steps, "us_per_step_aggregate": 1e6 * sec / total_steps,
+            "positions_per_s": wl.B * wl.K * total_steps / sec, "achieved_GBs": wl.logit_bytes * total_steps / sec / 1e9,
+            "frac_of_measured_peak": wl.logit_bytes * total_steps / sec / 1e9 / peak, "peak_source": f"of {kind}", "repeats": 7,
+            "launch": f"{n_streams} streams, each a CUDA graph of {steps} steps, replayed together on one shared memory",
+            "ocm": {k: st[k] for k in ("n_keys", "n_dropped", "rescues", "rejections", "flags")}}
 
 
 def measure_lmhead(wl, tau, device, H=4096, steps=12, repeats=7):
