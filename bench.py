@@ -481,6 +481,8 @@ def run_ours(args, wl, tau):
                 from synth_inputs import WORKLOADS
                 torch.cuda.empty_cache()
                 line["lmhead"] = measure_lmhead(WORKLOADS["batched_serving"], 0.3, device)
+                torch.cuda.empty_cache()
+                line["lmhead"]["single_stream"] = measure_lmhead(WORKLOADS["single_stream"], 0.3, device)
                 pkg.csd_set_overlap(overlap)
             except Exception as e:
                 line["lmhead"] = {"error": repr(e)}
@@ -814,7 +816,7 @@ def measure_lmhead(wl, tau, device, H=4096, steps=12, repeats=7):
             "bound": "hbm" if hbm_bytes / (hbm * 1e9) >= flops / (tensor_peak * 1e12) else "tensor",
             "roofline_us": 1e6 * t_bound, "frac_of_roofline": t_bound / fused, "peak_source": f"of {kind}",
             "unfused_us_per_step": 1e6 * plain,
-            "unfused": "torch.matmul (bf16 logits stored, 58 MB written and read back) followed by csd_step",
+            "unfused": f"torch.matmul (bf16 logits stored, {R * wl.V * 2 / 1e6:.0f} MB written and read back) followed by csd_step",
             "launches_per_step": 3, "launch": "eager",
             "ocm": {k: st[k] for k in ("n_keys", "rescues", "rejections", "flags")}}
 
@@ -832,6 +834,10 @@ def run_lmhead(args, wl, tau):
     sampler = ClockSampler(device.index, period_s=0.005)
     sampler.start()
     m = measure_lmhead(wl, tau, device, H=args.hidden, steps=max(3, min(args.steps, 48)))
+    if wl.name != "single_stream":
+        from synth_inputs import WORKLOADS
+        torch.cuda.empty_cache()
+        m["single_stream"] = measure_lmhead(WORKLOADS["single_stream"], 0.3, device, H=args.hidden, steps=m["steps"])
     clocks = sampler.stop()
     line = {"metric": METRIC, "value": m["positions_per_s"], "unit": UNIT, "n_gpus": 1, "steps": m["steps"],
             "warmup": 3, "ms_per_step": m["us_per_step"] * 1e-3, "higher_is_better": True, "scaling": "weak",
@@ -842,7 +848,7 @@ def run_lmhead(args, wl, tau):
             "roofline": {"bound": m["bound"], "achieved": m["hbm_GBs"] if m["bound"] == "hbm" else m["tensor_TFLOPs"],
                          "peak": measured_peak()[0] if m["bound"] == "hbm" else None, "unit": "GB/s" if m["bound"] == "hbm" else "TFLOP/s",
                          "frac": m["frac_of_roofline"], "traffic": None, "peak_source": m["peak_source"],
-                         "kernel": "lmhead_stats_kernel", "tensor_TFLOPs": m["tensor_TFLOPs"], "tensor_frac": m["tensor_frac"]},
+                         "kernel": m["shape"]["kernel"], "tensor_TFLOPs": m["tensor_TFLOPs"], "tensor_frac": m["tensor_frac"]},
             "gpu_launches": 3 * m["steps"], "clocks": clocks, "lmhead": m}
     print(json.dumps(line), flush=True)
 

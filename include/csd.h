@@ -382,10 +382,24 @@ csd_status_t csd_step_lmhead(const void *hidden, const void *weight, int B, int 
 /* How the vocabulary is cut for this shape: blocks of the GEMM grid, columns per tile, number of tiles and
  * tiles per block.  Host function; for reports and tests. */
 csd_status_t csd_lmhead_shape(int B, int K, int H, int V, int *grid, int *tile_cols, int *tiles, int *tiles_per_block);
-/* Expert knob, process-wide: how many 64-column k-blocks travel through the shared-memory ring together
- * (1 to 4; 0 = automatic).  More per stage means longer contiguous reads of each weight row and fewer, larger
- * stages.  Results do not depend on it beyond the rounding order of the accumulation.  Host function. */
-csd_status_t csd_lmhead_set_tuning(int kblocks_per_stage);
+/* 1 if the GEMM of this shape would run as pairs of blocks (see csd_lmhead_set_pairing), else 0.  Host function. */
+int csd_lmhead_uses_pairs(int B, int K);
+/* Expert knobs, process-wide.  kblocks_per_stage: how many 64-column k-blocks travel through the shared-memory
+ * ring together (1 to 4; 0 = automatic; the pair kernel always takes 1).  More per stage means longer contiguous
+ * reads of each weight row and fewer, larger stages.  mma_cols: the N of one tensor-core instruction, a multiple
+ * of 16 from 16 to 256 (0 = automatic: the widest that gives every block the same number of tiles); a tile has
+ * mma_cols columns with one block per SM and 2 mma_cols with pairs.  Results do not depend on either beyond the
+ * rounding order of the sums.  Host function; INVALID_ARG outside these ranges. */
+csd_status_t csd_lmhead_set_tuning(int kblocks_per_stage, int mma_cols);
+/* Expert knob, process-wide: which GEMM kernel runs.  0 = automatic (the default), 1 = one block per SM, each on
+ * its own vocabulary tiles with up to 256 logit rows; 2 = pairs of blocks on neighbouring SMs (thread-block clusters
+ * of two), each block holding half of the logit rows against a tile twice as wide, which halves the share of the
+ * hidden states in an SM's shared-memory traffic.  Automatic takes pairs for more than 128 logit rows.  Results
+ * are the same up to which vocabulary ranges the per-block partial sums cover (the last bits of s, lse and the
+ * probabilities).  csd_lmhead_shape reports the cut of the kernel that would run; for pairs, tile_cols is the
+ * width of a pair's tile and tiles_per_block the tiles per pair.  A wait that runs out in the pair kernel reports
+ * debug_site 31.  Host function; INVALID_ARG outside 0..2. */
+csd_status_t csd_lmhead_set_pairing(int mode);
 
 /* csd_step for callers whose tensors live in HOST memory (pinned memory gives
  * the full copy rate).  Copies logits and draft to `staging`, runs the step, and

@@ -30,7 +30,7 @@ EXPORTS = [
     "csd_sampled_workspace_bytes", "csd_verify_sampled", "csd_step_sampled",
     "csd_ocm_age", "csd_ocm_merge", "csd_ocm_save", "csd_ocm_load", "csd_ocm_set_shared",
     "csd_lmhead_workspace_bytes", "csd_verify_lmhead", "csd_step_lmhead", "csd_lmhead_shape",
-    "csd_early_exit_workspace_bytes", "csd_step_early_exit", "csd_lmhead_set_tuning",
+    "csd_early_exit_workspace_bytes", "csd_step_early_exit", "csd_lmhead_set_tuning", "csd_lmhead_set_pairing", "csd_lmhead_uses_pairs",
 ]
 
 
@@ -101,7 +101,9 @@ def lib():
         "csd_lmhead_shape": (c_int, [c_int, c_int, c_int, c_int, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]),
         "csd_early_exit_workspace_bytes": (c_size_t, [c_int, c_int, c_int, c_int, c_int]),
         "csd_step_early_exit": (c_int, step_args[:10] + [c_int] + step_args[10:]),
-        "csd_lmhead_set_tuning": (c_int, [c_int]),
+        "csd_lmhead_set_tuning": (c_int, [c_int, c_int]),
+        "csd_lmhead_set_pairing": (c_int, [c_int]),
+        "csd_lmhead_uses_pairs": (c_int, [c_int, c_int]),
         "csd_ocm_age": (c_int, [c_void_p, c_void_p]),
         "csd_ocm_set_shared": (c_int, [c_void_p, c_int]),
         "csd_ocm_merge": (c_int, [c_void_p, c_void_p, c_void_p]),
@@ -437,7 +439,9 @@ class LmheadBuffers(StepBuffers):
 def csd_lmhead_shape(B, K, H, V):
     g, n, t, per = c_int(), c_int(), c_int(), c_int()
     _check(lib().csd_lmhead_shape(B, K, H, V, byref(g), byref(n), byref(t), byref(per)), "csd_lmhead_shape")
-    return dict(grid=g.value, tile_cols=n.value, tiles=t.value, tiles_per_block=per.value)
+    pairs = bool(lib().csd_lmhead_uses_pairs(B, K))
+    return dict(grid=g.value, tile_cols=n.value, tiles=t.value, tiles_per_block=per.value,
+                kernel="lmhead_stats_pair_kernel" if pairs else "lmhead_stats_kernel")
 
 
 def _lmhead_call(fn_name, hidden, weight, draft, ocm: Ocm, tau, buf: LmheadBuffers, stream):
@@ -488,5 +492,10 @@ def csd_step_early_exit(logits, draft, ocm: Ocm, tau: float, buf: EarlyExitBuffe
     _check(rc, "csd_step_early_exit")
 
 
-def csd_lmhead_set_tuning(kblocks_per_stage: int = 0):
-    _check(lib().csd_lmhead_set_tuning(kblocks_per_stage), "csd_lmhead_set_tuning")
+def csd_lmhead_set_tuning(kblocks_per_stage: int = 0, mma_cols: int = 0):
+    _check(lib().csd_lmhead_set_tuning(kblocks_per_stage, mma_cols), "csd_lmhead_set_tuning")
+
+
+def csd_lmhead_set_pairing(mode: int = 0):
+    """0 automatic, 1 one block per SM, 2 pairs of blocks (clusters of two)."""
+    _check(lib().csd_lmhead_set_pairing(mode), "csd_lmhead_set_pairing")

@@ -861,8 +861,9 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
 namespace {
 
 struct LmheadPlan {
+    bool pair;              // CTA pairs (clusters of two) instead of lone CTAs
     int grid, n_tile, tiles_total, tiles_per_cta;
-    int rows2, a_bytes, sub_bytes, kps, n_stages, smem_bytes;
+    int rows1, rows2, a_bytes, sub_bytes, kps, n_stages, smem_bytes;
     size_t partials_off, zd_off, total;
 };
 
@@ -874,12 +875,23 @@ bool lmhead_shape_ok(int B, int K, int H, int V)
 }
 
 int g_lmhead_kblocks_per_stage = 0;   // 0 = automatic
+int g_lmhead_pairing = 0;             // 0 = automatic, 1 = lone CTAs, 2 = CTA pairs
+int g_lmhead_tile_cols = 0;           // 0 = automatic; else the columns of one MMA (a multiple of 16, 16..256)
+int g_lmhead_wide_fetch = 1;          // W rows come into L2 256 bytes at a time (two consecutive k-blocks of a row)
 
-// The vocabulary is cut into tiles of n_tile columns (a multiple of 16, at most 256) such that every CTA of a
-// one-per-SM grid owns the same number of consecutive tiles.
-LmheadPlan lmhead_plan(int B, int K, int H, int V)
+void lmhead_place_workspace(LmheadPlan &pl, size_t rows, int B, int K)
+{
+    pl.partials_off = 0;
+    pl.zd_off = align_up(rows * pl.grid * sizeof(Partial), 256);
+    pl.total = align_up(pl.zd_off + static_cast<size_t>(B) * K * sizeof(float), 256);
+}
+
+// Lone CTAs: the vocabulary is cut into tiles of n_tile columns (a multiple of 16, at most 256) such that every CTA of
+// a one-per-SM grid owns the same number of consecutive tiles.
+LmheadPlan lmhead_plan_lone(int B, int K, int H, int V)
 {
     LmheadPlan pl;
+    pl.pair = false;
     const long long sms = sm_count();
     long long per = (V + sms * lmhead::kNMax - 1) / (sms * lmhead::kNMax);          // tiles per CTA
     if (per < 1) per = 1;
@@ -887,6 +899,10 @@ LmheadPlan lmhead_plan(int B, int K, int H, int V)
     width = (width + 15) / 16 * 16;
     if (width > lmhead::kNMax) width = lmhead::kNMax;
     if (width < 16) width = 16;
+    if (g_lmhead_tile_cols > 0) {
+        width = g_lmhead_tile_cols;
+        per = (V + sms * width - 1) / (sms * width);
+    }
     pl.n_tile = static_cast<int>(width);
     pl.tiles_total = static_cast<int>((V + width - 1) / width);
     pl.tiles_per_cta = static_cast<int>(per);
@@ -897,8 +913,10 @@ LmheadPlan lmhead_plan(int B, int K, int H, int V)
     const size_t groups = (rows + lmhead::kRowsMax - 1) / lmhead::kRowsMax;
     const size_t rows_last = rows - (groups - 1) * lmhead::kRowsMax;
     pl.rows2 = rows_last > lmhead::kMTile ? static_cast<int>((rows_last - lmhead::kMTile + 7) / 8 * 8) : 0;
+    pl.rows1 = rows_last >= lmhead::kMTile ? lmhead::kMTile : static_cast<int>((rows_last + 7) / 8 * 8);
     const int rows2_most = groups > 1 ? lmhead::kMTile : pl.rows2;
-    pl.a_bytes = static_cast<int>(align_up(static_cast<size_t>(lmhead::kMTile + rows2_most) * lmhead::kRowBytes, 1024));
+    const int rows1_most = groups > 1 ? lmhead::kMTile : pl.rows1;           // a lone short group: W follows its rows at once
+    pl.a_bytes = static_cast<int>(align_up(static_cast<size_t>(rows1_most + rows2_most) * lmhead::kRowBytes, 1024));
     pl.sub_bytes = pl.a_bytes + static_cast<int>(align_up(static_cast<size_t>(pl.n_tile) * lmhead::kRowBytes, 1024));
     const int fixed = 1024 + lmhead::kBarrierBytes + lmhead::kSlackBytes;
     pl.kps = g_lmhead_kblocks_per_stage > 0 ? g_lmhead_kblocks_per_stage : 1;
@@ -906,10 +924,70 @@ LmheadPlan lmhead_plan(int B, int K, int H, int V)
     int stages = (lmhead::kSmemLimit - fixed) / (pl.kps * pl.sub_bytes);
     pl.n_stages = stages > lmhead::kMaxStages ? lmhead::kMaxStages : stages;
     pl.smem_bytes = fixed + pl.n_stages * pl.kps * pl.sub_bytes;
-    pl.partials_off = 0;
-    pl.zd_off = align_up(rows * pl.grid * sizeof(Partial), 256);
-    pl.total = align_up(pl.zd_off + static_cast<size_t>(B) * K * sizeof(float), 256);
+    lmhead_place_workspace(pl, rows, B, K);
     return pl;
+}
+
+// CTA pairs: a pair's tile has 2 n_tile columns (n_tile a multiple of 16, at most 256), every pair of a one-CTA-per-SM
+// grid owns the same number of consecutive tiles; each CTA holds half of a row group's rows.
+LmheadPlan lmhead_plan_pair(int B, int K, int /*H*/, int V)
+{
+    LmheadPlan pl;
+    pl.pair = true;
+    const long long pairs = sm_count() / 2;
+    const long long widest = 2 * lmhead::kNMax;
+    long long per = (V + pairs * widest - 1) / (pairs * widest);                    // tiles per pair
+    if (per < 1) per = 1;
+    long long width = (V + pairs * per - 1) / (pairs * per);                        // columns of a pair's tile
+    long long n = ((width + 1) / 2 + 15) / 16 * 16;
+    if (n > lmhead::kNMax) n = lmhead::kNMax;
+    if (n < 16) n = 16;
+    if (g_lmhead_tile_cols > 0) {
+        n = g_lmhead_tile_cols;
+        per = (V + pairs * 2 * n - 1) / (pairs * 2 * n);
+    }
+    pl.n_tile = static_cast<int>(n);
+    pl.tiles_total = static_cast<int>((V + 2 * n - 1) / (2 * n));
+    pl.tiles_per_cta = static_cast<int>(per);
+    long long used = (pl.tiles_total + per - 1) / per;
+    pl.grid = static_cast<int>(2 * (used < 1 ? 1 : used));
+    const size_t rows = static_cast<size_t>(B) * (K + 1);
+    const size_t groups = (rows + lmhead::kRowsMax - 1) / lmhead::kRowsMax;
+    const size_t rows_last = rows - (groups - 1) * lmhead::kRowsMax;
+    pl.rows2 = static_cast<int>(((rows_last + 1) / 2 + 7) / 8 * 8);                 // rows per CTA in the last group
+    pl.rows1 = pl.rows2;
+    const int half_most = groups > 1 ? lmhead::kMTile : pl.rows2;
+    pl.a_bytes = half_most * lmhead::kRowBytes;                                      // a multiple of 1 KiB: 8 rows
+    pl.sub_bytes = pl.a_bytes + pl.n_tile * lmhead::kRowBytes;                       // + two sub-tiles of n_tile / 2 rows
+    const int fixed = 1024 + lmhead::kBarrierBytes + lmhead::kSlackBytes;
+    pl.kps = 1;
+    int stages = (lmhead::kSmemLimit - fixed) / pl.sub_bytes;
+    pl.n_stages = stages > lmhead::kMaxStages ? lmhead::kMaxStages : stages;
+    pl.smem_bytes = fixed + pl.n_stages * pl.sub_bytes;
+    lmhead_place_workspace(pl, rows, B, K);
+    return pl;
+}
+
+// Pairs pay when the hidden rows are a large part of what a k-block brings into shared memory.
+bool lmhead_wants_pair(int B, int K)
+{
+    if (sm_count() < 2) return false;
+    if (g_lmhead_pairing == 1) return false;
+    if (g_lmhead_pairing == 2) return true;
+    return static_cast<long long>(B) * (K + 1) > lmhead::kMTile;
+}
+
+LmheadPlan lmhead_plan(int B, int K, int H, int V)
+{
+    return lmhead_wants_pair(B, K) ? lmhead_plan_pair(B, K, H, V) : lmhead_plan_lone(B, K, H, V);
+}
+
+// What a workspace must hold whichever kernel runs.
+size_t lmhead_workspace_most(int B, int K, int H, int V)
+{
+    const size_t a = lmhead_plan_lone(B, K, H, V).total;
+    const size_t b = sm_count() >= 2 ? lmhead_plan_pair(B, K, H, V).total : 0;
+    return a > b ? a : b;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
@@ -936,7 +1014,7 @@ EncodeTiledFn encode_tiled_fn()
 
 // A [rows, cols] row-major bf16 matrix as a tensor map whose box is box_rows x 64 columns, 128-byte swizzle;
 // elements outside the matrix read as zero.
-bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool wide_fetch = false)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
@@ -945,7 +1023,8 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, 
     const cuuint32_t box[2] = {static_cast<cuuint32_t>(lmhead::kBlockK), box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              wide_fetch ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -977,7 +1056,9 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
         std::lock_guard<std::mutex> lock(attr_mutex);
         if (!attr_set[dev]) {
             if (cudaFuncSetAttribute(lmhead::lmhead_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lmhead::kSmemLimit) !=
-                cudaSuccess) {
+                    cudaSuccess ||
+                cudaFuncSetAttribute(lmhead::lmhead_stats_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     lmhead::kSmemLimit) != cudaSuccess) {
                 (void)cudaGetLastError();
                 return CSD_ERR_CUDA;
             }
@@ -986,8 +1067,10 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     }
     CUtensorMap map_h, map_h2, map_w;
     if (!make_map(&map_h, hidden, static_cast<uint64_t>(R), static_cast<uint64_t>(H), lmhead::kMTile) ||
-        !make_map(&map_h2, hidden, static_cast<uint64_t>(R), static_cast<uint64_t>(H), static_cast<uint32_t>(pl.rows2 ? pl.rows2 : 8)) ||
-        !make_map(&map_w, weight, static_cast<uint64_t>(V), static_cast<uint64_t>(H), static_cast<uint32_t>(pl.n_tile)))
+        !make_map(&map_h2, hidden, static_cast<uint64_t>(R), static_cast<uint64_t>(H),
+                  static_cast<uint32_t>(pl.rows2 ? pl.rows2 : pl.rows1)) ||
+        !make_map(&map_w, weight, static_cast<uint64_t>(V), static_cast<uint64_t>(H),
+                  static_cast<uint32_t>(pl.pair ? pl.n_tile / 2 : pl.n_tile), g_lmhead_wide_fetch != 0))
         return CSD_ERR_CUDA;
 
     char *ws = static_cast<char *>(workspace);
@@ -997,6 +1080,7 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     p.n_tile = pl.n_tile;
     p.tiles_total = pl.tiles_total;
     p.tiles_per_cta = pl.tiles_per_cta;
+    p.rows1 = pl.rows1;
     p.rows2 = pl.rows2;
     p.a_bytes = pl.a_bytes;
     p.sub_bytes = pl.sub_bytes;
@@ -1006,8 +1090,32 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     p.partials = reinterpret_cast<Partial *>(ws + pl.partials_off);
     p.zd = reinterpret_cast<float *>(ws + pl.zd_off);
     p.stats = ocm->stats;
-    lmhead::lmhead_stats_kernel<<<pl.grid, lmhead::kThreads, pl.smem_bytes, st>>>(map_h, map_h2, map_w, p);
-    if (cudaGetLastError() != cudaSuccess) return CSD_ERR_CUDA;
+    {
+        // Launched programmatically: behind this library's own update kernel (which lets its dependents in at once) the
+        // GEMM of this step streams W while the decisions and the update of the step before finish; it waits for them
+        // before its first store.  Behind any other kernel this is an ordinary launch.
+        cudaLaunchConfig_t cfg;
+        std::memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = dim3(static_cast<unsigned int>(pl.grid));
+        cfg.blockDim = dim3(lmhead::kThreads);
+        cfg.dynamicSmemBytes = static_cast<size_t>(pl.smem_bytes);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 2;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pl.pair ? 2 : 1;
+        const cudaError_t err = pl.pair ? cudaLaunchKernelEx(&cfg, lmhead::lmhead_stats_pair_kernel, map_h, map_h2, map_w, p)
+                                        : cudaLaunchKernelEx(&cfg, lmhead::lmhead_stats_kernel, map_h, map_h2, map_w, p);
+        if (err != cudaSuccess) {
+            (void)cudaGetLastError();
+            return CSD_ERR_CUDA;
+        }
+    }
 
     lmhead::FinalizeParams f;
     std::memset(&f, 0, sizeof f);
@@ -1023,8 +1131,8 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     {
         cudaLaunchConfig_t cfg;
         std::memset(&cfg, 0, sizeof cfg);
-        cfg.gridDim = dim3(static_cast<unsigned int>((B + 3) / 4));
-        cfg.blockDim = dim3(128);
+        cfg.gridDim = dim3(static_cast<unsigned int>(B));
+        cfg.blockDim = dim3(32 * lmhead::kFinalizeWarps);
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1045,7 +1153,7 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
 size_t csd_lmhead_workspace_bytes(int B, int K, int H, int V)
 {
     if (!lmhead_shape_ok(B, K, H, V)) return 0;
-    return lmhead_plan(B, K, H, V).total;
+    return lmhead_workspace_most(B, K, H, V);
 }
 
 csd_status_t csd_verify_lmhead(const void *hidden, const void *weight, int B, int K, int H, int V, const int32_t *draft,
@@ -1065,11 +1173,25 @@ csd_status_t csd_step_lmhead(const void *hidden, const void *weight, int B, int 
                       diag, workspace, workspace_bytes, stream, true);
 }
 
-csd_status_t csd_lmhead_set_tuning(int kblocks_per_stage)
+csd_status_t csd_lmhead_set_tuning(int kblocks_per_stage, int mma_cols)
 {
     if (kblocks_per_stage < 0 || kblocks_per_stage > 4) return CSD_ERR_INVALID_ARG;
+    if (mma_cols != 0 && (mma_cols < 16 || mma_cols > lmhead::kNMax || mma_cols % 16 != 0)) return CSD_ERR_INVALID_ARG;
     g_lmhead_kblocks_per_stage = kblocks_per_stage;
+    g_lmhead_tile_cols = mma_cols;
     return CSD_OK;
+}
+
+csd_status_t csd_lmhead_set_pairing(int mode)
+{
+    if (mode < 0 || mode > 2) return CSD_ERR_INVALID_ARG;
+    g_lmhead_pairing = mode;
+    return CSD_OK;
+}
+
+int csd_lmhead_uses_pairs(int B, int K)
+{
+    return (B > 0 && K > 0 && lmhead_wants_pair(B, K)) ? 1 : 0;
 }
 
 csd_status_t csd_lmhead_shape(int B, int K, int H, int V, int *grid, int *tile_cols, int *tiles, int *tiles_per_block)
@@ -1077,7 +1199,7 @@ csd_status_t csd_lmhead_shape(int B, int K, int H, int V, int *grid, int *tile_c
     if (!lmhead_shape_ok(B, K, H, V)) return CSD_ERR_UNSUPPORTED;
     const LmheadPlan pl = lmhead_plan(B, K, H, V);
     if (grid) *grid = pl.grid;
-    if (tile_cols) *tile_cols = pl.n_tile;
+    if (tile_cols) *tile_cols = pl.pair ? 2 * pl.n_tile : pl.n_tile;
     if (tiles) *tiles = pl.tiles_total;
     if (tiles_per_block) *tiles_per_block = pl.tiles_per_cta;
     return CSD_OK;

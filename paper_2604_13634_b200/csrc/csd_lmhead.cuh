@@ -41,9 +41,9 @@ constexpr int kNMax = 256;                  // widest vocabulary tile
 constexpr int kThreads = 320;                // warp 0 loads, warp 1 issues MMAs, warps 2..5 / 6..9 reduce the first / second row tile
 constexpr int kRowBytes = kBlockK * 2;      // one row of a k-block
 constexpr int kBarrierBytes = 1024;
-// The second row tile's operand is read as 128 rows although only the rows that exist are loaded: the read
-// runs on into whatever follows (the stage's W tile, the next stage, or this slack), which only feeds
-// accumulator rows that nobody reads.
+// A row tile's operand is read as 128 rows although only the rows that exist are loaded: the read runs on into
+// whatever follows (the stage's W tile, the next stage, or this slack), which only feeds accumulator rows that
+// nobody reads.
 constexpr int kSlackBytes = kMTile * kRowBytes;
 constexpr int kSmemLimit = 226 * 1024;      // of the 227 KiB a block may have (some is static)
 constexpr int kTmemCols = 512;
@@ -54,6 +54,7 @@ struct Params {
     int n_tile;             // columns of a vocabulary tile: multiple of 16, at most kNMax
     int tiles_total;        // ceil(V / n_tile)
     int tiles_per_cta;
+    int rows1;              // rows loaded for the first row tile of the LAST row group: 128, or the rows it has rounded up to 8
     int rows2;              // rows loaded for the second row tile of the LAST row group (0 if it has <= 128 rows), a multiple of 8
     int a_bytes;            // bytes of a hidden k-block in a stage (both row tiles), a multiple of 1 KiB
     int sub_bytes;          // a_bytes + the W tile's k-block, a multiple of 1 KiB
@@ -290,7 +291,9 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
                 const bool last_group = g == n_groups - 1;
                 // the second row tile: 128 rows in a full group, the rows that exist (rounded up to 8) in the last one
                 const int rows2 = rows > kMTile ? (last_group ? p.rows2 : kMTile) : 0;
-                const unsigned int tx = static_cast<unsigned int>(kps * (kMTile + rows2 + p.n_tile) * kRowBytes);
+                // the first: 128 rows, or in a last group of fewer only those (map_hidden2's box is then this one)
+                const int rows1 = last_group ? p.rows1 : kMTile;
+                const unsigned int tx = static_cast<unsigned int>(kps * (rows1 + rows2 + p.n_tile) * kRowBytes);
                 for (int t = tile0; t < tile1 && !*give_up; ++t) {
                     const int v0 = t * p.n_tile;
                     for (int ks = 0; ks < k_steps; ++ks, ++it) {
@@ -300,7 +303,7 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
                         for (int sub = 0; sub < kps; ++sub) {
                             const unsigned int a = stages + s * stage_bytes + sub * sub_bytes, b = a + a_bytes;
                             const int x = (ks * kps + sub) * kBlockK;
-                            tma_load_2d(a, &map_hidden, full_bar(s), x, g * kRowsMax);
+                            tma_load_2d(a, rows1 == kMTile ? &map_hidden : &map_hidden2, full_bar(s), x, g * kRowsMax);
                             if (rows2 == kMTile)
                                 tma_load_2d(a + kMTile * kRowBytes, &map_hidden, full_bar(s), x, g * kRowsMax + kMTile);
                             else if (rows2 > 0)
@@ -410,6 +413,9 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
                 tc_fence_before();
                 mbar_arrive(tmem_empty);
             }
+            // the partials of the step before may still be being read: this grid may have started ahead of the end of the
+            // kernels before it on the stream, and waits for them here, ahead of its first store
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             if (has) {
                 float s0, s1, s2, s3;
                 unpack2(rr.acc0, s0, s1);
@@ -444,6 +450,289 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
     }
 }
 
+// ---- the same reduction by PAIRS of CTAs (thread-block clusters of two, tcgen05 cta_group::2) -------------------
+//
+// Two SMs work on one vocabulary tile: the pair's MMA has M = 256, each CTA holding HALF of a row group's rows (128
+// each in a full group; the last group's rows are split evenly, rounded up to 8) in its shared memory and their
+// accumulators in its tensor memory, and each CTA brings in only half of every W tile -- the pair's MMA reads both
+// halves.  A CTA's tensor memory then holds its rows against 2 N <= 512 columns (two MMAs per k-step, accumulators at
+// columns 0 and 256), twice the width a lone CTA can hold for 256 rows, so the hidden states, which are read again for
+// every vocabulary tile, are spread over twice as many columns: a k-block costs an SM (rows / 2 + N) x 128 bytes of
+// shared-memory traffic instead of (rows + N) x 128.
+//   both CTAs   warp 0: TMA loads of the CTA's own operands (cp.async.bulk.tensor with cta_group::2: the bytes are
+//               counted on CTA 0's "full" barrier); warps 2..9: epilogue on the CTA's own tensor memory (warps 2..5
+//               columns [0, N) of the tile, warps 6..9 columns [N, 2N)), one arrival per warp on CTA 0's "accumulators
+//               drained" barrier
+//   CTA 0 only  warp 1: issues the pair's MMAs; its commits arrive on the "stage empty" and "accumulators full"
+//               barriers of BOTH CTAs (tcgen05.commit with a CTA mask: barrier arrivals, no data is moved)
+// Partials: one per (pair, column half) and row, slot 2 * pair + half.  Bounded waits as above (debug_site 31); the two
+// CTAs meet at a cluster barrier before the first signal crosses and before the tensor memory is freed.
+constexpr unsigned int kPeerMask = 0xFEFFFFFFu;       // a shared-memory address with this mask applied is CTA 0's copy of it
+
+__device__ __forceinline__ unsigned int cluster_rank()
+{
+    unsigned int r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(unsigned int dst, const CUtensorMap *map, unsigned int bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+                 "l"(map), "r"(bar & kPeerMask), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(unsigned int d_tmem, unsigned long long a_desc, unsigned long long b_desc, unsigned int idesc,
+                                                 unsigned int accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+                 "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+                 : "memory");
+}
+// Arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far are complete.
+__device__ __forceinline__ void tc_commit_pair(unsigned int bar)
+{
+    const unsigned short both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"(both)
+                 : "memory");
+}
+// One arrival on CTA 0's copy of a barrier, from either CTA.
+__device__ __forceinline__ void mbar_arrive_cta0(unsigned int bar)
+{
+    asm volatile("{\n\t.reg .b32 remote;\n\tmapa.shared::cluster.u32 remote, %0, 0;\n\tmbarrier.arrive.release.cluster.shared::cluster.b64 _, [remote];\n\t}" ::"r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ unsigned int instr_desc_pair(int n)
+{
+    // as instr_desc, M = 256 over the two CTAs
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<unsigned int>(n >> 3) << 17) | (static_cast<unsigned int>(256 >> 4) << 24);
+}
+
+// Params as for the lone-CTA kernel, read this way: n_tile = N, the columns of one MMA (a tile of the pair has 2 N);
+// tiles_per_cta = tiles per pair; rows2 = rows per CTA in the last row group (a multiple of 8, at most 128; map_hidden2's
+// box); a_bytes = a CTA's hidden k-block; sub_bytes = a stage: a_bytes + two half W sub-tiles of N / 2 rows each.
+__global__ void __launch_bounds__(kThreads, 1)
+lmhead_stats_pair_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_hidden2,
+                         const __grid_constant__ CUtensorMap map_weight, const Params p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ unsigned int tmem_base_slot;
+    __shared__ int give_up_flag;
+    volatile int *give_up = &give_up_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int rank = static_cast<int>(cluster_rank());      // 0 issues the MMAs
+    const int pair = blockIdx.x >> 1;
+    const unsigned int raw = smem_u32(smem_raw);
+    const unsigned int bars = (raw + 1023u) & ~1023u;
+    const unsigned int stages = bars + kBarrierBytes;
+    const int n_stages = p.n_stages;
+    const int a_bytes = p.a_bytes, stage_bytes = p.sub_bytes;
+    const int half_bytes = (stage_bytes - a_bytes) / 2;      // this CTA's half of one W sub-tile
+    const int N = p.n_tile;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kMaxStages + s); };
+    const unsigned int tmem_full = bars + 8u * (2 * kMaxStages);
+    const unsigned int tmem_empty = bars + 8u * (2 * kMaxStages + 1);
+
+    const int n_groups = (p.R + kRowsMax - 1) / kRowsMax;
+    const int kblocks = p.H / kBlockK;
+    const int tile0 = pair * p.tiles_per_cta;
+    int tile1 = tile0 + p.tiles_per_cta;
+    if (tile1 > p.tiles_total) tile1 = p.tiles_total;
+    const int my_tiles = tile1 > tile0 ? tile1 - tile0 : 0;
+    // rows a CTA holds of group g: CTA 0 rows [256 g, + half), CTA 1 rows [256 g + half, + half)
+    auto half_of = [&](int g) { return g == n_groups - 1 ? p.rows2 : kMTile; };
+
+    if (threadIdx.x == 0) {
+        give_up_flag = 0;
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        mbar_init(tmem_full, 1);
+        mbar_init(tmem_empty, 2 * 8);                        // one arrival per epilogue warp of both CTAs
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                      // both CTAs' barriers exist before a signal crosses
+    tc_fence_after();
+    const unsigned int tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // ---- loader (both CTAs) ----
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int g = 0; g < n_groups && ok && !*give_up; ++g) {
+                const int half = half_of(g);
+                const bool full_group = half == kMTile && g != n_groups - 1;
+                const unsigned int tx_pair = static_cast<unsigned int>((2 * half + 2 * N) * kRowBytes);      // the bytes of both CTAs
+                const int row0 = g * kRowsMax + rank * half;
+                for (int t = tile0; t < tile1 && ok && !*give_up; ++t) {
+                    const int v0 = t * 2 * N + rank * (N / 2);
+                    for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                        const int s = it % n_stages;
+                        if (!mbar_wait(empty_bar(s), ((it / n_stages) & 1) ^ 1, give_up)) {
+                            ok = false;
+                            break;
+                        }
+                        if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
+                        const unsigned int a = stages + s * stage_bytes, b0 = a + a_bytes, b1 = b0 + half_bytes;
+                        const int x = kb * kBlockK;
+                        tma_load_2d_pair(a, full_group ? &map_hidden : &map_hidden2, full_bar(s), x, row0);
+                        tma_load_2d_pair(b0, &map_weight, full_bar(s), x, v0);           // W rows [v0, + N / 2) of the first N columns
+                        tma_load_2d_pair(b1, &map_weight, full_bar(s), x, v0 + N);       // and of the second N
+                    }
+                }
+            }
+            // every commit aimed at this CTA's "empty" barriers has landed before the CTA goes on towards its end
+            for (int k = 0; k < n_stages && ok; ++k, ++it) ok = mbar_wait(empty_bar(it % n_stages), ((it / n_stages) & 1) ^ 1, give_up);
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer (CTA 0 of the pair) ----
+        if (lane == 0 && rank == 0) {
+            const unsigned int idesc = instr_desc_pair(N);
+            int it = 0, tt = 0;
+            bool ok = true;
+            for (int g = 0; g < n_groups && ok && !*give_up; ++g) {
+                for (int t = 0; t < my_tiles && ok && !*give_up; ++t, ++tt) {
+                    if (!mbar_wait(tmem_empty, (tt & 1) ^ 1, give_up)) {      // both CTAs have drained the previous tile
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                        const int s = it % n_stages;
+                        if (!mbar_wait(full_bar(s), (it / n_stages) & 1, give_up)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        const unsigned int a = stages + s * stage_bytes, b0 = a + a_bytes, b1 = b0 + half_bytes;
+                        const unsigned long long a_desc = operand_desc(a), b0_desc = operand_desc(b0), b1_desc = operand_desc(b1);
+#pragma unroll
+                        for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
+                            const unsigned int acc = (kb | k4) != 0 ? 1u : 0u;
+                            tc_mma_bf16_pair(tmem_base, a_desc + 2ull * k4, b0_desc + 2ull * k4, idesc, acc);
+                            tc_mma_bf16_pair(tmem_base + kNMax, a_desc + 2ull * k4, b1_desc + 2ull * k4, idesc, acc);
+                        }
+                        tc_commit_pair(empty_bar(s));
+                    }
+                    if (ok) tc_commit_pair(tmem_full);
+                }
+            }
+        }
+    } else {
+        // ---- epilogue (both CTAs): warps 2..5 the tile's first N columns, warps 6..9 its second N; a thread owns one
+        // logit row of its CTA for one column half ----
+        const int q = warp & 3;
+        const int chalf = warp >= 6 ? 1 : 0;
+        const unsigned int lane_base = tmem_base + (static_cast<unsigned int>(32 * q) << 16) + (chalf ? kNMax : 0);
+        int tt = 0;
+        bool ok = true;
+        for (int g = 0; g < n_groups && ok; ++g) {
+            const int half = half_of(g);
+            const int row = g * kRowsMax + rank * half + 32 * q + lane;
+            const bool has = 32 * q + lane < half && row < p.R;
+            const bool warp_has = 32 * q < half && g * kRowsMax + rank * half + 32 * q < p.R;
+            RowRun rr;
+            row_init(rr);
+            int d = -1;
+            if (has) {
+                const int b = row / (p.K + 1), i = row - b * (p.K + 1);
+                if (i < p.K) d = __ldg(p.draft + b * p.K + i);
+            }
+            float zd = 0.f;
+            bool got = false;
+            for (int t = 0; t < my_tiles; ++t, ++tt) {
+                if (!mbar_wait(tmem_full, tt & 1, give_up)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const int v0 = (tile0 + t) * 2 * N + chalf * N;
+                const int v_end = min(p.V, v0 + N);
+                if (warp_has) {
+                    for (int c0 = 0; c0 < N; c0 += 64) {
+                        const int vc = v0 + c0;
+                        if (vc >= v_end) break;
+                        const bool second = c0 + 32 < N && vc + 32 < v_end;
+                        float x[32], y[32];
+                        if (second)
+                            tmem_ld64(lane_base + c0, x, y);
+                        else
+                            tmem_ld32(lane_base + c0, x);
+                        auto take = [&](float (&v)[32], int vb) {
+                            if (vb + 32 > v_end) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) v[j] = (vb + j < v_end) ? v[j] : -INFINITY;
+                            }
+                            if (has) {
+                                row_take(rr, v, vb);
+                                if (static_cast<unsigned int>(d - vb) < 32u && d < v_end) {
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) zd = (d - vb == j) ? v[j] : zd;
+                                    got = true;
+                                }
+                            }
+                        };
+                        take(x, vc);
+                        if (second) take(y, vc + 32);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cta0(tmem_empty);
+            }
+            // the partials of the step before may still be being read: this grid may have started ahead of the end of the
+            // kernels before it on the stream, and waits for them here, ahead of its first store
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            if (has) {
+                float s0, s1, s2, s3;
+                unpack2(rr.acc0, s0, s1);
+                unpack2(rr.acc1, s2, s3);
+                Partial out;
+                out.m = rr.m;
+                out.idx = rr.idx;
+                out.c = rr.c;
+                out.s = (s0 + s1) + (s2 + s3);
+                st_partial_cg(p.partials + static_cast<size_t>(row) * gridDim.x + 2 * pair + chalf, out);
+                if (got) {
+                    const int b = row / (p.K + 1), i = row - b * (p.K + 1);
+                    __stcg(p.zd + b * p.K + i, zd);
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*give_up) {
+        if (threadIdx.x == 0) index_check_failed(p.stats, 31u);
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000ll) {
+        }
+        __syncthreads();
+    }
+    cluster_sync_all();                                      // no signal is on its way to a CTA that has left; the pair frees together
+    if (warp == 2) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
 // ---- S1 (last level) and S2..S5 per batch row, from the partials of the LM-head kernel ----------------
 struct FinalizeParams {
     int B, K, V, n_parts;
@@ -460,32 +749,42 @@ struct FinalizeParams {
     csd_diag_t diag;
 };
 
-__global__ void __launch_bounds__(128) lmhead_finalize_kernel(const FinalizeParams p)
+constexpr int kFinalizeWarps = 8;
+
+// One block per batch row.  Its warps fold the partials of the row's K + 1 logit rows (a warp per logit row, all
+// loads of a round in flight together: the fold costs a few memory latencies, not one per partial); warp 0 then takes
+// the decisions.
+__global__ void __launch_bounds__(32 * kFinalizeWarps) lmhead_finalize_kernel(const FinalizeParams p)
 {
-    __shared__ float sm_m[4][CSD_MAX_K + 1], sm_s[4][CSD_MAX_K + 1];
-    __shared__ int sm_t[4][CSD_MAX_K + 1];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int b = blockIdx.x * 4 + w;
+    __shared__ float sm_m[1][CSD_MAX_K + 1], sm_s[1][CSD_MAX_K + 1];
+    __shared__ int sm_t[1][CSD_MAX_K + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int w = 0;
+    const int b = blockIdx.x;
     // launched programmatically behind the GEMM kernel: let the memory's update kernel in, then wait for the GEMM
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (b >= p.B) return;
     const int K = p.K, K1 = K + 1;
     // the draft tokens and their logits do not depend on the fold: requested first
     int d = -1;
     bool valid = false;
     float zd = __int_as_float(0x7fc00000);
-    if (lane < K) {
+    if (warp == 0 && lane < K) {
         d = __ldg(p.draft + (size_t)b * K + lane);
         valid = static_cast<unsigned int>(d) < static_cast<unsigned int>(p.V);
         if (valid) zd = __ldcg(p.zd + (size_t)b * K + lane);
     }
-    for (int i = 0; i < K1; ++i) {
+    for (int i = warp; i < K1; i += kFinalizeWarps) {
         const Partial *src = p.partials + (static_cast<size_t>(b) * K1 + i) * p.n_parts;
         Partial v = partial_identity();
-        for (int k = lane; k < p.n_parts; k += 32) {          // lane k folds parts k, k + 32, ... in order
-            const Partial x = ld_partial_cg(src + k);
-            v = (k == lane) ? x : combine(v, x);
+        for (int k0 = lane; k0 < p.n_parts; k0 += 128) {      // lane k folds parts k, k + 32, ... in order, four loads at a time
+            Partial x[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (k0 + 32 * j < p.n_parts) x[j] = ld_partial_cg(src + k0 + 32 * j);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (k0 + 32 * j < p.n_parts) v = (k0 + 32 * j == lane) ? x[j] : combine(v, x[j]);
         }
         // fixed-shape butterfly: maximum and its lowest index, then the sums rescaled (exactly) to its reference
         float m = v.m;
@@ -506,6 +805,8 @@ __global__ void __launch_bounds__(128) lmhead_finalize_kernel(const FinalizePara
             sm_t[w][i] = idx;
         }
     }
+    __syncthreads();
+    if (warp != 0) return;
     __syncwarp();
     for (int row = lane; row <= K; row += 32) {
         const size_t at = (size_t)b * K1 + row;

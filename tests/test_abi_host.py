@@ -134,10 +134,19 @@ def test_plans_of_the_other_entry_points(L):
         else:
             assert L.csd_early_exit_workspace_bytes(B, K, V, dt, 0) == 0
     g, n, t, per = (ctypes.c_int() for _ in range(4))
-    for (B, K, H, V) in ((32, 5, 4096, 151936), (64, 6, 4096, 152064), (128, 8, 4096, 128256), (1, 1, 64, 17), (2, 3, 128, 1000)):
-        assert L.csd_lmhead_shape(B, K, H, V, ctypes.byref(g), ctypes.byref(n), ctypes.byref(t), ctypes.byref(per)) == 0
-        assert 1 <= g.value <= 148 and n.value % 16 == 0 and 16 <= n.value <= 256
-        assert t.value == -(-V // n.value) and g.value * per.value >= t.value and (g.value - 1) * per.value < t.value
-        assert L.csd_lmhead_workspace_bytes(B, K, H, V) >= B * (K + 1) * g.value * 16 + 4 * B * K
+    L.csd_lmhead_set_pairing.argtypes, L.csd_lmhead_set_pairing.restype = [ctypes.c_int], ctypes.c_int
+    assert L.csd_lmhead_set_pairing(3) != 0 and L.csd_lmhead_set_pairing(-1) != 0
+    try:
+        for mode in (1, 2):                              # one block per SM; pairs of blocks, a pair's tile twice as wide
+            assert L.csd_lmhead_set_pairing(mode) == 0
+            for (B, K, H, V) in ((32, 5, 4096, 151936), (64, 6, 4096, 152064), (128, 8, 4096, 128256), (1, 1, 64, 17), (2, 3, 128, 1000)):
+                assert L.csd_lmhead_shape(B, K, H, V, ctypes.byref(g), ctypes.byref(n), ctypes.byref(t), ctypes.byref(per)) == 0
+                owners = g.value // mode                 # blocks or pairs: each owns `per` consecutive tiles
+                assert 1 <= g.value <= 148 and g.value % mode == 0
+                assert n.value % (16 * mode) == 0 and 16 * mode <= n.value <= 256 * mode
+                assert t.value == -(-V // n.value) and owners * per.value >= t.value and (owners - 1) * per.value < t.value
+                assert L.csd_lmhead_workspace_bytes(B, K, H, V) >= B * (K + 1) * g.value * 16 + 4 * B * K
+    finally:
+        L.csd_lmhead_set_pairing(0)
     assert L.csd_lmhead_workspace_bytes(2, 3, 100, 1000) == 0            # H must be a multiple of 64
     assert L.csd_lmhead_shape(2, 33, 128, 1000, None, None, None, None) != 0

@@ -13,10 +13,19 @@ import pytest
 import torch
 
 from oracle import csd_lmhead_oracle as ORACLE
-from paper_2604_13634_b200 import LmheadBuffers, Ocm, csd_lmhead_shape, csd_step_lmhead, csd_verify_lmhead
+from paper_2604_13634_b200 import (LmheadBuffers, Ocm, csd_lmhead_set_pairing, csd_lmhead_shape, csd_step_lmhead,
+                                   csd_verify_lmhead)
 from synth_inputs import WORKLOADS, Synth
 
 pytestmark = pytest.mark.gpu
+
+KERNELS = {"lone": 1, "pairs": 2}        # one block per SM / clusters of two blocks (csd_lmhead_set_pairing)
+
+
+@pytest.fixture(autouse=True)
+def _automatic_kernel_choice_afterwards():
+    yield
+    csd_lmhead_set_pairing(0)
 
 
 def _f64(t):
@@ -100,19 +109,24 @@ def lockstep(wl, H, steps, tau, lam, seed=0):
 
 SMALL = [(2, 3, 64, 96), (1, 1, 128, 1000), (5, 4, 256, 5000), (16, 7, 512, 4099), (7, 32, 128, 777), (32, 5, 1024, 20000),
          (42, 5, 320, 33000),      # 252 rows, two row tiles
-         (64, 6, 256, 9000), (50, 8, 192, 5000), (128, 8, 128, 3000)]      # 448, 450 and 1152 rows: two to five row groups
+         (64, 6, 256, 9000), (50, 8, 192, 5000), (128, 8, 128, 3000),      # 448, 450 and 1152 rows: two to five row groups
+         (30, 9, 128, 2000)]                                               # 300 rows: a last group of 44
 
 
+@pytest.mark.parametrize("kernel", list(KERNELS))
 @pytest.mark.parametrize("B,K,H,V", SMALL)
-def test_small_shapes(B, K, H, V):
+def test_small_shapes(B, K, H, V, kernel):
+    csd_lmhead_set_pairing(KERNELS[kernel])
     wl = dataclasses.replace(WORKLOADS["batched_serving"], B=B, K=K, V=V, n_pairs=min(5000, V // 2), ocm_slots=4096)
     out = lockstep(wl, H, 4, 0.3, 1)
     assert out["excused"] <= max(1, B // 8), out
     print((B, K, H, V), csd_lmhead_shape(B, K, H, V), out)
 
 
-def test_batched_serving_shape_with_a_llm_sized_head():
+@pytest.mark.parametrize("kernel", ["automatic"] + list(KERNELS))
+def test_batched_serving_shape_with_a_llm_sized_head(kernel):
     """The serving workload with H = 4096: 192 logit rows, 151 936 tokens, a 1.2 GB weight matrix."""
+    csd_lmhead_set_pairing(KERNELS.get(kernel, 0))
     wl = WORKLOADS["batched_serving"]
     out = lockstep(wl, 4096, 4, 0.3, 2)
     assert out["rescued"] > 0 and out["excused"] <= 2, out
@@ -123,17 +137,35 @@ def test_batched_serving_shape_with_a_llm_sized_head():
 def test_more_k_blocks_per_stage(kps):
     from paper_2604_13634_b200 import csd_lmhead_set_tuning
     try:
-        csd_lmhead_set_tuning(kps)
+        csd_lmhead_set_tuning(kps, 0)
         for (B, K, H, V) in ((16, 7, 512, 4099), (42, 5, 256, 33000), (64, 6, 256, 9000)):
             wl = dataclasses.replace(WORKLOADS["batched_serving"], B=B, K=K, V=V, n_pairs=min(5000, V // 2), ocm_slots=4096)
             out = lockstep(wl, H, 3, 0.3, 1)
             assert out["excused"] <= max(1, B // 8), out
     finally:
-        csd_lmhead_set_tuning(0)
+        csd_lmhead_set_tuning(0, 0)
 
 
-def test_verify_is_read_only_reproducible_and_checks_its_arguments():
+@pytest.mark.parametrize("kernel", list(KERNELS))
+def test_other_mma_widths(kernel):
+    """Tile widths other than the automatic cut: narrow, odd multiples of 16, the widest; ragged last tiles."""
+    from paper_2604_13634_b200 import csd_lmhead_set_tuning
+    csd_lmhead_set_pairing(KERNELS[kernel])
+    try:
+        for cols in (16, 48, 112, 256):
+            csd_lmhead_set_tuning(0, cols)
+            for (B, K, H, V) in ((5, 4, 256, 5000), (42, 5, 128, 33000), (50, 8, 192, 5000)):
+                wl = dataclasses.replace(WORKLOADS["batched_serving"], B=B, K=K, V=V, n_pairs=min(5000, V // 2), ocm_slots=4096)
+                out = lockstep(wl, H, 2, 0.3, 1)
+                assert out["excused"] <= max(1, B // 8), out
+    finally:
+        csd_lmhead_set_tuning(0, 0)
+
+
+@pytest.mark.parametrize("kernel", list(KERNELS))
+def test_verify_is_read_only_reproducible_and_checks_its_arguments(kernel):
     from paper_2604_13634_b200 import CsdError
+    csd_lmhead_set_pairing(KERNELS[kernel])
     wl = dataclasses.replace(WORKLOADS["batched_serving"], B=4, V=8192, n_pairs=2000)
     syn = Synth(wl, 3, "cuda")
     W = syn.lmhead_weight(256)
