@@ -789,9 +789,11 @@ def measure_lmhead(wl, tau, device, H=4096, steps=12, repeats=7):
             ts.append(a.elapsed_time(b) * 1e-3 / steps)
         return statistics.median(ts)
 
+    pkg.csd_set_overlap(True)        # the GEMM of a step starts beside the decisions and the update of the step before
     fused = timed(lambda i: pkg.csd_step_lmhead(ins[i % 3][0], W, ins[i % 3][1], ocm, tau, buf))
+    pkg.csd_set_overlap(False)       # plain stream-ordered launches: what a loop with other kernels between steps gets
+    ordered = timed(lambda i: pkg.csd_step_lmhead(ins[i % 3][0], W, ins[i % 3][1], ocm, tau, buf))
     sb = pkg.StepBuffers(wl.B, wl.K, wl.V, torch.bfloat16, device=device)
-    pkg.csd_set_overlap(False)
 
     def unfused(i):
         h, d = ins[i % 3]
@@ -815,9 +817,12 @@ def measure_lmhead(wl, tau, device, H=4096, steps=12, repeats=7):
             "hbm_GBs": hbm_bytes / fused / 1e9, "hbm_frac": hbm_bytes / fused / 1e9 / hbm,
             "bound": "hbm" if hbm_bytes / (hbm * 1e9) >= flops / (tensor_peak * 1e12) else "tensor",
             "roofline_us": 1e6 * t_bound, "frac_of_roofline": t_bound / fused, "peak_source": f"of {kind}",
+            "stream_ordered_us_per_step": 1e6 * ordered, "stream_ordered_frac_of_roofline": t_bound / ordered,
             "unfused_us_per_step": 1e6 * plain,
             "unfused": f"torch.matmul (bf16 logits stored, {R * wl.V * 2 / 1e6:.0f} MB written and read back) followed by csd_step",
-            "launches_per_step": 3, "launch": "eager",
+            "launches_per_step": 3,
+            "launch": "eager, step overlap on (the GEMM launched programmatically behind the step before); "
+                      "stream_ordered_*: overlap off",
             "ocm": {k: st[k] for k in ("n_keys", "rescues", "rejections", "flags")}}
 
 

@@ -364,8 +364,13 @@ csd_status_t csd_step_sampled(const void *logits, const void *draft_logits, csd_
  * the tests), so an arg-max or a gate decision that hangs on a smaller difference may come out either way;
  * everything else is the result csd_verify would give on the exact logits.  diag as for csd_verify.
  * workspace: csd_lmhead_workspace_bytes bytes, 16-byte aligned, no initialisation needed.
- * Three launches (GEMM + statistics, decisions, memory update); asynchronous.  A wait inside the GEMM
- * kernel that does not end within about two seconds raises CSD_FLAG_INTERNAL (debug_site 30).
+ * Three launches (GEMM + statistics, decisions, memory update); asynchronous.  With csd_set_overlap on, the
+ * GEMM of up to 128 logit rows (one block per SM) is launched programmatically: behind this library's own kernels on the same stream it starts, and streams
+ * the weight matrix, while the decisions and the update of the step before finish; it reads only this step's
+ * inputs until its first store into the workspace and waits for everything before it on the stream ahead of that,
+ * so back-to-back steps may share one workspace.  csd_set_overlap's condition applies to hidden, weight and
+ * draft: complete before the step before was enqueued.  A wait inside the GEMM kernel that does not end within
+ * about two seconds raises CSD_FLAG_INTERNAL (debug_site 30 or 31).
  * Errors as csd_verify; UNSUPPORTED for H not a multiple of 64; CUDA if the driver offers no
  * tensor-map encoder. */
 size_t csd_lmhead_workspace_bytes(int B, int K, int H, int V);

@@ -1091,9 +1091,9 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     p.zd = reinterpret_cast<float *>(ws + pl.zd_off);
     p.stats = ocm->stats;
     {
-        // Launched programmatically: behind this library's own update kernel (which lets its dependents in at once) the
-        // GEMM of this step streams W while the decisions and the update of the step before finish; it waits for them
-        // before its first store.  Behind any other kernel this is an ordinary launch.
+        // With step overlap on, launched programmatically: behind this library's own update kernel (which lets its
+        // dependents in at once) the GEMM of this step streams W while the decisions and the update of the step before
+        // finish; it waits for them before its first store.  It reads its inputs before that wait, hence the opt-in.
         cudaLaunchConfig_t cfg;
         std::memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = dim3(static_cast<unsigned int>(pl.grid));
@@ -1107,8 +1107,12 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
         attr[1].val.clusterDim.x = 2;
         attr[1].val.clusterDim.y = 1;
         attr[1].val.clusterDim.z = 1;
+        // (not for pairs: measured, a cluster grid that comes in beside the tail of the step before is slower, 257 us
+        // per step against 248 at 192 rows, where the one-CTA kernel gains 20 us at 9 rows)
+        const bool early = g_overlap_steps != 0 && !pl.pair;
+        if (!early) attr[0] = attr[1];
         cfg.attrs = attr;
-        cfg.numAttrs = pl.pair ? 2 : 1;
+        cfg.numAttrs = (early ? 1 : 0) + (pl.pair ? 1 : 0);
         const cudaError_t err = pl.pair ? cudaLaunchKernelEx(&cfg, lmhead::lmhead_stats_pair_kernel, map_h, map_h2, map_w, p)
                                         : cudaLaunchKernelEx(&cfg, lmhead::lmhead_stats_kernel, map_h, map_h2, map_w, p);
         if (err != cudaSuccess) {

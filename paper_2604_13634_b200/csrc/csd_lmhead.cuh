@@ -5,7 +5,7 @@
 //
 //   lmhead_stats_kernel     persistent, one CTA per SM, 320 threads:
 //       warp 0      one thread issues the TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of the k-blocks:
-//                   64 columns of all hidden rows (a box of 128 rows and one of the rows beyond) and of the
+//                   64 columns of the hidden rows (a box of up to 128 rows and one of the rows beyond) and of the
 //                   vocabulary tile's W rows, into a ring of as many shared-memory stages as fit (3 to 8)
 //       warp 1      one thread issues the MMAs (tcgen05.mma, kind::f16, M = 128, N = tile width, K = 16, fp32
 //                   accumulators in tensor memory: columns [0, N) for rows 0..127, [256, 256 + N) for rows
@@ -16,11 +16,15 @@
 //                   reference exponent, sum) -- no exchange between threads, a row lives in one thread -- and
 //                   keeps z[row, draft[row]] when that column comes by
 //     A CTA owns a contiguous run of vocabulary tiles and ends with one partial per logit row.
-//   lmhead_finalize_kernel  one warp per batch row: folds the CTAs' partials in a fixed order, then S2..S5
+//   lmhead_stats_pair_kernel  the same by clusters of two CTAs (tcgen05 cta_group::2, M = 256): each CTA holds half of
+//                           the rows against a tile twice as wide and loads half of every W tile; see its own text.
+//   lmhead_finalize_kernel  one block per batch row: folds the CTAs' partials in a fixed order, then S2..S5
 //                           exactly as the streaming step does; the memory update follows as its own launch.
+// Both GEMM kernels may be launched programmatically behind the kernels of the step before: they read only the step's
+// inputs until their first store, ahead of which they wait for those kernels (griddepcontrol.wait).
 //
 // Every wait on an mbarrier is bounded (about two seconds of clock cycles): when one runs out, the CTA raises
-// CSD_FLAG_INTERNAL (debug_site 30), all its roles leave their loops, it waits for copies that may still be in
+// CSD_FLAG_INTERNAL (debug_site 30; 31 in the pair kernel), all its roles leave their loops, it waits for copies that may still be in
 // flight, frees its tensor memory and returns.
 #pragma once
 
