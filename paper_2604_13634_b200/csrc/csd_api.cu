@@ -968,10 +968,56 @@ LmheadPlan lmhead_plan_pair(int B, int K, int /*H*/, int V)
     return pl;
 }
 
+// Once per device: lets both GEMM kernels use the shared memory they need and asks whether the device can hold a
+// cluster of two such blocks at all (it cannot in some partitioned configurations).  -1: a CUDA call failed;
+// 0: no device in this process (planning only); 1: one-CTA kernel only; 2: pairs possible.
+int lmhead_device_state()
+{
+    static std::mutex m;
+    static int state[kMaxLmheadDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    if (dev < 0 || dev >= kMaxLmheadDevices) return -1;
+    std::lock_guard<std::mutex> lock(m);
+    if (state[dev] == 0) {
+        if (cudaFuncSetAttribute(lmhead::lmhead_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lmhead::kSmemLimit) !=
+                cudaSuccess ||
+            cudaFuncSetAttribute(lmhead::lmhead_stats_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 lmhead::kSmemLimit) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return -1;
+        }
+        cudaLaunchConfig_t probe;
+        std::memset(&probe, 0, sizeof probe);
+        probe.gridDim = dim3(2);
+        probe.blockDim = dim3(lmhead::kThreads);
+        probe.dynamicSmemBytes = static_cast<size_t>(lmhead::kSmemLimit);
+        cudaLaunchAttribute cl[1];
+        cl[0].id = cudaLaunchAttributeClusterDimension;
+        cl[0].val.clusterDim.x = 2;
+        cl[0].val.clusterDim.y = 1;
+        cl[0].val.clusterDim.z = 1;
+        probe.attrs = cl;
+        probe.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, lmhead::lmhead_stats_pair_kernel, &probe) != cudaSuccess) {
+            (void)cudaGetLastError();
+            clusters = 0;
+        }
+        state[dev] = clusters >= 1 ? 2 : 1;
+    }
+    return state[dev];
+}
+
 // Pairs pay when the hidden rows are a large part of what a k-block brings into shared memory.
 bool lmhead_wants_pair(int B, int K)
 {
     if (sm_count() < 2) return false;
+    const int dev_state = lmhead_device_state();
+    if (dev_state == 1 || dev_state < 0) return false;
     if (g_lmhead_pairing == 1) return false;
     if (g_lmhead_pairing == 2) return true;
     return static_cast<long long>(B) * (K + 1) > lmhead::kMTile;
@@ -1040,31 +1086,12 @@ csd_status_t run_lmhead(const void *hidden, const void *weight, int B, int K, in
     if (!lmhead_shape_ok(B, K, H, V)) return CSD_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(weight) & 15u)) return CSD_ERR_INVALID_ARG;
     const LmheadPlan pl = lmhead_plan(B, K, H, V);
-    if (workspace_bytes < pl.total || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
+    if (workspace_bytes < lmhead_workspace_most(B, K, H, V) || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CSD_ERR_WORKSPACE;
     chain_break();
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int R = B * (K + 1);
 
-    static std::mutex attr_mutex;
-    static bool attr_set[kMaxLmheadDevices] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxLmheadDevices) {
-        (void)cudaGetLastError();
-        return CSD_ERR_CUDA;
-    }
-    {
-        std::lock_guard<std::mutex> lock(attr_mutex);
-        if (!attr_set[dev]) {
-            if (cudaFuncSetAttribute(lmhead::lmhead_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, lmhead::kSmemLimit) !=
-                    cudaSuccess ||
-                cudaFuncSetAttribute(lmhead::lmhead_stats_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     lmhead::kSmemLimit) != cudaSuccess) {
-                (void)cudaGetLastError();
-                return CSD_ERR_CUDA;
-            }
-            attr_set[dev] = true;
-        }
-    }
+    if (lmhead_device_state() < 0) return CSD_ERR_CUDA;
     CUtensorMap map_h, map_h2, map_w;
     if (!make_map(&map_h, hidden, static_cast<uint64_t>(R), static_cast<uint64_t>(H), lmhead::kMTile) ||
         !make_map(&map_h2, hidden, static_cast<uint64_t>(R), static_cast<uint64_t>(H),

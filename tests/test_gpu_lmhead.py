@@ -117,6 +117,7 @@ SMALL = [(2, 3, 64, 96), (1, 1, 128, 1000), (5, 4, 256, 5000), (16, 7, 512, 4099
 @pytest.mark.parametrize("B,K,H,V", SMALL)
 def test_small_shapes(B, K, H, V, kernel):
     csd_lmhead_set_pairing(KERNELS[kernel])
+    assert csd_lmhead_shape(B, K, H, V)["kernel"] == ("lmhead_stats_pair_kernel" if kernel == "pairs" else "lmhead_stats_kernel")
     wl = dataclasses.replace(WORKLOADS["batched_serving"], B=B, K=K, V=V, n_pairs=min(5000, V // 2), ocm_slots=4096)
     out = lockstep(wl, H, 4, 0.3, 1)
     assert out["excused"] <= max(1, B // 8), out
