@@ -42,6 +42,8 @@ DEFAULT_WORKLOAD = "large_batch"
 # DRAM bytes per launch of the step kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); a workload is absent where no capture of the current kernel exists.
 NCU_TRAFFIC_BYTES = {"large_batch": 596126208, "ocm_contention": 140787712, "batched_serving": 58522880}
+# the same for the LM-head GEMM kernels at H = 4096 (profiles/lmhead_stats_kernel_batched_serving_h4096.md), by workload
+NCU_TRAFFIC_BYTES_LMHEAD = {"batched_serving": 1252566000 + 4133120, "single_stream": 1051026000 + 3639040}
 
 
 def measured_peak():
@@ -817,6 +819,7 @@ def measure_lmhead(wl, tau, device, H=4096, steps=12, repeats=7):
             "hbm_GBs": hbm_bytes / fused / 1e9, "hbm_frac": hbm_bytes / fused / 1e9 / hbm,
             "bound": "hbm" if hbm_bytes / (hbm * 1e9) >= flops / (tensor_peak * 1e12) else "tensor",
             "roofline_us": 1e6 * t_bound, "frac_of_roofline": t_bound / fused, "peak_source": f"of {kind}",
+            "algorithmic_bytes": hbm_bytes, "traffic": NCU_TRAFFIC_BYTES_LMHEAD.get(wl.name) if H == 4096 else None,
             "stream_ordered_us_per_step": 1e6 * ordered, "stream_ordered_frac_of_roofline": t_bound / ordered,
             "unfused_us_per_step": 1e6 * plain,
             "unfused": f"torch.matmul (bf16 logits stored, {R * wl.V * 2 / 1e6:.0f} MB written and read back) followed by csd_step",
@@ -852,7 +855,7 @@ def run_lmhead(args, wl, tau):
                                                 "l2_policy": "the 1.2 GB weight matrix is larger than L2"}),
             "roofline": {"bound": m["bound"], "achieved": m["hbm_GBs"] if m["bound"] == "hbm" else m["tensor_TFLOPs"],
                          "peak": measured_peak()[0] if m["bound"] == "hbm" else None, "unit": "GB/s" if m["bound"] == "hbm" else "TFLOP/s",
-                         "frac": m["frac_of_roofline"], "traffic": None, "peak_source": m["peak_source"],
+                         "frac": m["frac_of_roofline"], "traffic": m["traffic"], "peak_source": m["peak_source"],
                          "kernel": m["shape"]["kernel"], "tensor_TFLOPs": m["tensor_TFLOPs"], "tensor_frac": m["tensor_frac"]},
             "gpu_launches": 3 * m["steps"], "clocks": clocks, "lmhead": m}
     print(json.dumps(line), flush=True)
