@@ -190,6 +190,38 @@ def test_back_to_back_steps_with_step_overlap(shape, kernel):
 
 
 @pytest.mark.parametrize("kernel", list(KERNELS))
+def test_steps_captured_in_a_cuda_graph(kernel):
+    """The three launches of a call can be captured (after one eager call has set the device up) and replayed:
+    same bits as the eager call."""
+    csd_lmhead_set_pairing(KERNELS[kernel])
+    wl = dataclasses.replace(WORKLOADS["batched_serving"], B=24, K=5, V=20000, n_pairs=5000, ocm_slots=4096)
+    syn = Synth(wl, 9, "cuda")
+    W = syn.lmhead_weight(256)
+    ins = [syn.step_lmhead(s, W) for s in range(3)]
+    ocm = Ocm(wl.ocm_slots, 1)
+    eager = [LmheadBuffers(wl.B, wl.K, 256, wl.V, diag=True) for _ in ins]
+    for (h, d), buf in zip(ins, eager):
+        csd_verify_lmhead(h, W, d, ocm, 0.3, buf)
+    torch.cuda.synchronize()
+    replayed = [LmheadBuffers(wl.B, wl.K, 256, wl.V, diag=True) for _ in ins]
+    g, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for (h, d), buf in zip(ins, replayed):
+                csd_verify_lmhead(h, W, d, ocm, 0.3, buf)
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(eager, replayed):
+        for k in ("accept_len", "next_token", "rescued_mask", "rej_draft", "rej_target"):
+            assert torch.equal(getattr(a, k), getattr(b, k)), k
+        for k in a.diag:
+            assert torch.equal(a.diag[k].view(torch.int32), b.diag[k].view(torch.int32)), k
+    assert ocm.stats()["flags"] == 0
+    ocm.close()
+
+
+@pytest.mark.parametrize("kernel", list(KERNELS))
 def test_other_mma_widths(kernel):
     """Tile widths other than the automatic cut: narrow, odd multiples of 16, the widest; ragged last tiles."""
     from paper_2604_13634_b200 import csd_lmhead_set_tuning
