@@ -570,7 +570,7 @@ def measure_sampled(args, wl, tau, device, graph_steps, min_steps, count_draws=T
     achieved = algo_bytes * steps / sec / 1e9
     st = ocm.stats()
     ocm.close()
-    launches = pkg.sampled_launches_per_step()
+    launches = pkg.sampled_launches_per_step(wl.B, wl.K, wl.V, wl.torch_dtype)
     return {"positions_per_s": wl.B * wl.K * steps / sec, "us_per_step": 1e6 * sec / steps, "steps": steps, "repeats": 7,
             "temperature": T, "achieved_GBs": achieved, "frac": achieved / peak, "peak_source": f"of {peak_kind}",
             "algorithmic_bytes_per_step": algo_bytes, "failed_positions_per_step": mean(failed),

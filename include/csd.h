@@ -302,9 +302,13 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
  *     (n & 3) of counter (n >> 2, row, s, 0).  Group g uses clock g of stream 0; token v of the
  *     winning group uses clock v of stream 1.  The group size and the clock grid are part of
  *     this contract: a caller can reproduce every drawn token from (seed, b, i) and the logits.
- * Draws are made only where a row can need them: for its first failed position, for the later failed
- * positions if that one was rescued, and the bonus draw if every position went through; diag.t_star and
- * diag.bonus are -1 where no draw was made (never at a position the row reaches).
+ * Draws are made only where a row can need them.  A large step makes them in two rounds: first for every
+ * row's first failed position (or its bonus draw if every position went through), then the later failed
+ * positions and the bonus draw of the rows whose first failure was rescued.  A small step (the two logit
+ * tensors under 32 MB; see csd_sampled_set_rounds) makes every failed position's draw and every bonus draw
+ * in one round, because two more launches cost more there than the draws saved.  diag.t_star and diag.bonus
+ * are -1 where no draw was made (never at a position the row reaches); which draws are made beyond those a row
+ * reaches is not part of the contract, their values are.
  * Look-ups see the memory as it is when the call starts; a draft id outside [0,V) fails
  * the test, cannot be rescued and is not recorded.
  *
@@ -312,7 +316,8 @@ csd_status_t csd_verify_static(const void *logits, csd_dtype_t dtype, int B, int
  * temperature > 0; tau as for csd_verify.  workspace: csd_sampled_workspace_bytes bytes,
  * 16-byte aligned, no initialisation needed.  diag: NULL or a HOST struct of optional
  * device arrays.  Six kernel launches (statistics, decision, two rounds of races and
- * finalisation); csd_step_sampled appends the memory update of the recorded pairs in (b,i) order.
+ * finalisation) or four (one round); csd_step_sampled appends the memory update of the recorded
+ * pairs in (b,i) order.
  * Errors as csd_verify; also INVALID_ARG for temperature <= 0 or NaN.  Asynchronous. */
 typedef struct {
     float    *alpha;     /* [B,K]   min(1, p(d)/q(d))                                        */
@@ -326,6 +331,12 @@ typedef struct {
 } csd_sampled_diag_t;
 
 size_t csd_sampled_workspace_bytes(int B, int K, int V, csd_dtype_t dtype);
+/* Expert knob, process-wide: 0 = automatic (above), 1 = always one round of draws, 2 = always two.  Outputs do
+ * not depend on it.  Host function; INVALID_ARG outside 0..2. */
+csd_status_t csd_sampled_set_rounds(int mode);
+/* Kernel launches of one csd_step_sampled call of this shape under the current setting (7 or 5; csd_verify_sampled
+ * makes one fewer); 0 for an unsupported shape.  Host function. */
+int csd_sampled_launches(int B, int K, int V, csd_dtype_t dtype);
 
 csd_status_t csd_verify_sampled(const void *logits, const void *draft_logits, csd_dtype_t dtype,
                                 int B, int K, int V,

@@ -31,6 +31,7 @@ EXPORTS = [
     "csd_ocm_age", "csd_ocm_merge", "csd_ocm_save", "csd_ocm_load", "csd_ocm_set_shared",
     "csd_lmhead_workspace_bytes", "csd_verify_lmhead", "csd_step_lmhead", "csd_lmhead_shape",
     "csd_early_exit_workspace_bytes", "csd_step_early_exit", "csd_lmhead_set_tuning", "csd_lmhead_set_pairing", "csd_lmhead_uses_pairs",
+    "csd_sampled_set_rounds", "csd_sampled_launches",
 ]
 
 
@@ -103,6 +104,8 @@ def lib():
         "csd_step_early_exit": (c_int, step_args[:10] + [c_int] + step_args[10:]),
         "csd_lmhead_set_tuning": (c_int, [c_int, c_int]),
         "csd_lmhead_set_pairing": (c_int, [c_int]),
+        "csd_sampled_set_rounds": (c_int, [c_int]),
+        "csd_sampled_launches": (c_int, [c_int, c_int, c_int, c_int]),
         "csd_lmhead_uses_pairs": (c_int, [c_int, c_int]),
         "csd_ocm_age": (c_int, [c_void_p, c_void_p]),
         "csd_ocm_set_shared": (c_int, [c_void_p, c_int]),
@@ -418,9 +421,14 @@ def csd_step_sampled(logits, draft_logits, draft, r_accept, seed: int, temperatu
     _sampled_call("csd_step_sampled", logits, draft_logits, draft, r_accept, seed, temperature, ocm, tau, buf, stream)
 
 
-def sampled_launches_per_step() -> int:
-    """Kernel launches one csd_step_sampled call makes (for launch counts in reports)."""
-    return 7
+def sampled_launches_per_step(B: int, K: int, V: int, dtype) -> int:
+    """Kernel launches one csd_step_sampled call of this shape makes (for launch counts in reports)."""
+    return int(lib().csd_sampled_launches(B, K, V, CSD_BF16 if dtype == torch.bfloat16 else CSD_F32))
+
+
+def csd_sampled_set_rounds(mode: int = 0):
+    """0 automatic, 1 every draw in one round, 2 two rounds of draws on demand."""
+    _check(lib().csd_sampled_set_rounds(mode), "csd_sampled_set_rounds")
 
 
 class LmheadBuffers(StepBuffers):

@@ -411,7 +411,8 @@ __global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_const
     const int K = p.K;
     const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
     const long long draws = sampled_rows_z(p);
-    // round 1 has one draw per batch row (tiles run over batch rows), round 2 up to K per pending row
+    // round 1 has one draw per batch row (tiles run over batch rows), round 2 up to K per pending row; round 0 is the
+    // single round of a step that makes every draw a row could need at once (all failed positions, every bonus row)
     const long long tiles = (round == 1 ? static_cast<long long>(p.B) : draws) * p.race_nchunks;
     pdl_launch_dependents();
     pdl_wait();
@@ -426,6 +427,7 @@ __global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_const
         const int i = round == 1 ? f0 : static_cast<int>(unit - b * (K + 1));
         const bool bonus = i == K;
         if (round == 2 && !(i > f0 && (bonus || ((failed >> i) & 1u)))) continue;
+        if (round == 0 && !(bonus || ((failed >> i) & 1u))) continue;
         const long long row = b * (K + 1) + i;
         const long long yrow = draws + b * K + i;
         const DrawCoef cf = draw_coef(p, row, bonus, yrow);
@@ -561,7 +563,7 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
     // round 2 all the others of this row.  Lane i < K takes its residual draw t* ~ norm(max(0, p - q)),
     // lane K the bonus draw t ~ p_{gamma+1} -- one code path, so that they run side by side.
     const bool is_bonus = lane == K;
-    const bool have = round == 1 ? lane == f0 : ((lane < K && !passed) || is_bonus);
+    const bool have = round == 1 ? lane == f0 : ((lane < K && !passed) || is_bonus);       // round 0: all of them exist
     int drawn = -1;
     if (have && lane <= K)
         drawn = race_winner<L>(p, row0 + lane, is_bonus, sampled_rows_z(p) + b * K + lane, p.rownorm[row0 + lane].argmax);
@@ -595,7 +597,7 @@ __global__ void __launch_bounds__(128) sampled_finalize_kernel(const __grid_cons
         if (p.diag.cnt) p.diag.cnt[pos] = cnt;
     }
     int bonus_t = K < 32 ? drawn : -1;          // lane K's, if there is a lane K and the draw was made
-    if (K == 32 && lane == 0 && (round == 2 || f0 == K)) bonus_t = race_winner<L>(p, row0 + K, true, 0, p.rownorm[row0 + K].argmax);
+    if (K == 32 && lane == 0 && (round != 1 || f0 == K)) bonus_t = race_winner<L>(p, row0 + K, true, 0, p.rownorm[row0 + K].argmax);
     bonus_t = __shfl_sync(kFull, bonus_t, K < 32 ? K : 0);
     const unsigned int kmask = (K == 32) ? kFull : ((1u << K) - 1u);
     const unsigned int okmask = __ballot_sync(kFull, ok) & kmask;

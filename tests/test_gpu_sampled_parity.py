@@ -16,7 +16,8 @@ import torch
 
 from oracle import csd_sampled_oracle as ORACLE
 from oracle.csd_oracle import bf16_bits_to_f64
-from paper_2604_13634_b200 import CSD_BF16, CSD_F32, Ocm, SampledBuffers, csd_step_sampled, csd_verify_sampled
+from paper_2604_13634_b200 import (CSD_BF16, CSD_F32, Ocm, SampledBuffers, csd_sampled_set_rounds, csd_step_sampled,
+                                   csd_verify_sampled)
 from synth_inputs import WORKLOADS, Synth, logits_bits_numpy
 
 pytestmark = pytest.mark.gpu
@@ -127,8 +128,16 @@ SHAPES = [
 ]
 
 
+@pytest.fixture(autouse=True)
+def _automatic_rounds_afterwards():
+    yield
+    csd_sampled_set_rounds(0)
+
+
+@pytest.mark.parametrize("rounds", [1, 2], ids=["one_round", "two_rounds"])
 @pytest.mark.parametrize("B,K,V,dtype,T", SHAPES)
-def test_elementwise_parity_small(B, K, V, dtype, T):
+def test_elementwise_parity_small(B, K, V, dtype, T, rounds):
+    csd_sampled_set_rounds(rounds)       # every draw at once / draws on demand in two rounds: same outputs
     ocm = Ocm(1024, 1)
     mem = ORACLE.OCM(1024, 1)
     buf = SampledBuffers(B, K, V, dtype)
