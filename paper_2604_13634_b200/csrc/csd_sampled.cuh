@@ -462,6 +462,7 @@ __global__ void __launch_bounds__(256, 4) sampled_race_kernel(const __grid_const
                 // One Philox block serves four consecutive groups, i.e. four consecutive lanes: the
                 // first of them computes it when any of the four has a weight, the others take its words.
                 const unsigned int need = __ballot_sync(kFull, W > 0.0f);
+                if (need == 0u) continue;                    // (the whole warp) nothing here can win: no clocks
                 const int leader = lane & ~3;
                 uint4 rnd = make_uint4(0u, 0u, 0u, 0u);
                 if (lane == leader && ((need >> leader) & 0xfu))
