@@ -16,8 +16,10 @@
 // draws therefore run in two rounds: round 1 races each row's first failed position (or its bonus row if
 // every position passed) and finalises every row that stops there; round 2 races the remaining failed
 // positions and the bonus row of the rows whose first failure was rescued, and finalises those.
+// A step of a few megabytes makes all of them in ONE round instead (round 0: every failed position and every bonus
+// row; B and C once): there two launches cost more than the draws that are saved.
 //
-// Six launches (A, A2, B1, C1, B2, C2) plus the memory's update kernel.  Each is launched programmatically
+// Six launches (A, A2, B1, C1, B2, C2; or four: A, A2, B0, C0) plus the memory's update kernel.  Each is launched programmatically
 // behind the one before and waits for it (griddepcontrol.wait) before it reads or writes anything that
 // others share.  B, C and the update kernel let their successor in before they wait, the decision kernel
 // only when it exits.  Kernel A reads only the step's inputs and writes only the chunk statistics, which
