@@ -133,6 +133,18 @@ def test_plans_of_the_other_entry_points(L):
             assert L.csd_early_exit_workspace_bytes(B, K, V, dt, K - 1) > 0
         else:
             assert L.csd_early_exit_workspace_bytes(B, K, V, dt, 0) == 0
+    # launches of the stochastic step: one round of draws for steps of a few megabytes, two rounds beyond
+    L.csd_sampled_launches.argtypes, L.csd_sampled_launches.restype = [ctypes.c_int] * 4, ctypes.c_int
+    L.csd_sampled_set_rounds.argtypes, L.csd_sampled_set_rounds.restype = [ctypes.c_int], ctypes.c_int
+    assert L.csd_sampled_launches(1, 8, 128256, 1) == 5 and L.csd_sampled_launches(32, 5, 151936, 1) == 7
+    assert L.csd_sampled_launches(1, 4, 32000, 0) == 5 and L.csd_sampled_launches(128, 8, 128256, 0) == 7
+    assert L.csd_sampled_launches(1, 40, 1000, 0) == 0                       # K beyond the limit
+    try:
+        assert L.csd_sampled_set_rounds(1) == 0 and L.csd_sampled_launches(128, 8, 128256, 0) == 5
+        assert L.csd_sampled_set_rounds(2) == 0 and L.csd_sampled_launches(1, 8, 128256, 1) == 7
+        assert L.csd_sampled_set_rounds(3) != 0 and L.csd_sampled_set_rounds(-1) != 0
+    finally:
+        L.csd_sampled_set_rounds(0)
     g, n, t, per = (ctypes.c_int() for _ in range(4))
     L.csd_lmhead_set_pairing.argtypes, L.csd_lmhead_set_pairing.restype = [ctypes.c_int], ctypes.c_int
     assert L.csd_lmhead_set_pairing(3) != 0 and L.csd_lmhead_set_pairing(-1) != 0
