@@ -342,6 +342,7 @@ csd_status_t run_step(const void *logits, csd_dtype_t dtype, int B, int K, int V
     }
     const bool follows = chain_follows(stream, workspace, ocm, accept_len, B, K, V, static_cast<int>(dtype));
     p.chain_by_flag = (may_chain && follows) ? 1 : 0;
+    p.stream_ordered = (g_overlap_steps && may_overlap) ? 0 : 1;
 
     const int eb = elt_bytes(dtype);
     const int per_vec = 16 / eb;

@@ -317,6 +317,8 @@ lmhead_stats_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid
                     }
                 }
             }
+            // every commit aimed at the "empty" barriers has landed before the CTA goes on towards its end
+            for (int k = 0; k < n_stages && !*give_up; ++k, ++it) mbar_wait(empty_bar(it % n_stages), ((it / n_stages) & 1) ^ 1, give_up);
         }
     } else if (warp == 1) {
         // ---- MMA issuer ----

@@ -91,6 +91,7 @@ struct StepParams {
     int chunk_units;         // units per chunk
     long long total_units;   // T = R * U
     int narrow;              // 1 if the span arithmetic fits 32 bits
+    int stream_ordered;      // 1 for a plain launch: everything before it on the stream is complete when it starts
     int chain_by_flag;       // 1 if the host vouches that the previous step launch on the stream used this
                              // very workspace, memory and outputs: its completion word is then enough
     // ---- a launch that covers only some positions of some batch rows (the two phases of the early-exit step) ----
@@ -593,8 +594,9 @@ __device__ __forceinline__ void prefetch_l2(const void *ptr) { asm volatile("pre
 
 template <typename L>
 __device__ int finalize_batch_row(const StepParams &p, const Extent &e, unsigned int seq, int b, int lane, RowScratch &rs,
-                                  const BlockState &bs)
+                                  const BlockState &bs, int &hint_reg)
 {
+    hint_reg = kHintNone;
     const int K = p.K;
     const RowPlace at_b = place_of(p, b);
 
@@ -675,6 +677,7 @@ __device__ int finalize_batch_row(const StepParams &p, const Extent &e, unsigned
                 if (slot >= 0 && cnt > room) hint |= kHintCareful;
             }
             __stcg(sc.slot_hint + (size_t)b * K + lane, hint);
+            hint_reg = hint;
         }
     } else if (p.K_total != 0 && p.pos0 == 0 && lane < p.K_total) {
         // first phase of a step in two phases: the positions it does not cover start out as "not reached"
@@ -700,6 +703,23 @@ __device__ int finalize_batch_row(const StepParams &p, const Extent &e, unsigned
     }
     __syncwarp();
     return regime;
+}
+
+// One recorded pair's add, from the slot its look-up left (every lane of the warp calls this).
+__device__ __forceinline__ void apply_hint(const StepParams &p, int hint)
+{
+    if (hint >= 0) {
+        const unsigned long long s = static_cast<unsigned long long>(hint & ~kHintCareful);
+        if (CSD_INDEX_OK(s <= p.ocm.mask, p.ocm.stats, 4u)) {
+            if (hint & kHintCareful)
+                ocm_add(p.ocm, s, 1u);
+            else
+                atomicAdd(&p.ocm.slots[s].count, 1u);
+        }
+    }
+    const unsigned int dropped = __popc(__ballot_sync(kFull, hint == kHintAbsent));
+    if ((threadIdx.x & 31) == 0 && dropped) atomicAdd(&p.ocm.stats->n_dropped, static_cast<unsigned long long>(dropped));
+    __syncwarp();
 }
 
 // S6, second half, by the warp that finalised the last batch row: every look-up of the
@@ -754,7 +774,7 @@ __device__ void publish_parts(const StepParams &p, const Extent &e, BlockState &
     // complete the scratch can be written right away; otherwise wait for it (launches
     // complete in order).
     const unsigned int need = seq - (kScratchRing - 1u);
-    if (static_cast<int>(ld_acquire(p.completed) - need) < 0) wait_completed(p, need);
+    if (!p.stream_ordered && static_cast<int>(ld_acquire(p.completed) - need) < 0) wait_completed(p, need);
     int my_b = -1;
     if (lane < nseg) {
         const int row = first_row + lane;
@@ -789,13 +809,19 @@ __device__ void finalize_and_update(const StepParams &p, const Extent &e, unsign
                                     CanonScratch &canon, const BlockState &bs)
 {
     const ScratchCopy sc = scratch_of(p, seq);
-    const int regime = finalize_batch_row<L>(p, e, seq, b, lane, rs, bs);   // the same for every row of a launch
+    int own_hint;
+    const int regime = finalize_batch_row<L>(p, e, seq, b, lane, rs, bs, own_hint);   // the same for every row of a launch
     bool last = false;
     if (lane == 0) sc.b_ticket[b] = 0u;               // ready for this copy's next launch
     __syncwarp();                                     // each lane's outputs and hints of this row before the row's ticket,
-    if (lane == 0) last = atom_add_acq_rel(sc.g_ticket, 1u) == static_cast<unsigned int>(e.B) - 1u;   // whose add releases them
-    last = __shfl_sync(kFull, last, 0);
-    if (!last) return;
+    // a launch of ONE batch row (the paper's own setting, batch 1) has no other row to wait for: no ticket, and the
+    // slot hints go from this warp's look-ups to its adds in registers
+    const bool lone_row = e.B == 1 && p.B == 1;
+    if (!lone_row) {
+        if (lane == 0) last = atom_add_acq_rel(sc.g_ticket, 1u) == static_cast<unsigned int>(e.B) - 1u;   // whose add releases them
+        last = __shfl_sync(kFull, last, 0);
+        if (!last) return;
+    }
 
     // ---- every batch row is final (lane 0 has acquired what their warps released): S6 ----
     __syncwarp();
@@ -805,7 +831,12 @@ __device__ void finalize_and_update(const StepParams &p, const Extent &e, unsign
     const bool keys_settled = !p.do_update || regime != kRegimeTransition;
     unsigned long long nk = 0;
     if (lane == 0 && keys_settled) nk = atomicAdd(&st->n_keys, 0ull);   // in flight next to the hint loads
-    if (p.do_update) apply_step_update(p, sc, lane, canon, regime);
+    if (p.do_update) {
+        if (lone_row && regime != kRegimeTransition)
+            apply_hint(p, own_hint);
+        else
+            apply_step_update(p, sc, lane, canon, regime);
+    }
     if (p.K_total != 0 && p.alive_out) {
         // the batch rows that accepted every position of this launch go on to the next phase: their list, ascending
         int n_alive = 0;
