@@ -311,6 +311,21 @@ def test_contention_fills_the_table():
     assert st["n_keys"] == 256 and st["n_dropped"] > 0
 
 
+@pytest.mark.parametrize("overlap", [False, True], ids=["alone", "overlap"])
+def test_one_batch_row_fills_the_table(overlap):
+    """One batch row (the paper's own setting): the launch's only finalising warp takes no global ticket and adds
+    from the slots its own look-ups left.  A table far too small takes the run through all three update regimes;
+    the memory, its key count and every step match the oracle."""
+    from paper_2604_13634_b200 import csd_set_overlap
+    wl = dataclasses.replace(WORKLOADS["ocm_contention"], B=1, K=8, V=32768, ocm_slots=128)
+    try:
+        csd_set_overlap(overlap)
+        tot, near, st = lockstep(wl, steps=400, tau=0.3, check_every=1, diag=False)
+    finally:
+        csd_set_overlap(False)
+    assert st["n_keys"] == 64 and st["n_dropped"] > 0 and tot["resc"] > 0
+
+
 # ---------------------------------------------------------------------------------------
 # the memory on its own
 # ---------------------------------------------------------------------------------------
