@@ -27,8 +27,9 @@
  *     table) set sticky flags / counters readable with csd_ocm_stats; the device
  *     never traps.  Within a launch no block waits for another (arrival counters
  *     only); the one exception are the two blocks of a thread-block cluster in the
- *     LM-head pair kernel, which the hardware schedules together and whose waits on
- *     each other are bounded like every other wait.  With csd_set_overlap on, the warps that finalise a batch row wait for
+ *     LM-head pair kernel, which the hardware schedules together: their barrier
+ *     waits on each other are bounded in time, and every path of both blocks reaches
+ *     the two cluster barriers they meet at.  With csd_set_overlap on, the warps that finalise a batch row wait for
  *     the PREVIOUS launch on the stream: a bounded poll (2^14 loads) of a completion
  *     word, then the hardware's wait for that grid to retire, which always ends.
  *   - Determinism: for fixed (B,K,V,dtype) every output, including the sums s,
