@@ -153,6 +153,22 @@ __device__ __forceinline__ RowNorm fold_row_norm(const SampledParams &p, long lo
     return n;
 }
 
+// The same for two rows at once (a position's target and draft row): both rows' loads are in flight together.
+__device__ __forceinline__ void fold_row_norm2(const SampledParams &p, long long row_a, long long row_b, int lane, RowNorm &na, RowNorm &nb)
+{
+    Partial a = partial_identity(), b = partial_identity();
+    for (int c = lane; c < p.nchunks; c += 32) {
+        const Partial xa = ld_partial_cg(p.stat_part + row_a * p.nchunks + c);
+        const Partial xb = ld_partial_cg(p.stat_part + row_b * p.nchunks + c);
+        a = (c == lane) ? xa : combine(a, xa);
+        b = (c == lane) ? xb : combine(b, xb);
+    }
+    a = butterfly_fold(a, 32, p.l2e_T);
+    b = butterfly_fold(b, 32, p.l2e_T);
+    na.m = a.m; na.lse2 = a.c + log2f(a.s); na.argmax = a.idx; na.zcut = -INFINITY;
+    nb.m = b.m; nb.lse2 = b.c + log2f(b.s); nb.argmax = b.idx; nb.zcut = -INFINITY;
+}
+
 // The logit below which p(v) <= race_skip_bound(w0): (z - m) * l2e_T - (lse2 - m * l2e_T) <= log2(bound),
 // lowered by 1e-3 so that rounding can only make the cut more cautious.
 __device__ __forceinline__ float race_logit_cut(const RowNorm &n, float w0, float l2e_T)
@@ -188,9 +204,13 @@ __global__ void __launch_bounds__(128) sampled_decide_kernel(const __grid_consta
             yd = L::load_elem(sampled_row_ptr<E>(p, yrow), d);
         }
     }
-    RowNorm np_ = fold_row_norm(p, j, lane);
-    RowNorm nq = np_;
-    if (i < K) nq = fold_row_norm(p, yrow, lane);
+    RowNorm np_, nq;
+    if (i < K) {
+        fold_row_norm2(p, j, yrow, lane, np_, nq);
+    } else {
+        np_ = fold_row_norm(p, j, lane);
+        nq = np_;
+    }
     if (lane != 0) return;
     p.race_best[j] = 0ull;
     if (!(np_.lse2 == np_.lse2) || np_.lse2 == INFINITY || np_.m == -INFINITY) atomicOr(&p.ocm.stats->flags, CSD_FLAG_NAN_LOGIT);
